@@ -1,0 +1,137 @@
+"""ctypes front end of the CPU oracle (``owl_oracle.c``).
+
+TEST INFRASTRUCTURE ONLY: imported by the tests, the smoke check and the
+benchmark's CPU-baseline leg.  The CUDA library and its Python binding never
+import this package, and this package never imports them.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from typing import Optional, Tuple
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "owl_oracle.c")
+_LIB = os.path.join(_HERE, "liboracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile ``owl_oracle.c`` with gcc (-O2, OpenMP) into ``liboracle.so`` beside it."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + f".tmp{os.getpid()}"
+        subprocess.check_call(["gcc", "-O2", "-fopenmp", "-fPIC", "-shared", "-std=c11", "-o", tmp, _SRC, "-lm"])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        build()
+        lib = ctypes.CDLL(_LIB)
+        i32p = ctypes.POINTER(ctypes.c_int32)
+        u16p = ctypes.POINTER(ctypes.c_uint16)
+        f64p = ctypes.POINTER(ctypes.c_double)
+        lib.owl_oracle_attn.restype = ctypes.c_int
+        lib.owl_oracle_attn.argtypes = [ctypes.c_int] * 7 + [ctypes.c_double, u16p, u16p, u16p, i32p, i32p, i32p, i32p,
+                                                              ctypes.c_int64, i32p, i32p, f64p, f64p]
+        lib.owl_oracle_argmax.restype = None
+        lib.owl_oracle_argmax.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.c_int64, ctypes.c_int64, i32p]
+        lib.owl_oracle_accept.restype = ctypes.c_int
+        lib.owl_oracle_accept.argtypes = [ctypes.c_int, i32p, i32p, i32p, i32p, ctypes.c_int, i32p, i32p, i32p]
+        lib.owl_oracle_num_threads.restype = ctypes.c_int
+        _lib = lib
+    return _lib
+
+
+def num_threads() -> int:
+    return int(_load().owl_oracle_num_threads())
+
+
+def _p(a: Optional[np.ndarray], ct):
+    if a is None:
+        return None
+    return a.ctypes.data_as(ctypes.POINTER(ct))
+
+
+def _c(a, dtype) -> np.ndarray:
+    a = np.ascontiguousarray(a, dtype=dtype)
+    return a
+
+
+def verify_attn(q, k_cache, v_cache, block_table, ctx_lens, node_offsets, tree_parent, sm_scale: float,
+                rows: Optional[Tuple[np.ndarray, np.ndarray]] = None) -> Tuple[np.ndarray, np.ndarray]:
+    """Tree-masked attention in fp64.
+
+    q uint16 [N,Hq,D] (bf16 bits); k_cache/v_cache uint16 [pages,Hkv,page,D]; block_table int32
+    [B,max_pages]; ctx_lens int32 [B]; node_offsets int32 [B+1]; tree_parent int32 [N].
+    Returns (out, lse): without ``rows`` shapes [N,Hq,D] and [N,Hq]; with
+    ``rows=(nodes, heads)`` shapes [R,D] and [R] for the listed (packed node, query head) pairs.
+    """
+    lib = _load()
+    q = _c(q, np.uint16); k_cache = _c(k_cache, np.uint16); v_cache = _c(v_cache, np.uint16)
+    block_table = _c(block_table, np.int32); ctx_lens = _c(ctx_lens, np.int32)
+    node_offsets = _c(node_offsets, np.int32); tree_parent = _c(tree_parent, np.int32)
+    N, Hq, D = q.shape
+    num_pages, Hkv, page, D2 = k_cache.shape
+    assert D2 == D and v_cache.shape == k_cache.shape
+    B = ctx_lens.shape[0]
+    assert block_table.shape[0] == B and node_offsets.shape[0] == B + 1 and int(node_offsets[-1]) == N
+    if rows is None:
+        n_rows = N * Hq
+        rn = rh = None
+        out = np.empty((N, Hq, D), dtype=np.float64)
+        lse = np.empty((N, Hq), dtype=np.float64)
+    else:
+        rn = _c(rows[0], np.int32); rh = _c(rows[1], np.int32)
+        n_rows = rn.shape[0]
+        assert rh.shape[0] == n_rows
+        out = np.empty((n_rows, D), dtype=np.float64)
+        lse = np.empty((n_rows,), dtype=np.float64)
+    rc = lib.owl_oracle_attn(B, Hq, Hkv, D, page, block_table.shape[1], num_pages, float(sm_scale),
+                             _p(q, ctypes.c_uint16), _p(k_cache, ctypes.c_uint16), _p(v_cache, ctypes.c_uint16),
+                             _p(block_table, ctypes.c_int32), _p(ctx_lens, ctypes.c_int32),
+                             _p(node_offsets, ctypes.c_int32), _p(tree_parent, ctypes.c_int32),
+                             n_rows, _p(rn, ctypes.c_int32), _p(rh, ctypes.c_int32),
+                             _p(out, ctypes.c_double), _p(lse, ctypes.c_double))
+    if rc != 0:
+        raise ValueError(f"owl_oracle_attn failed with code {rc}")
+    return out, lse
+
+
+def row_argmax(logits) -> np.ndarray:
+    """Lowest index of the maximum of every row of fp32 ``logits`` [N,V]."""
+    lib = _load()
+    logits = _c(logits, np.float32)
+    N, V = logits.shape
+    am = np.empty(N, dtype=np.int32)
+    lib.owl_oracle_argmax(_p(logits, ctypes.c_float), N, V, _p(am, ctypes.c_int32))
+    return am
+
+
+def accept_from_argmax(node_offsets, tree_parent, draft_tokens, am, path_stride: int = 64):
+    """Greedy tree acceptance given per-node arg-max tokens. Returns (accept_len, accept_path, bonus)."""
+    lib = _load()
+    node_offsets = _c(node_offsets, np.int32); tree_parent = _c(tree_parent, np.int32)
+    draft_tokens = _c(draft_tokens, np.int32); am = _c(am, np.int32)
+    B = node_offsets.shape[0] - 1
+    alen = np.empty(B, dtype=np.int32)
+    path = np.empty((B, path_stride), dtype=np.int32)
+    bonus = np.empty(B, dtype=np.int32)
+    rc = lib.owl_oracle_accept(B, _p(node_offsets, ctypes.c_int32), _p(tree_parent, ctypes.c_int32),
+                               _p(draft_tokens, ctypes.c_int32), _p(am, ctypes.c_int32), path_stride,
+                               _p(alen, ctypes.c_int32), _p(path, ctypes.c_int32), _p(bonus, ctypes.c_int32))
+    if rc != 0:
+        raise ValueError(f"owl_oracle_accept failed with code {rc}")
+    return alen, path, bonus
+
+
+def tree_accept(logits, draft_tokens, node_offsets, tree_parent, path_stride: int = 64):
+    """Row arg-max followed by the acceptance walk. Returns (accept_len, accept_path, bonus, argmax)."""
+    am = row_argmax(logits)
+    alen, path, bonus = accept_from_argmax(node_offsets, tree_parent, draft_tokens, am, path_stride)
+    return alen, path, bonus, am

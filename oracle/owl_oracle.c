@@ -1,0 +1,235 @@
+/*
+ * CPU oracle for the verify step of long-context speculative decoding
+ * (tree-masked attention of drafted tokens against a KV cache + greedy acceptance).
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, plain statement of what the
+ * step computes; it shares no code with the CUDA library and the product path
+ * never calls it.  Only the tests, the smoke check and the benchmark's
+ * CPU-baseline leg load it.
+ *
+ * What it follows in the paper:
+ *  - "Decode Stage" paragraph (Section 3.2.2): the drafted tree is verified in one
+ *    pass in which every node (including an appended [SPEC] leaf) attends to the
+ *    context plus exactly the nodes on its own root path - the worked example lists
+ *    the paths (t_{N+1}), (t_{N+1}, t_{N+2}), (t_{N+1}, t_{N+2'}).
+ *  - Introduction / Related Work: the target model verifies all drafted tokens in
+ *    parallel and the decoding algorithm accepts the tokens that keep the output
+ *    distribution; "acceptance length" (caption of Figure 1) is the number of
+ *    tokens accepted per verification step.  Under greedy decoding a drafted token
+ *    keeps the distribution iff it equals the target's own arg-max continuation of
+ *    its parent.
+ *  - Non-tree verification (Section 3.2.3, Algorithm 1 line 8) is the same pass with
+ *    a chain-shaped tree.
+ *
+ * Parity pins (tests, CPU only): brute-force dense-mask softmax in numpy fp64,
+ * single-node == decode attention and chain == causal attention against a library
+ * SDPA in fp64, the paper's worked mask example, softmax invariants, hand-worked
+ * acceptance cases, losslessness on a toy model, a closed-form expectation, and
+ * the acceptance-length bounds the paper states.  No function here is unpinned.
+ *
+ * Arithmetic: bf16 inputs are decoded exactly to double; dot products, the
+ * two-pass softmax and the weighted sum run in double; nothing is blocked, fused
+ * or reordered.  Outputs are double (not rounded to bf16).
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+#define ORACLE_OK 0
+#define ORACLE_BAD_ARG (-1)
+#define ORACLE_BAD_TREE (-2)
+#define ORACLE_BAD_PAGE (-3)
+
+int owl_oracle_num_threads(void) {
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+static double bf16_to_double(uint16_t h) {
+    uint32_t u = ((uint32_t)h) << 16;
+    float f;
+    memcpy(&f, &u, sizeof f);
+    return (double)f;
+}
+
+/* Sequence that owns packed node `n` (node_offsets has B+1 entries). */
+static int seq_of_node(const int32_t* node_offsets, int B, int n) {
+    for (int b = 0; b < B; ++b)
+        if (n >= node_offsets[b] && n < node_offsets[b + 1]) return b;
+    return -1;
+}
+
+/* Pointer to the D values of token `pos` of sequence b, KV head h, in the paged cache
+ * laid out [page][kv_head][slot][d]. */
+static const uint16_t* kv_row(const uint16_t* cache, const int32_t* block_table, int b,
+                              int max_pages_per_seq, int num_pages, int Hkv, int page_size, int D,
+                              int h, int64_t pos) {
+    int64_t lp = pos / page_size, slot = pos % page_size;
+    int32_t page = block_table[(int64_t)b * max_pages_per_seq + lp];
+    if (page < 0 || page >= num_pages) return NULL;
+    return cache + (((int64_t)page * Hkv + h) * page_size + slot) * D;
+}
+
+/* Check the node order the interface requires: node 0 is the only root, parent[i] < i. */
+static int tree_ok(const int32_t* parent, int n) {
+    if (n < 1 || parent[0] != -1) return 0;
+    for (int i = 1; i < n; ++i)
+        if (parent[i] < 0 || parent[i] >= i) return 0;
+    return 1;
+}
+
+/*
+ * Tree-masked attention, one (packed node, query head) row at a time.
+ *
+ * Row (n, hq): let b be the sequence of node n, i its local index, L = ctx_lens[b].
+ * Visible keys = {0..L-1} (the whole committed context) plus L+j for every j on the
+ * root path of i, found by following parent pointers from i (i itself included).
+ *   s_k = sm_scale * <q, K_k>;  m = max s_k;  Z = sum exp(s_k - m)
+ *   lse = m + ln Z;  out = sum exp(s_k - m) V_k / Z
+ *
+ * rows: if row_node == NULL every (n, hq) pair is computed in order n*Hq + hq and
+ * n_rows must be N*Hq; otherwise rows r = (row_node[r], row_head[r]).
+ * out is [n_rows, D] doubles, lse [n_rows] doubles.
+ */
+int owl_oracle_attn(int B, int Hq, int Hkv, int D, int page_size, int max_pages_per_seq,
+                    int num_pages, double sm_scale, const uint16_t* q, const uint16_t* k_cache,
+                    const uint16_t* v_cache, const int32_t* block_table, const int32_t* ctx_lens,
+                    const int32_t* node_offsets, const int32_t* tree_parent, int64_t n_rows,
+                    const int32_t* row_node, const int32_t* row_head, double* out, double* lse) {
+    if (B < 1 || Hq < 1 || Hkv < 1 || Hq % Hkv != 0 || D < 1 || page_size < 1) return ORACLE_BAD_ARG;
+    const int G = Hq / Hkv;
+    const int N = node_offsets[B];
+    if (row_node == NULL && n_rows != (int64_t)N * Hq) return ORACLE_BAD_ARG;
+    for (int b = 0; b < B; ++b)
+        if (!tree_ok(tree_parent + node_offsets[b], node_offsets[b + 1] - node_offsets[b]))
+            return ORACLE_BAD_TREE;
+
+    int status = ORACLE_OK;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t r = 0; r < n_rows; ++r) {
+        const int n = row_node ? row_node[r] : (int)(r / Hq);
+        const int hq = row_head ? row_head[r] : (int)(r % Hq);
+        const int b = seq_of_node(node_offsets, B, n);
+        if (b < 0 || hq < 0 || hq >= Hq) {
+#pragma omp atomic write
+            status = ORACLE_BAD_ARG;
+            continue;
+        }
+        const int base = node_offsets[b];
+        const int nb = node_offsets[b + 1] - base;
+        const int i = n - base;
+        const int64_t L = ctx_lens[b];
+        const int h = hq / G;
+        const int32_t* parent = tree_parent + base;
+
+        /* visible keys: prefix, then the root path of i by literal pointer chasing */
+        int64_t nvis = 0;
+        int64_t* vis = (int64_t*)malloc((size_t)(L + nb) * sizeof(int64_t));
+        double* s = (double*)malloc((size_t)(L + nb) * sizeof(double));
+        for (int64_t k = 0; k < L; ++k) vis[nvis++] = k;
+        {
+            char* on_path = (char*)calloc((size_t)nb, 1);
+            for (int j = i; j >= 0; j = parent[j]) on_path[j] = 1;
+            for (int j = 0; j < nb; ++j)
+                if (on_path[j]) vis[nvis++] = L + j;
+            free(on_path);
+        }
+
+        const uint16_t* qrow = q + ((int64_t)n * Hq + hq) * D;
+        int bad = 0;
+        double m = -INFINITY;
+        for (int64_t t = 0; t < nvis; ++t) {
+            const uint16_t* krow = kv_row(k_cache, block_table, b, max_pages_per_seq, num_pages,
+                                          Hkv, page_size, D, h, vis[t]);
+            if (!krow) { bad = 1; break; }
+            double acc = 0.0;
+            for (int d = 0; d < D; ++d) acc += bf16_to_double(qrow[d]) * bf16_to_double(krow[d]);
+            s[t] = sm_scale * acc;
+            if (s[t] > m) m = s[t];
+        }
+        if (bad) {
+#pragma omp atomic write
+            status = ORACLE_BAD_PAGE;
+            free(vis); free(s);
+            continue;
+        }
+        double Z = 0.0;
+        for (int64_t t = 0; t < nvis; ++t) Z += exp(s[t] - m);
+        double* o = out + r * D;
+        for (int d = 0; d < D; ++d) o[d] = 0.0;
+        for (int64_t t = 0; t < nvis; ++t) {
+            const uint16_t* vrow = kv_row(v_cache, block_table, b, max_pages_per_seq, num_pages,
+                                          Hkv, page_size, D, h, vis[t]);
+            const double p = exp(s[t] - m);
+            for (int d = 0; d < D; ++d) o[d] += p * bf16_to_double(vrow[d]);
+        }
+        for (int d = 0; d < D; ++d) o[d] /= Z;
+        lse[r] = m + log(Z);
+        free(vis); free(s);
+    }
+    return status;
+}
+
+/*
+ * Row arg-max over the vocabulary: the smallest index attaining the row maximum.
+ * Scalar scan with a strict '>' so the first maximum wins; NaN is read as -inf
+ * (so +0.0 and -0.0 tie and an all-NaN row gives 0).
+ */
+void owl_oracle_argmax(const float* logits, int64_t N, int64_t V, int32_t* am) {
+#pragma omp parallel for schedule(static)
+    for (int64_t n = 0; n < N; ++n) {
+        const float* row = logits + n * V;
+        float best = isnan(row[0]) ? -INFINITY : row[0];
+        int32_t bi = 0;
+        for (int64_t j = 1; j < V; ++j) {
+            float x = isnan(row[j]) ? -INFINITY : row[j];
+            if (x > best) { best = x; bi = (int32_t)j; }
+        }
+        am[n] = bi;
+    }
+}
+
+/*
+ * Greedy tree acceptance.  The root is the target's own, already chosen token and
+ * is always accepted.  A non-root node c is accepted iff every edge (p -> c') on
+ * its root path has a drafted token draft[c'] >= 0 equal to am[p], the target's
+ * arg-max continuation of p.  The winner is the accepted node of greatest depth
+ * (lowest index among equals); accept_len = depth + 1 (nodes on the path, root
+ * included), accept_path lists the path root -> winner padded with -1, and
+ * bonus_token = am[winner] is the target's next token after the accepted path.
+ */
+int owl_oracle_accept(int B, const int32_t* node_offsets, const int32_t* tree_parent,
+                      const int32_t* draft_tokens, const int32_t* am, int path_stride,
+                      int32_t* accept_len, int32_t* accept_path, int32_t* bonus_token) {
+    for (int b = 0; b < B; ++b) {
+        const int base = node_offsets[b];
+        const int nb = node_offsets[b + 1] - base;
+        const int32_t* parent = tree_parent + base;
+        if (!tree_ok(parent, nb)) return ORACLE_BAD_TREE;
+        int win = 0, win_depth = 0;
+        for (int i = 0; i < nb; ++i) {
+            int ok = 1, depth = 0;
+            for (int c = i; parent[c] >= 0; c = parent[c]) {
+                const int p = parent[c];
+                if (!(draft_tokens[base + c] >= 0 && draft_tokens[base + c] == am[base + p])) ok = 0;
+                ++depth;
+            }
+            if (ok && depth > win_depth) { win = i; win_depth = depth; }
+        }
+        if (win_depth + 1 > path_stride) return ORACLE_BAD_ARG;
+        accept_len[b] = win_depth + 1;
+        for (int k = 0; k < path_stride; ++k) accept_path[(int64_t)b * path_stride + k] = -1;
+        int k = win_depth;
+        for (int c = win; c >= 0; c = parent[c]) accept_path[(int64_t)b * path_stride + k--] = c;
+        bonus_token[b] = am[base + win];
+    }
+    return ORACLE_OK;
+}
