@@ -1,0 +1,166 @@
+/*
+ * libowlverify - the target model's verification step of long-context speculative
+ * decoding (OWL / HOWL), for one NVIDIA B200 (sm_100a).
+ *
+ * Two operations, as the paper states the problem:
+ *   owl_verify_attn  - every drafted token (a chain, or a token tree with [SPEC]
+ *                      leaves) attends to the whole cached context plus the nodes on
+ *                      its own root path, all nodes in one pass (Introduction;
+ *                      Section 3.2.2 "Decode Stage": attention mask manipulated so that
+ *                      each appended token follows exactly one tree path; Section 3.2.3 /
+ *                      Algorithm 1: NonTreeVerify is the same pass on a chain).
+ *   owl_tree_accept  - the decoding algorithm then accepts the drafted tokens that keep
+ *                      the target's output distribution (Introduction); under greedy
+ *                      decoding: per-node arg-max over the vocabulary, the longest root
+ *                      path whose drafted tokens equal their parent's arg-max, and the
+ *                      arg-max of the last accepted node as the next token.  The number
+ *                      of tokens accepted per step is the paper's "acceptance length"
+ *                      (Figure 1 caption), at least 1 and at most tree depth + 1
+ *                      (Appendix "Inference Details": depth 8, maximum 9).
+ *
+ * General rules of this interface
+ *  - Plain C ABI.  Unless an argument says "host", every tensor pointer is a DEVICE
+ *    pointer on the context's device, owned by the caller; the library reads inputs,
+ *    writes outputs, and neither frees nor keeps any of them after the call's work
+ *    has run on the stream.
+ *  - Calls enqueue work on the caller's stream (a cudaStream_t passed as void*;
+ *    NULL = the default stream) and return without synchronising the host, except
+ *    owl_get_status and the *_host convenience call, which synchronise that stream.
+ *  - Return value: OWL_OK or a negative owl_status.  Errors that can be seen from the
+ *    arguments alone are returned immediately and launch nothing.  Errors that need
+ *    device data (a malformed tree, a page id out of range) are recorded in a device
+ *    status word read by owl_get_status; the kernels then leave the outputs of the
+ *    offending sequence unwritten and finish normally.
+ *  - One owl_ctx serves one stream at a time (its workspace is reused by every call).
+ *
+ * Layouts (B sequences, N = total drafted nodes packed sequence after sequence,
+ * Hq query heads, Hkv key/value heads, G = Hq/Hkv, D = head_dim = 128):
+ *  - q, out       bf16 [N, Hq, D]
+ *  - lse          fp32 [N, Hq]   natural log of sum_k exp(sm_scale * q.k) over visible keys
+ *  - k_cache/v_cache  bf16 [num_pages, Hkv, page_size, D]; one (page, head) block is
+ *                 page_size*D contiguous elements.  A contiguous cache is the same
+ *                 layout with an identity block_table.
+ *  - block_table  int32 [B, max_pages_per_seq]: physical page of each logical page
+ *  - ctx_lens     int32 [B]: committed context length L_b.  The K/V of drafted node i
+ *                 of sequence b are already stored at logical position L_b + i, so the
+ *                 cache holds L_b + n_b valid positions.  Q and K arrive with their
+ *                 rotary position (the paper's position-id manipulation) applied.
+ *                 Cache slots of a sequence's last page beyond L_b + n_b must hold
+ *                 finite values (they are multiplied by an exact zero weight).
+ *  - node_offsets int32 [B+1], packed offsets of each sequence's nodes; NULL means
+ *                 every sequence has N/B nodes.
+ *  - tree_parent  int32 [N]: parent of each node as an index local to its sequence,
+ *                 -1 for the root.  Node 0 of a sequence is its only root and
+ *                 parent[i] < i (topological / BFS order).  The root is the target's own
+ *                 already chosen token t_{N+1}.
+ */
+#ifndef OWLVERIFY_H_
+#define OWLVERIFY_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum owl_status {
+    OWL_OK = 0,
+    OWL_ERR_INVALID_ARG = -1, /* null pointer, batch < 1, total_nodes < 1, Hq % Hkv != 0, ...       */
+    OWL_ERR_UNSUPPORTED = -2, /* head_dim != 128, max_nodes > 64, G*max_nodes > 256, page size, ... */
+    OWL_ERR_CUDA = -3,        /* a CUDA call failed; see owl_last_error                             */
+    OWL_ERR_BAD_TREE = -4,    /* device-detected: parent[i] >= i, parent < -1, node 0 not the root  */
+    OWL_ERR_BAD_PAGE = -5,    /* device-detected: block_table entry outside [0, num_pages)          */
+    OWL_ERR_TIMEOUT = -6,     /* device-detected: a bounded wait inside a kernel expired            */
+    OWL_ERR_TOO_LARGE = -7    /* dims exceed what the context was created for                       */
+} owl_status;
+
+typedef struct owl_ctx owl_ctx; /* opaque: device workspace (split partials, status word) */
+
+typedef struct owl_dims {
+    int32_t batch;             /* B >= 1                                                        */
+    int32_t total_nodes;       /* N = sum of n_b >= B                                           */
+    int32_t max_nodes;         /* T = max n_b, 1..64 (the paper's trees have 60 nodes)          */
+    int32_t num_q_heads;       /* Hq                                                            */
+    int32_t num_kv_heads;      /* Hkv, divides Hq; G*T <= 256                                   */
+    int32_t head_dim;          /* must be 128                                                   */
+    int32_t page_size;         /* tokens per page: 16 (also 32, 64, 128)                        */
+    int32_t max_pages_per_seq; /* row stride of block_table                                     */
+    int32_t num_pages;         /* pages in k_cache / v_cache; block_table entries are checked   */
+    int32_t vocab;             /* V (owl_tree_accept only; may be 0 for attention-only use)     */
+    int32_t path_stride;       /* row stride of accept_path, >= deepest path + 1 (64 always is) */
+    float sm_scale;            /* multiplies q.k before the softmax; always explicit            */
+} owl_dims;
+
+/* Create a context on `device` with workspace for any call whose dims do not exceed
+ * `max_dims` (batch, total_nodes, max_nodes, heads).  Allocates device memory once;
+ * later calls allocate nothing.  Host-synchronous. */
+int owl_create(owl_ctx** ctx, int device, const owl_dims* max_dims);
+
+/* Free the context's device memory.  The caller must have synchronised every stream
+ * that used it. */
+int owl_destroy(owl_ctx* ctx);
+
+/*
+ * Tree-masked attention of the drafted nodes against the paged KV cache
+ * (Section 3.2.2 "Decode Stage"; Algorithm 1, NonTreeVerify / OurTreeVerify).
+ *
+ * For packed node n = node_offsets[b] + i and query head hq (KV head hq / G):
+ *   visible keys = {0 .. L_b-1}  union  {L_b + j : j on the root path of i, i included}
+ *   out[n,hq,:]  = sum_k softmax_k(sm_scale * q[n,hq].K_k) * V_k   (rounded to bf16)
+ *   lse[n,hq]    = ln sum_k exp(sm_scale * q[n,hq].K_k)
+ * Computed by split-KV kernels: per KV chunk an online-softmax pass on the tensor
+ * cores producing fp32 partials in the context's workspace, then an LSE merge.
+ * Asynchronous on `stream`.  `lse` may be NULL.
+ */
+int owl_verify_attn(owl_ctx* ctx, const owl_dims* dims, const void* q, const void* k_cache,
+                    const void* v_cache, const int32_t* block_table, const int32_t* ctx_lens,
+                    const int32_t* node_offsets, const int32_t* tree_parent, void* out, float* lse,
+                    void* stream);
+
+/*
+ * Greedy tree acceptance (Introduction: accepted tokens keep the target's output
+ * distribution; Figure 1 caption: acceptance length; Section 3.2.2: paths start at the
+ * root t_{N+1}, [SPEC] leaves are never candidate tokens).
+ *
+ *   am[n]      = lowest index attaining the maximum of logits[n, :] (NaN reads as -inf)
+ *   ok(root)   = true;  ok(i) = ok(parent(i)) and draft_tokens[i] >= 0
+ *                              and draft_tokens[i] == am[parent(i)]
+ *   winner     = ok node of greatest depth, lowest index among equals
+ *   accept_len[b]    = depth(winner) + 1            (nodes on the path, root included)
+ *   accept_path[b,:] = local node indices root..winner, then -1 up to path_stride
+ *   bonus_token[b]   = am[winner]                   (the target's next token)
+ *
+ * logits fp32 [N, V] row-major (row n = packed node n); draft_tokens int32 [N]
+ * (the root's entry is ignored; a negative entry, e.g. a [SPEC] leaf, never matches);
+ * node_argmax optional int32 [N] (NULL to skip) receives am.  Asynchronous on `stream`.
+ */
+int owl_tree_accept(owl_ctx* ctx, const owl_dims* dims, const float* logits,
+                    const int32_t* draft_tokens, const int32_t* node_offsets,
+                    const int32_t* tree_parent, int32_t* accept_len, int32_t* accept_path,
+                    int32_t* bonus_token, int32_t* node_argmax, void* stream);
+
+/* Synchronise `stream`, return the device status word of the calls issued on this
+ * context since the last owl_get_status (OWL_OK, OWL_ERR_BAD_TREE, OWL_ERR_BAD_PAGE,
+ * OWL_ERR_TIMEOUT; the first error wins) and clear it. */
+int owl_get_status(owl_ctx* ctx, void* stream);
+
+/* Text for a status code; never NULL. */
+const char* owl_status_string(int status);
+
+/* Text of the last CUDA error seen by this context ("" if none); valid until the next call. */
+const char* owl_last_error(const owl_ctx* ctx);
+
+/* Number of kernels the library has launched through this context since creation. */
+int64_t owl_launch_count(const owl_ctx* ctx);
+
+/* Seconds of device time (CUDA events on `stream`) of the most recent call's kernels, by
+ * kernel: t[0] verify-attention, t[1] combine, t[2] arg-max, t[3] acceptance walk.  Only
+ * measured while profiling is on (owl_set_profiling(ctx, 1)); synchronises `stream`. */
+int owl_set_profiling(owl_ctx* ctx, int on);
+int owl_last_kernel_times(owl_ctx* ctx, void* stream, double t[4]);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* OWLVERIFY_H_ */

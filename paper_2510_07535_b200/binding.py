@@ -1,0 +1,160 @@
+"""Thin ctypes binding of libowlverify (argument marshalling only; every step runs in the CUDA
+kernels).  PyTorch supplies device memory and streams.  There is no fallback: if the shared
+library has not been built, loading raises."""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libowlverify.so")
+_lib = None
+
+OWL_OK = 0
+STATUS = {0: "OWL_OK", -1: "OWL_ERR_INVALID_ARG", -2: "OWL_ERR_UNSUPPORTED", -3: "OWL_ERR_CUDA",
+          -4: "OWL_ERR_BAD_TREE", -5: "OWL_ERR_BAD_PAGE", -6: "OWL_ERR_TIMEOUT", -7: "OWL_ERR_TOO_LARGE"}
+
+
+class OwlDims(ctypes.Structure):
+    _fields_ = [("batch", ctypes.c_int32), ("total_nodes", ctypes.c_int32), ("max_nodes", ctypes.c_int32),
+                ("num_q_heads", ctypes.c_int32), ("num_kv_heads", ctypes.c_int32), ("head_dim", ctypes.c_int32),
+                ("page_size", ctypes.c_int32), ("max_pages_per_seq", ctypes.c_int32), ("num_pages", ctypes.c_int32),
+                ("vocab", ctypes.c_int32), ("path_stride", ctypes.c_int32), ("sm_scale", ctypes.c_float)]
+
+
+class OwlError(RuntimeError):
+    def __init__(self, code: int, where: str, detail: str = ""):
+        self.code = code
+        super().__init__(f"{where}: {STATUS.get(code, code)} {detail}".strip())
+
+
+def load_library() -> ctypes.CDLL:
+    """dlopen the in-tree libowlverify.so; raises if it was not built (no CPU fallback exists)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2510_07535_b200.build` "
+                          "(nvcc, sm_100a). There is no fallback path.")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i32, i64 = ctypes.c_void_p, ctypes.c_int, ctypes.c_int64
+    dp = ctypes.POINTER(OwlDims)
+    lib.owl_create.restype = i32
+    lib.owl_create.argtypes = [ctypes.POINTER(vp), i32, dp]
+    lib.owl_destroy.restype = i32
+    lib.owl_destroy.argtypes = [vp]
+    lib.owl_verify_attn.restype = i32
+    lib.owl_verify_attn.argtypes = [vp, dp] + [vp] * 10
+    lib.owl_tree_accept.restype = i32
+    lib.owl_tree_accept.argtypes = [vp, dp] + [vp] * 9
+    lib.owl_get_status.restype = i32
+    lib.owl_get_status.argtypes = [vp, vp]
+    lib.owl_status_string.restype = ctypes.c_char_p
+    lib.owl_status_string.argtypes = [i32]
+    lib.owl_last_error.restype = ctypes.c_char_p
+    lib.owl_last_error.argtypes = [vp]
+    lib.owl_launch_count.restype = i64
+    lib.owl_launch_count.argtypes = [vp]
+    lib.owl_set_profiling.restype = i32
+    lib.owl_set_profiling.argtypes = [vp, i32]
+    lib.owl_last_kernel_times.restype = i32
+    lib.owl_last_kernel_times.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_double)]
+    _lib = lib
+    return lib
+
+
+def _ptr(t: Optional[torch.Tensor], dtype: torch.dtype, device: torch.device, name: str):
+    if t is None:
+        return None
+    if t.dtype != dtype or t.device != device or not t.is_contiguous():
+        raise TypeError(f"{name}: expected contiguous {dtype} tensor on {device}, got {t.dtype} on {t.device}")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(device: torch.device) -> ctypes.c_void_p:
+    return ctypes.c_void_p(torch.cuda.current_stream(device).cuda_stream)
+
+
+def make_dims(*, batch, total_nodes, max_nodes, num_q_heads=0, num_kv_heads=0, head_dim=128, page_size=16,
+              max_pages_per_seq=0, num_pages=0, vocab=0, path_stride=64, sm_scale=1.0) -> OwlDims:
+    return OwlDims(batch, total_nodes, max_nodes, num_q_heads, num_kv_heads, head_dim, page_size,
+                   max_pages_per_seq, num_pages, vocab, path_stride, sm_scale)
+
+
+class OwlContext:
+    """Owner of one ``owl_ctx`` (device workspace).  Methods mirror the C entry points."""
+
+    def __init__(self, max_dims: OwlDims, device: Optional[torch.device] = None):
+        self.lib = load_library()
+        self.device = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
+        if self.device.index is None:
+            self.device = torch.device("cuda", torch.cuda.current_device())
+        self._h = ctypes.c_void_p()
+        torch.cuda.init()
+        rc = self.lib.owl_create(ctypes.byref(self._h), self.device.index, ctypes.byref(max_dims))
+        if rc != OWL_OK:
+            raise OwlError(rc, "owl_create")
+
+    def close(self):
+        if getattr(self, "_h", None) and self._h.value:
+            torch.cuda.synchronize(self.device)
+            self.lib.owl_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def owl_verify_attn(self, dims: OwlDims, q, k_cache, v_cache, block_table, ctx_lens, node_offsets, tree_parent,
+                        out, lse, check: bool = True) -> int:
+        dev = self.device
+        rc = self.lib.owl_verify_attn(
+            self._h, ctypes.byref(dims), _ptr(q, torch.bfloat16, dev, "q"), _ptr(k_cache, torch.bfloat16, dev, "k_cache"),
+            _ptr(v_cache, torch.bfloat16, dev, "v_cache"), _ptr(block_table, torch.int32, dev, "block_table"),
+            _ptr(ctx_lens, torch.int32, dev, "ctx_lens"), _ptr(node_offsets, torch.int32, dev, "node_offsets"),
+            _ptr(tree_parent, torch.int32, dev, "tree_parent"), _ptr(out, torch.bfloat16, dev, "out"),
+            _ptr(lse, torch.float32, dev, "lse"), _stream(dev))
+        if check and rc != OWL_OK:
+            raise OwlError(rc, "owl_verify_attn", self.last_error())
+        return rc
+
+    def owl_tree_accept(self, dims: OwlDims, logits, draft_tokens, node_offsets, tree_parent, accept_len, accept_path,
+                        bonus_token, node_argmax=None, check: bool = True) -> int:
+        dev = self.device
+        rc = self.lib.owl_tree_accept(
+            self._h, ctypes.byref(dims), _ptr(logits, torch.float32, dev, "logits"),
+            _ptr(draft_tokens, torch.int32, dev, "draft_tokens"), _ptr(node_offsets, torch.int32, dev, "node_offsets"),
+            _ptr(tree_parent, torch.int32, dev, "tree_parent"), _ptr(accept_len, torch.int32, dev, "accept_len"),
+            _ptr(accept_path, torch.int32, dev, "accept_path"), _ptr(bonus_token, torch.int32, dev, "bonus_token"),
+            _ptr(node_argmax, torch.int32, dev, "node_argmax"), _stream(dev))
+        if check and rc != OWL_OK:
+            raise OwlError(rc, "owl_tree_accept", self.last_error())
+        return rc
+
+    def owl_get_status(self) -> int:
+        return int(self.lib.owl_get_status(self._h, _stream(self.device)))
+
+    def last_error(self) -> str:
+        return self.lib.owl_last_error(self._h).decode()
+
+    def launch_count(self) -> int:
+        return int(self.lib.owl_launch_count(self._h))
+
+    def set_profiling(self, on: bool) -> None:
+        self.lib.owl_set_profiling(self._h, 1 if on else 0)
+
+    def last_kernel_times(self):
+        t = (ctypes.c_double * 4)()
+        rc = self.lib.owl_last_kernel_times(self._h, _stream(self.device), t)
+        if rc != OWL_OK:
+            raise OwlError(rc, "owl_last_kernel_times")
+        return list(t)
+
+
+def status_string(code: int) -> str:
+    return load_library().owl_status_string(code).decode()

@@ -1,0 +1,145 @@
+// Greedy tree acceptance: row arg-max over the vocabulary, then the acceptance walk.
+//
+// Kernel 1 scans fp32 logits with 16-byte loads.  Every (value, index) candidate is folded into
+// one 64-bit key, high word = the float mapped to an unsigned integer that sorts like the float
+// (NaN mapped to -inf, -0 to +0), low word = ~index, so that an unsigned max picks the larger
+// value and, among equal values, the lower index.  Per-thread, warp (shuffle) and block maxima
+// give one key per (row, vocabulary chunk), stored to part_keys[row][chunk] (no atomics, nothing
+// to initialise).
+//
+// Kernel 2 (one CTA per sequence) reduces the chunk keys to arg-max tokens, evaluates for every node
+// whether all edges on its root path match (draft token == parent's arg-max), picks the deepest
+// matching node (lowest index among equals) and writes accept_len / accept_path / bonus_token.
+#pragma once
+
+#include "owl_common.cuh"
+
+namespace owl {
+
+constexpr int kArgmaxThreads = 256;
+constexpr int kArgmaxChunk = 8192;  // floats per CTA: 8 x float4 per thread
+
+struct AcceptParams {
+    const float* logits;
+    const int32_t* draft_tokens;
+    const int32_t* node_offsets;
+    const int32_t* tree_parent;
+    int32_t* accept_len;
+    int32_t* accept_path;
+    int32_t* bonus_token;
+    int32_t* node_argmax;
+    unsigned long long* part_keys;   // [total_nodes, chunks]
+    int32_t* status;
+    int32_t batch, total_nodes, nodes_uniform, max_nodes, vocab, path_stride, chunks;
+};
+
+__device__ __forceinline__ unsigned long long argmax_key(float x, uint32_t idx) {
+    if (x != x) x = -INFINITY;   // NaN never wins
+    x += 0.0f;                   // -0.0 -> +0.0
+    uint32_t u = __float_as_uint(x);
+    u = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+    return ((unsigned long long)u << 32) | (uint32_t)(~idx);
+}
+
+__global__ void __launch_bounds__(kArgmaxThreads) argmax_partial_kernel(const AcceptParams p) {
+    const int row = blockIdx.y;
+    const long long V = p.vocab;
+    const long long c0 = (long long)blockIdx.x * kArgmaxChunk;
+    const long long c1 = c0 + kArgmaxChunk < V ? c0 + kArgmaxChunk : V;
+    const float* base = p.logits + row * V;
+
+    // [c0, a0) scalar head up to 16-byte alignment, [a0, a1) float4 body, [a1, c1) scalar tail
+    const uintptr_t addr = reinterpret_cast<uintptr_t>(base + c0);
+    long long a0 = c0 + (long long)(((16 - (addr & 15)) & 15) >> 2);
+    if (a0 > c1) a0 = c1;
+    const long long a1 = a0 + ((c1 - a0) & ~3ll);
+
+    float bv = -INFINITY;
+    uint32_t bi = 0xffffffffu;   // "no candidate yet"
+    unsigned long long key = 0;
+    const float4* body = reinterpret_cast<const float4*>(base + a0);
+    const int nvec = (int)((a1 - a0) >> 2);
+    for (int v = threadIdx.x; v < nvec; v += kArgmaxThreads) {
+        const float4 x = __ldg(body + v);
+        const uint32_t i0 = (uint32_t)(a0 + 4ll * v);
+        // NaN reads as -inf; strict '>' keeps the first maximum (indices grow along this thread's walk)
+        const float e0 = x.x != x.x ? -INFINITY : x.x, e1 = x.y != x.y ? -INFINITY : x.y;
+        const float e2 = x.z != x.z ? -INFINITY : x.z, e3 = x.w != x.w ? -INFINITY : x.w;
+        if (bi == 0xffffffffu || e0 > bv) { bv = e0; bi = i0; }
+        if (e1 > bv) { bv = e1; bi = i0 + 1; }
+        if (e2 > bv) { bv = e2; bi = i0 + 2; }
+        if (e3 > bv) { bv = e3; bi = i0 + 3; }
+    }
+    if (bi != 0xffffffffu) key = argmax_key(bv, bi);
+    // ragged ends: at most 3 + 3 elements per chunk
+    if (threadIdx.x < 8) {
+        long long j = threadIdx.x < 4 ? c0 + threadIdx.x : a1 + (threadIdx.x - 4);
+        const long long lim = threadIdx.x < 4 ? a0 : c1;
+        if (j < lim) {
+            const unsigned long long k2 = argmax_key(base[j], (uint32_t)j);
+            key = k2 > key ? k2 : key;
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const unsigned long long other = __shfl_xor_sync(0xffffffffu, key, o);
+        key = other > key ? other : key;
+    }
+    __shared__ unsigned long long s_key[kArgmaxThreads / 32];
+    if ((threadIdx.x & 31) == 0) s_key[threadIdx.x >> 5] = key;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+#pragma unroll
+        for (int w = 1; w < kArgmaxThreads / 32; ++w) key = s_key[w] > key ? s_key[w] : key;
+        p.part_keys[(long long)row * p.chunks + blockIdx.x] = key;
+    }
+}
+
+__global__ void __launch_bounds__(kMaxNodes) accept_walk_kernel(const AcceptParams p) {
+    const int b = blockIdx.x, i = threadIdx.x;
+    const int base = p.node_offsets ? p.node_offsets[b] : b * p.nodes_uniform;
+    const int n = p.node_offsets ? p.node_offsets[b + 1] - base : p.nodes_uniform;
+    __shared__ int s_parent[kMaxNodes], s_am[kMaxNodes], s_tok[kMaxNodes];
+    __shared__ int s_bad, s_win;
+    if (i == 0) { s_bad = (n < 1 || n > p.max_nodes || n > p.path_stride || base < 0 || base + n > p.total_nodes) ? 1 : 0; s_win = 0; }
+    __syncthreads();
+    if (s_bad) { if (i == 0) report(p.status, kErrBadTree); return; }
+    if (i < n) {
+        const int pi = p.tree_parent[base + i];
+        s_parent[i] = pi;
+        s_tok[i] = p.draft_tokens[base + i];
+        unsigned long long k = 0;
+        const unsigned long long* pk = p.part_keys + (long long)(base + i) * p.chunks;
+        for (int c = 0; c < p.chunks; ++c) k = pk[c] > k ? pk[c] : k;
+        const int am = (int)(~(uint32_t)(k & 0xffffffffull));
+        s_am[i] = am;
+        if (p.node_argmax) p.node_argmax[base + i] = am;
+        if ((i == 0 && pi != -1) || (i > 0 && (pi < 0 || pi >= i))) atomicExch(&s_bad, 1);
+    }
+    __syncthreads();
+    if (s_bad) { if (i == 0) report(p.status, kErrBadTree); return; }
+
+    // ok(i): every edge on the root path of i matches; depth(i): number of edges
+    int key = 0;
+    if (i < n) {
+        bool ok = true;
+        int depth = 0;
+        for (int c = i; s_parent[c] >= 0 && depth < kMaxNodes; c = s_parent[c], ++depth)
+            ok = ok && s_tok[c] >= 0 && s_tok[c] == s_am[s_parent[c]];
+        if (ok) key = ((depth + 1) << 8) | (kMaxNodes - 1 - i);   // deeper first, then lower index
+    }
+    atomicMax(&s_win, key);
+    __syncthreads();
+    if (i == 0) {
+        const int win = kMaxNodes - 1 - (s_win & 0xff);
+        const int len = s_win >> 8;
+        p.accept_len[b] = len;
+        p.bonus_token[b] = s_am[win];
+        int32_t* path = p.accept_path + (long long)b * p.path_stride;
+        for (int k = len; k < p.path_stride; ++k) path[k] = -1;
+        int k = len - 1;
+        for (int c = win; c >= 0 && k >= 0; c = s_parent[c]) path[k--] = c;
+    }
+}
+
+}  // namespace owl

@@ -1,0 +1,167 @@
+// Shared device/host helpers of libowlverify: work partition of the split-KV pass,
+// status reporting, small PTX wrappers.  sm_100a only.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace owl {
+
+constexpr int kHeadDim = 128;
+constexpr int kMaxNodes = 64;     // drafted nodes per sequence (the paper's trees have 60)
+constexpr int kMaxBatch = 1024;   // sequences per call (schedule prefix sums live in shared memory)
+constexpr int kMaxRows = 256;     // packed rows (query heads of a KV group x nodes) per (sequence, KV head)
+
+// Device-detected status codes: same values as owl_status in owlverify.h.
+constexpr int kErrBadTree = -4;
+constexpr int kErrBadPage = -5;
+constexpr int kErrTimeout = -6;
+
+// Problem description handed to every kernel of the attention path.
+struct AttnParams {
+    const __nv_bfloat16* q;
+    const __nv_bfloat16* k_cache;
+    const __nv_bfloat16* v_cache;
+    const int32_t* block_table;
+    const int32_t* ctx_lens;
+    const int32_t* node_offsets;  // may be null: uniform nodes_uniform per sequence
+    const int32_t* tree_parent;
+    __nv_bfloat16* out;
+    float* lse;                   // may be null
+    float* part_o;                // [slots, rows_per_slot, D] fp32, normalised partial outputs
+    float* part_lse;              // [slots, rows_per_slot] fp32, natural-log partial LSE (-inf if empty)
+    int32_t* status;              // device status word (0 = ok, first error wins)
+    int32_t* seq_bad;             // [B] epoch of the call in which the sequence was found malformed
+    int32_t epoch;
+    int32_t batch, total_nodes, nodes_uniform, max_nodes;
+    int32_t num_q_heads, num_kv_heads, group;  // group = Hq / Hkv
+    int32_t page_size, page_shift, max_pages_per_seq, num_pages;
+    int32_t rows_per_slot;        // row stride of one partial slot
+    int32_t num_ctas;             // CTAs of the split-KV pass (the flat tile range is cut into this many pieces)
+    float sm_scale;
+};
+
+// 2^x by the special-function unit (ex2.approx, denormals flushed); ex2(-inf) = 0.
+__device__ __forceinline__ float fast_exp2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+__device__ __forceinline__ void report(int32_t* status, int code) { atomicCAS(status, 0, code); }
+
+// ---------------------------------------------------------------------------------------------
+// Flat partition of the split-KV pass.
+//
+// A unit is (sequence b, KV head h, row block mb); it owns tiles_b = ceil((L_b + n_b) / TileKeys)
+// key tiles.  Units are laid out sequence-major, then head, then row block; all their tiles form
+// one flat range [0, total) which is cut into num_ctas contiguous, nearly equal pieces.  A CTA's
+// piece may start and end inside a unit; each (CTA, unit) intersection yields one partial
+// (o, lse) stored in slot cta + unit, which is unique because pieces and units are both ordered.
+// ---------------------------------------------------------------------------------------------
+struct SeqSched {
+    long long tile_begin;  // first flat tile of the sequence
+    int unit_begin;        // first unit of the sequence
+    int tiles;             // key tiles per unit
+    int row_blocks;        // row blocks per (sequence, head)
+    int n, L;              // drafted nodes, committed context length
+    int node_base;
+};
+
+struct Partition {
+    long long total, q;
+    int rem, ctas;
+    __device__ __host__ void init(long long total_, int ctas_) {
+        total = total_; ctas = ctas_; q = total_ / ctas_; rem = (int)(total_ % ctas_);
+    }
+    __device__ __host__ long long begin(int c) const { return (long long)c * q + (c < rem ? c : rem); }
+    __device__ __host__ int owner(long long t) const {
+        long long big = (long long)rem * (q + 1);
+        return t < big ? (int)(t / (q + 1)) : rem + (int)((t - big) / q);
+    }
+};
+
+__device__ __forceinline__ int seq_nodes(const AttnParams& p, int b) {
+    return p.node_offsets ? p.node_offsets[b + 1] - p.node_offsets[b] : p.nodes_uniform;
+}
+__device__ __forceinline__ int seq_node_base(const AttnParams& p, int b) {
+    return p.node_offsets ? p.node_offsets[b] : b * p.nodes_uniform;
+}
+
+// A sequence is schedulable when its node count and lengths are inside the interface's limits.
+__device__ __forceinline__ bool seq_tree_shape_ok(const AttnParams& p, int b, int n) {
+    const int base = seq_node_base(p, b);
+    return n >= 1 && n <= p.max_nodes && base >= 0 && base + n <= p.total_nodes;
+}
+__device__ __forceinline__ bool seq_shape_ok(const AttnParams& p, int b, int n, int L) {
+    if (!seq_tree_shape_ok(p, b, n) || L < 0) return false;
+    long long keys = (long long)L + n;
+    return keys <= (long long)p.max_pages_per_seq * p.page_size;
+}
+
+// Every CTA derives the same per-sequence schedule into shared memory.
+// s_tile[b], s_unit[b] are exclusive prefix sums; entries [batch] hold the totals.
+template <int TileKeys, int RowsPerBlock>
+__device__ void build_schedule(const AttnParams& p, long long* s_tile, int* s_unit) {
+    // serial prefix by one thread per 32 sequences would be overkill: batch is at most 1024 and
+    // this runs once per CTA; thread 0 walks it after all threads staged the per-sequence counts.
+    for (int b = threadIdx.x; b < p.batch; b += blockDim.x) {
+        int n = seq_nodes(p, b), L = p.ctx_lens[b];
+        int units = 0, tiles = 0;
+        if (seq_shape_ok(p, b, n, L)) {
+            tiles = (L + n + TileKeys - 1) / TileKeys;
+            units = p.num_kv_heads * ((n * p.group + RowsPerBlock - 1) / RowsPerBlock);
+        } else {
+            report(p.status, seq_tree_shape_ok(p, b, n) ? kErrBadPage : kErrBadTree);
+            p.seq_bad[b] = p.epoch;
+        }
+        s_tile[b + 1] = (long long)tiles * units;
+        s_unit[b + 1] = units;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        s_tile[0] = 0; s_unit[0] = 0;
+        for (int b = 0; b < p.batch; ++b) { s_tile[b + 1] += s_tile[b]; s_unit[b + 1] += s_unit[b]; }
+    }
+    __syncthreads();
+}
+
+template <int TileKeys, int RowsPerBlock>
+__device__ __forceinline__ SeqSched seq_sched(const AttnParams& p, const long long* s_tile, const int* s_unit, int b) {
+    SeqSched s;
+    s.tile_begin = s_tile[b];
+    s.unit_begin = s_unit[b];
+    s.n = seq_nodes(p, b);
+    s.L = p.ctx_lens[b];
+    s.node_base = seq_node_base(p, b);
+    s.tiles = (s.L + s.n + TileKeys - 1) / TileKeys;
+    s.row_blocks = (s.n * p.group + RowsPerBlock - 1) / RowsPerBlock;
+    return s;
+}
+
+// Ancestor-or-self bitmasks of one sequence's tree: bit j of anc[i] is set iff node j lies on the
+// root path of node i (Section 3.2.2 "Decode Stage": a token sees exactly its own tree path).
+// Returns false (and writes nothing useful) if the tree violates parent[i] < i / single root.
+__device__ __forceinline__ bool build_ancestors(const int32_t* parent, int n, unsigned long long* anc /*smem[64]*/,
+                                                int* s_flag /*smem*/) {
+    if (threadIdx.x == 0) *s_flag = 0;
+    __syncthreads();
+    if (threadIdx.x < n) {
+        int i = threadIdx.x;
+        int pi = parent[i];
+        if ((i == 0 && pi != -1) || (i > 0 && (pi < 0 || pi >= i))) atomicExch(s_flag, 1);
+    }
+    __syncthreads();
+    bool ok = (*s_flag == 0);
+    if (ok && threadIdx.x < n) {
+        int i = threadIdx.x;
+        unsigned long long m = 0;
+        for (int j = i, guard = 0; j >= 0 && guard < kMaxNodes; j = parent[j], ++guard) m |= 1ull << j;
+        anc[i] = m;
+    }
+    __syncthreads();
+    return ok;
+}
+
+}  // namespace owl

@@ -1,0 +1,321 @@
+// Host side of libowlverify: argument checks, workspace, kernel launches.  C ABI in owlverify.h.
+#include "../../include/owlverify.h"
+
+#include <cuda_runtime.h>
+
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "accept.cuh"
+#include "combine.cuh"
+#include "owl_common.cuh"
+#include "verify_attn_mma.cuh"
+
+using namespace owl;
+
+struct owl_ctx {
+    int device = 0;
+    int sm_count = 0;
+    owl_dims max_dims{};
+    int num_ctas = 0;
+    int rows_per_slot = 0;
+    long long slots = 0;
+    float* part_o = nullptr;
+    float* part_lse = nullptr;
+    int32_t* status = nullptr;
+    int32_t* seq_bad = nullptr;
+    unsigned long long* part_keys = nullptr;
+    long long part_keys_len = 0;
+    int32_t epoch = 0;
+    int64_t launches = 0;
+    bool profiling = false;
+    cudaEvent_t ev[6] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
+    bool ev_attn_valid = false, ev_accept_valid = false;
+    char err[256] = {0};
+};
+
+namespace {
+
+struct DeviceGuard {
+    int prev = -1;
+    bool switched = false;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) == cudaSuccess && prev != dev) switched = (cudaSetDevice(dev) == cudaSuccess);
+    }
+    ~DeviceGuard() { if (switched) cudaSetDevice(prev); }
+};
+
+int cuda_fail(owl_ctx* ctx, cudaError_t e, const char* what) {
+    if (ctx) snprintf(ctx->err, sizeof ctx->err, "%s: %s", what, cudaGetErrorString(e));
+    return OWL_ERR_CUDA;
+}
+
+int log2_exact(int v) {
+    int s = 0;
+    while ((1 << s) < v) ++s;
+    return (1 << s) == v ? s : -1;
+}
+
+// Checks that need no device data.  `for_accept` also checks vocab / path_stride.
+int check_dims(const owl_dims* d, bool for_attn, bool for_accept) {
+    if (!d) return OWL_ERR_INVALID_ARG;
+    if (d->batch < 1 || d->total_nodes < d->batch || d->max_nodes < 1) return OWL_ERR_INVALID_ARG;
+    if (d->max_nodes > kMaxNodes || d->batch > kMaxBatch) return OWL_ERR_UNSUPPORTED;
+    if ((long long)d->max_nodes * d->batch < d->total_nodes) return OWL_ERR_INVALID_ARG;
+    if (for_attn) {
+        if (d->num_q_heads < 1 || d->num_kv_heads < 1 || d->num_q_heads % d->num_kv_heads != 0) return OWL_ERR_INVALID_ARG;
+        if (d->max_pages_per_seq < 1 || d->num_pages < 1) return OWL_ERR_INVALID_ARG;
+        if (!(d->sm_scale == d->sm_scale)) return OWL_ERR_INVALID_ARG;
+        if (d->head_dim != kHeadDim) return OWL_ERR_UNSUPPORTED;
+        if ((d->num_q_heads / d->num_kv_heads) * d->max_nodes > kMaxRows) return OWL_ERR_UNSUPPORTED;
+        if (!(d->page_size == 16 || d->page_size == 32 || d->page_size == 64 || d->page_size == 128)) return OWL_ERR_UNSUPPORTED;
+    }
+    if (for_accept) {
+        if (d->vocab < 1) return OWL_ERR_INVALID_ARG;
+        if (d->path_stride < d->max_nodes) return OWL_ERR_INVALID_ARG;
+    }
+    return OWL_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* owl_status_string(int status) {
+    switch (status) {
+        case OWL_OK: return "ok";
+        case OWL_ERR_INVALID_ARG: return "invalid argument";
+        case OWL_ERR_UNSUPPORTED: return "unsupported shape";
+        case OWL_ERR_CUDA: return "CUDA error";
+        case OWL_ERR_BAD_TREE: return "malformed tree (device-detected)";
+        case OWL_ERR_BAD_PAGE: return "page index or context length out of range (device-detected)";
+        case OWL_ERR_TIMEOUT: return "bounded device wait expired";
+        case OWL_ERR_TOO_LARGE: return "dims exceed the context's capacity";
+        default: return "unknown status";
+    }
+}
+
+const char* owl_last_error(const owl_ctx* ctx) { return ctx ? ctx->err : ""; }
+int64_t owl_launch_count(const owl_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+int owl_create(owl_ctx** out, int device, const owl_dims* max_dims) {
+    if (!out || !max_dims) return OWL_ERR_INVALID_ARG;
+    *out = nullptr;
+    const bool attn = max_dims->num_q_heads > 0;
+    const bool acc = max_dims->vocab > 0;
+    int rc = check_dims(max_dims, attn, false);
+    if (rc != OWL_OK) return rc;
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess || device < 0 || device >= ndev) return OWL_ERR_INVALID_ARG;
+
+    owl_ctx* ctx = new (std::nothrow) owl_ctx();
+    if (!ctx) return OWL_ERR_CUDA;
+    ctx->device = device;
+    ctx->max_dims = *max_dims;
+    DeviceGuard guard(device);
+    cudaError_t e;
+    cudaDeviceProp prop;
+    if ((e = cudaGetDeviceProperties(&prop, device)) != cudaSuccess) { delete ctx; return OWL_ERR_CUDA; }
+    if (prop.major != 10) { delete ctx; return OWL_ERR_UNSUPPORTED; }  // sm_100a code only
+    ctx->sm_count = prop.multiProcessorCount;
+    ctx->num_ctas = ctx->sm_count;
+
+    bool ok = true;
+    auto alloc = [&](void** p, size_t bytes) {
+        if (ok && (e = cudaMalloc(p, bytes ? bytes : 16)) != cudaSuccess) ok = false;
+    };
+    if (attn) {
+        const int G = max_dims->num_q_heads / max_dims->num_kv_heads;
+        const int M = G * max_dims->max_nodes;
+        const int row_blocks = (M + mma_path::kRows - 1) / mma_path::kRows;
+        ctx->rows_per_slot = mma_path::kRows;
+        ctx->slots = (long long)ctx->num_ctas + (long long)max_dims->batch * max_dims->num_kv_heads * row_blocks;
+        alloc((void**)&ctx->part_o, (size_t)ctx->slots * ctx->rows_per_slot * kHeadDim * sizeof(float));
+        alloc((void**)&ctx->part_lse, (size_t)ctx->slots * ctx->rows_per_slot * sizeof(float));
+    }
+    alloc((void**)&ctx->status, sizeof(int32_t));
+    alloc((void**)&ctx->seq_bad, (size_t)max_dims->batch * sizeof(int32_t));
+    if (acc) {
+        ctx->part_keys_len = (long long)max_dims->total_nodes * ((max_dims->vocab + kArgmaxChunk - 1) / kArgmaxChunk);
+        alloc((void**)&ctx->part_keys, (size_t)ctx->part_keys_len * sizeof(unsigned long long));
+    }
+    if (ok) {
+        ok = cudaMemset(ctx->status, 0, sizeof(int32_t)) == cudaSuccess &&
+             cudaMemset(ctx->seq_bad, 0, (size_t)max_dims->batch * sizeof(int32_t)) == cudaSuccess;
+    }
+    for (int i = 0; ok && i < 6; ++i) ok = cudaEventCreate(&ctx->ev[i]) == cudaSuccess;
+    if (ok && attn) {
+        ok = cudaFuncSetAttribute(mma_path::verify_attn_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  mma_path::kSmemBytes) == cudaSuccess;
+    }
+    if (!ok || cudaDeviceSynchronize() != cudaSuccess) {
+        cudaGetLastError();
+        owl_destroy(ctx);
+        return OWL_ERR_CUDA;
+    }
+    *out = ctx;
+    return OWL_OK;
+}
+
+int owl_destroy(owl_ctx* ctx) {
+    if (!ctx) return OWL_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    cudaFree(ctx->part_o);
+    cudaFree(ctx->part_lse);
+    cudaFree(ctx->status);
+    cudaFree(ctx->seq_bad);
+    cudaFree(ctx->part_keys);
+    for (auto& ev : ctx->ev)
+        if (ev) cudaEventDestroy(ev);
+    delete ctx;
+    return OWL_OK;
+}
+
+int owl_verify_attn(owl_ctx* ctx, const owl_dims* d, const void* q, const void* k_cache, const void* v_cache,
+                    const int32_t* block_table, const int32_t* ctx_lens, const int32_t* node_offsets,
+                    const int32_t* tree_parent, void* out, float* lse, void* stream_) {
+    if (!ctx) return OWL_ERR_INVALID_ARG;
+    int rc = check_dims(d, true, false);
+    if (rc != OWL_OK) return rc;
+    if (!q || !k_cache || !v_cache || !block_table || !ctx_lens || !tree_parent || !out) return OWL_ERR_INVALID_ARG;
+    if (!node_offsets && d->total_nodes % d->batch != 0) return OWL_ERR_INVALID_ARG;
+    if (!ctx->part_o) return OWL_ERR_TOO_LARGE;
+    const owl_dims& mx = ctx->max_dims;
+    const int G = d->num_q_heads / d->num_kv_heads;
+    const int row_blocks = (G * d->max_nodes + mma_path::kRows - 1) / mma_path::kRows;
+    if (d->batch > mx.batch || d->total_nodes > mx.total_nodes ||
+        (long long)ctx->num_ctas + (long long)d->batch * d->num_kv_heads * row_blocks > ctx->slots)
+        return OWL_ERR_TOO_LARGE;
+
+    DeviceGuard guard(ctx->device);
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    AttnParams p{};
+    p.q = static_cast<const __nv_bfloat16*>(q);
+    p.k_cache = static_cast<const __nv_bfloat16*>(k_cache);
+    p.v_cache = static_cast<const __nv_bfloat16*>(v_cache);
+    p.block_table = block_table;
+    p.ctx_lens = ctx_lens;
+    p.node_offsets = node_offsets;
+    p.tree_parent = tree_parent;
+    p.out = static_cast<__nv_bfloat16*>(out);
+    p.lse = lse;
+    p.part_o = ctx->part_o;
+    p.part_lse = ctx->part_lse;
+    p.status = ctx->status;
+    p.seq_bad = ctx->seq_bad;
+    p.epoch = ++ctx->epoch;
+    p.batch = d->batch;
+    p.total_nodes = d->total_nodes;
+    p.nodes_uniform = d->total_nodes / d->batch;
+    p.max_nodes = d->max_nodes;
+    p.num_q_heads = d->num_q_heads;
+    p.num_kv_heads = d->num_kv_heads;
+    p.group = G;
+    p.page_size = d->page_size;
+    p.page_shift = log2_exact(d->page_size);
+    p.max_pages_per_seq = d->max_pages_per_seq;
+    p.num_pages = d->num_pages;
+    p.rows_per_slot = ctx->rows_per_slot;
+    p.num_ctas = ctx->num_ctas;
+    p.sm_scale = d->sm_scale;
+
+    if (ctx->profiling) cudaEventRecord(ctx->ev[0], stream);
+    mma_path::verify_attn_mma_kernel<<<ctx->num_ctas, mma_path::kThreads, mma_path::kSmemBytes, stream>>>(p);
+    ++ctx->launches;
+    if (ctx->profiling) cudaEventRecord(ctx->ev[1], stream);
+    const long long rows = (long long)d->total_nodes * d->num_q_heads;
+    const unsigned grid = (unsigned)((rows + kCombineWarps - 1) / kCombineWarps);
+    combine_kernel<mma_path::kTileKeys, mma_path::kRows><<<grid, kCombineWarps * 32, 0, stream>>>(p);
+    ++ctx->launches;
+    if (ctx->profiling) { cudaEventRecord(ctx->ev[2], stream); ctx->ev_attn_valid = true; }
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "owl_verify_attn launch");
+    return OWL_OK;
+}
+
+int owl_tree_accept(owl_ctx* ctx, const owl_dims* d, const float* logits, const int32_t* draft_tokens,
+                    const int32_t* node_offsets, const int32_t* tree_parent, int32_t* accept_len,
+                    int32_t* accept_path, int32_t* bonus_token, int32_t* node_argmax, void* stream_) {
+    if (!ctx) return OWL_ERR_INVALID_ARG;
+    int rc = check_dims(d, false, true);
+    if (rc != OWL_OK) return rc;
+    if (!logits || !draft_tokens || !tree_parent || !accept_len || !accept_path || !bonus_token) return OWL_ERR_INVALID_ARG;
+    if (!node_offsets && d->total_nodes % d->batch != 0) return OWL_ERR_INVALID_ARG;
+    if (d->batch > ctx->max_dims.batch || d->total_nodes > ctx->max_dims.total_nodes) return OWL_ERR_TOO_LARGE;
+    if (d->total_nodes > 65535) return OWL_ERR_UNSUPPORTED;
+    const int chunks = (d->vocab + kArgmaxChunk - 1) / kArgmaxChunk;
+    if (!ctx->part_keys || (long long)d->total_nodes * chunks > ctx->part_keys_len) return OWL_ERR_TOO_LARGE;
+
+    DeviceGuard guard(ctx->device);
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    AcceptParams p{};
+    p.logits = logits;
+    p.draft_tokens = draft_tokens;
+    p.node_offsets = node_offsets;
+    p.tree_parent = tree_parent;
+    p.accept_len = accept_len;
+    p.accept_path = accept_path;
+    p.bonus_token = bonus_token;
+    p.node_argmax = node_argmax;
+    p.part_keys = ctx->part_keys;
+    p.chunks = chunks;
+    p.status = ctx->status;
+    p.batch = d->batch;
+    p.total_nodes = d->total_nodes;
+    p.nodes_uniform = d->total_nodes / d->batch;
+    p.max_nodes = d->max_nodes;
+    p.vocab = d->vocab;
+    p.path_stride = d->path_stride;
+
+    if (ctx->profiling) cudaEventRecord(ctx->ev[3], stream);
+    dim3 grid((unsigned)chunks, (unsigned)d->total_nodes);
+    argmax_partial_kernel<<<grid, kArgmaxThreads, 0, stream>>>(p);
+    ++ctx->launches;
+    if (ctx->profiling) cudaEventRecord(ctx->ev[4], stream);
+    accept_walk_kernel<<<d->batch, kMaxNodes, 0, stream>>>(p);
+    ++ctx->launches;
+    if (ctx->profiling) { cudaEventRecord(ctx->ev[5], stream); ctx->ev_accept_valid = true; }
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "owl_tree_accept launch");
+    return OWL_OK;
+}
+
+int owl_get_status(owl_ctx* ctx, void* stream_) {
+    if (!ctx) return OWL_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    int32_t st = 0;
+    cudaError_t e = cudaMemcpyAsync(&st, ctx->status, sizeof st, cudaMemcpyDeviceToHost, stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(ctx->status, 0, sizeof st, stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "owl_get_status");
+    return st;
+}
+
+int owl_set_profiling(owl_ctx* ctx, int on) {
+    if (!ctx) return OWL_ERR_INVALID_ARG;
+    ctx->profiling = on != 0;
+    ctx->ev_attn_valid = ctx->ev_accept_valid = false;
+    return OWL_OK;
+}
+
+int owl_last_kernel_times(owl_ctx* ctx, void* stream_, double t[4]) {
+    if (!ctx || !t) return OWL_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    cudaError_t e = cudaStreamSynchronize(static_cast<cudaStream_t>(stream_));
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "owl_last_kernel_times");
+    t[0] = t[1] = t[2] = t[3] = 0.0;
+    float ms = 0.f;
+    if (ctx->ev_attn_valid) {
+        if (cudaEventElapsedTime(&ms, ctx->ev[0], ctx->ev[1]) == cudaSuccess) t[0] = ms * 1e-3;
+        if (cudaEventElapsedTime(&ms, ctx->ev[1], ctx->ev[2]) == cudaSuccess) t[1] = ms * 1e-3;
+    }
+    if (ctx->ev_accept_valid) {
+        if (cudaEventElapsedTime(&ms, ctx->ev[3], ctx->ev[4]) == cudaSuccess) t[2] = ms * 1e-3;
+        if (cudaEventElapsedTime(&ms, ctx->ev[4], ctx->ev[5]) == cudaSuccess) t[3] = ms * 1e-3;
+    }
+    return OWL_OK;
+}
+
+}  // extern "C"

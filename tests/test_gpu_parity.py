@@ -1,0 +1,201 @@
+"""Parity of the CUDA path (through the C ABI) against the CPU oracle, element by element, on
+seeded inputs small enough for the oracle yet spanning several key tiles, ragged tails, several
+CTAs per unit and several units per CTA."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2510_07535_b200 import OwlContext, make_dims, workloads as W
+from paper_2510_07535_b200.runner import DeviceWorkload, dims_of
+
+pytestmark = pytest.mark.gpu
+
+OUT_TOL = 1e-2   # max |err| of the bf16 outputs against the fp64 oracle
+LSE_TOL = 1e-3   # max |err| of the fp32 LSE
+
+
+def check_attention(wl, ctx=None):
+    dw = DeviceWorkload.upload(wl)
+    own = ctx is None
+    ctx = ctx or OwlContext(dims_of(wl))
+    dw.attn(ctx)
+    assert ctx.owl_get_status() == 0
+    ref_out, ref_lse = oracle.verify_attn(wl.q, wl.k_cache, wl.v_cache, wl.block_table, wl.ctx_lens,
+                                          wl.node_offsets, wl.tree_parent, wl.sm_scale)
+    out, lse = dw.out_f32().astype(np.float64), dw.lse.cpu().numpy().astype(np.float64)
+    eo, el = np.abs(out - ref_out).max(), np.abs(lse - ref_lse).max()
+    # second run must be bit-identical (no races, no dependence on workspace contents)
+    out1 = dw.out.clone(); lse1 = dw.lse.clone()
+    dw.out.zero_(); dw.lse.zero_()
+    dw.attn(ctx)
+    assert torch.equal(out1, dw.out) and torch.equal(lse1, dw.lse)
+    if own:
+        ctx.close()
+    assert eo <= OUT_TOL, f"out err {eo}"
+    assert el <= LSE_TOL, f"lse err {el}"
+    return eo, el
+
+
+def check_accept(wl, ctx=None):
+    dw = DeviceWorkload.upload(wl)
+    own = ctx is None
+    ctx = ctx or OwlContext(dims_of(wl))
+    for _ in range(2):   # twice: the arg-max scratch must be reset by the call itself
+        dw.accept(ctx)
+        assert ctx.owl_get_status() == 0
+        alen, path, bonus, am = oracle.tree_accept(wl.logits, wl.draft_tokens, wl.node_offsets, wl.tree_parent, 64)
+        np.testing.assert_array_equal(dw.node_argmax.cpu().numpy(), am)
+        np.testing.assert_array_equal(dw.accept_len.cpu().numpy(), alen)
+        np.testing.assert_array_equal(dw.accept_path.cpu().numpy(), path)
+        np.testing.assert_array_equal(dw.bonus_token.cpu().numpy(), bonus)
+        dw.accept_len.zero_(); dw.accept_path.zero_(); dw.bonus_token.zero_(); dw.node_argmax.zero_()
+    if own:
+        ctx.close()
+
+
+@pytest.mark.parametrize("idx", [0, 1, 2, 3, 4])
+@pytest.mark.parametrize("prescaled", [True, False])
+def test_scaled_down_configs_attention(idx, prescaled):
+    """The five benchmark configurations with contexts shrunk 32x-64x (ragged), every output element."""
+    div = {0: 4, 1: 32, 2: 128, 3: 64, 4: 64}[idx]
+    spec = W.config_spec(idx, ctx_div=div, vocab=1024, q_prescaled=prescaled)
+    spec.with_logits = False
+    check_attention(W.generate(spec))
+
+
+@pytest.mark.parametrize("idx", [0, 1, 2, 3, 4])
+def test_configs_acceptance_full_vocab(idx):
+    """Acceptance at the full vocabulary (128256) of every configuration, bit-exact."""
+    spec = W.config_spec(idx, ctx_div=4096)
+    check_accept(W.generate(spec))
+
+
+@pytest.mark.parametrize("hq,hkv,trees,ctx", [
+    (8, 8, [("chain", 1)], [1]),                          # G = 1, one node, one context token
+    (8, 2, [("chain", 1)], [0]),                          # empty context: the root sees only itself
+    (4, 1, [("tree", 64, 8)], [0]),                       # empty context, full 64-node tree (M = 256)
+    (32, 8, [("tree", 64, 8), ("chain", 3)], [777, 15]),  # two row blocks + a tiny sequence
+    (16, 2, [("tree", 17, 4)] * 3, [63, 64, 65]),         # lengths around a tile edge
+    (64, 8, [("tree", 32, 6)], [5000]),                   # 70B head geometry
+    (12, 4, [("tree", 11, 4), ("chain", 7)], [300, 1000]),  # G = 3: rows of a node straddle nothing regular
+])
+def test_edge_shapes_attention(hq, hkv, trees, ctx):
+    wl = W.generate(W.Spec("edge", hq, hkv, ctx, trees, shuffle_pages=True, seed=hq * 1000 + ctx[0], with_logits=False))
+    check_attention(wl)
+
+
+def test_draft_keys_straddle_tiles_and_pages():
+    # L = 1020: draft positions 1020..1051 cross a 64-key tile edge and a page edge
+    wl = W.generate(W.Spec("straddle", 8, 2, [1020, 1080], [("tree", 32, 6), ("tree", 40, 6)], shuffle_pages=True,
+                           seed=77, with_logits=False))
+    check_attention(wl)
+
+
+def test_many_short_sequences_one_cta_many_units():
+    rng = np.random.default_rng(5)
+    ctx = [int(x) for x in rng.integers(1, 200, size=96)]
+    trees = [("chain", int(rng.integers(1, 9))) for _ in range(96)]
+    wl = W.generate(W.Spec("many", 8, 2, ctx, trees, shuffle_pages=True, seed=78, with_logits=False))
+    check_attention(wl)
+
+
+def test_uniform_node_offsets_null():
+    wl = W.generate(W.Spec("uniform", 8, 2, [100, 333, 90], [("tree", 8, 3)] * 3, seed=79, with_logits=True, vocab=1000))
+    dw = DeviceWorkload.upload(wl)
+    ctx = OwlContext(dims_of(wl))
+    dw.node_offsets = None
+    dw.step(ctx)
+    assert ctx.owl_get_status() == 0
+    ref_out, ref_lse = oracle.verify_attn(wl.q, wl.k_cache, wl.v_cache, wl.block_table, wl.ctx_lens,
+                                          wl.node_offsets, wl.tree_parent, wl.sm_scale)
+    assert np.abs(dw.out_f32() - ref_out).max() <= OUT_TOL
+    alen, path, bonus, am = oracle.tree_accept(wl.logits, wl.draft_tokens, wl.node_offsets, wl.tree_parent, 64)
+    np.testing.assert_array_equal(dw.accept_len.cpu().numpy(), alen)
+    np.testing.assert_array_equal(dw.bonus_token.cpu().numpy(), bonus)
+    ctx.close()
+
+
+def test_unused_tail_slots_may_hold_large_values():
+    """Slots past L+n in the last page are multiplied by zero weight: finite garbage must not leak."""
+    wl = W.generate(W.Spec("tail", 8, 2, [22], [("tree", 5, 2)], seed=80, with_logits=False))
+    wl.k_cache[1, :, 11:, :] = 0x7F00   # ~1.7e38
+    wl.v_cache[1, :, 11:, :] = 0x7F00
+    check_attention(wl)
+
+
+def test_large_scores_stress_relative_tolerance():
+    """Outputs of order 10 and scores of order 30: |err| <= 1e-2 + 2^-8 |ref| (bf16 half-ulp dominates)."""
+    wl = W.generate(W.Spec("stress", 8, 2, [500], [("tree", 16, 4)], seed=81, with_logits=False, q_prescaled=True))
+    v = W.bf16_bits_to_f32(wl.v_cache) * 10
+    wl.v_cache[...] = W.f32_to_bf16_bits(v)
+    wl.sm_scale = 3.0
+    dw = DeviceWorkload.upload(wl)
+    ctx = OwlContext(dims_of(wl))
+    dw.attn(ctx)
+    ref_out, ref_lse = oracle.verify_attn(wl.q, wl.k_cache, wl.v_cache, wl.block_table, wl.ctx_lens,
+                                          wl.node_offsets, wl.tree_parent, wl.sm_scale)
+    err = np.abs(dw.out_f32() - ref_out)
+    assert np.all(err <= 1e-2 + 2.0 ** -8 * np.abs(ref_out)), err.max()
+    assert np.abs(dw.lse.cpu().numpy() - ref_lse).max() <= LSE_TOL
+    ctx.close()
+
+
+# ----------------------------------------------------------------------------- acceptance edge cases
+
+def _accept_case(logits, tokens, offsets, parents, stride=64):
+    B = len(offsets) - 1
+    N = len(parents)
+    d = make_dims(batch=B, total_nodes=N, max_nodes=int(np.diff(offsets).max()), vocab=logits.shape[1],
+                  path_stride=stride)
+    ctx = OwlContext(d)
+    dev = "cuda"
+    t = lambda a, dt: torch.from_numpy(np.ascontiguousarray(a, dtype=dt)).to(dev)
+    alen = torch.zeros(B, dtype=torch.int32, device=dev); path = torch.zeros((B, stride), dtype=torch.int32, device=dev)
+    bonus = torch.zeros(B, dtype=torch.int32, device=dev); am = torch.zeros(N, dtype=torch.int32, device=dev)
+    ctx.owl_tree_accept(d, t(logits, np.float32), t(tokens, np.int32), t(offsets, np.int32), t(parents, np.int32),
+                        alen, path, bonus, am)
+    st = ctx.owl_get_status()
+    ctx.close()
+    return st, alen.cpu().numpy(), path.cpu().numpy(), bonus.cpu().numpy(), am.cpu().numpy()
+
+
+@pytest.mark.parametrize("V", [1, 2, 3, 5, 8191, 8192, 8193, 8195, 20000, 128256, 128257])
+def test_argmax_ragged_vocab_and_special_values(V):
+    rng = np.random.default_rng(V)
+    N = 9
+    lg = rng.standard_normal((N, V)).astype(np.float32)
+    if V > 4:
+        lg[1, 1] = lg[1, V - 1] = 9.0          # tie -> lower index
+        lg[2, :] = -np.inf                      # all -inf -> 0
+        lg[3, :] = 0.0; lg[3, 2] = -0.0         # signed zeros tie
+        lg[4, 0] = np.nan; lg[4, V // 2] = 30.0  # NaN never wins
+        lg[5, :] = np.nan                       # all NaN -> 0
+        lg[6, V - 1] = 99.0                     # last element of the row
+        lg[7, :] = 1e-41                        # denormals compare exactly
+        lg[7, V // 3] = 2e-41
+    parents = W.chain_parents(N)
+    tokens = rng.integers(0, V, size=N).astype(np.int32)
+    st, alen, path, bonus, am = _accept_case(lg, tokens, np.array([0, N]), parents)
+    assert st == 0
+    r_alen, r_path, r_bonus, r_am = oracle.tree_accept(lg, tokens, np.array([0, N], np.int32), parents, 64)
+    np.testing.assert_array_equal(am, r_am)
+    np.testing.assert_array_equal(alen, r_alen)
+    np.testing.assert_array_equal(path, r_path)
+    np.testing.assert_array_equal(bonus, r_bonus)
+
+
+def test_unaligned_logits_rows():
+    """Odd vocabulary: rows start at addresses that are not 16-byte aligned."""
+    rng = np.random.default_rng(9)
+    V, N = 30001, 12
+    lg = rng.standard_normal((N, V)).astype(np.float32)
+    lg[np.arange(N), rng.integers(0, V, N)] += 8
+    parents = W.random_tree_parents(rng, N, 4)
+    tokens = oracle.row_argmax(lg)[np.maximum(parents, 0)].astype(np.int32)   # every edge matches
+    tokens[5] = -1                                                            # a [SPEC]-style leaf
+    st, alen, path, bonus, am = _accept_case(lg, tokens, np.array([0, N]), parents)
+    r = oracle.tree_accept(lg, tokens, np.array([0, N], np.int32), parents, 64)
+    assert st == 0
+    np.testing.assert_array_equal(am, r[3]); np.testing.assert_array_equal(alen, r[0])
+    np.testing.assert_array_equal(path, r[1]); np.testing.assert_array_equal(bonus, r[2])
