@@ -1,0 +1,364 @@
+#!/usr/bin/env python
+"""Benchmark of the verify step (tree-masked attention + greedy acceptance) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 0..4] [--impl reference]
+
+One "step" is one pass of the whole hot path (owl_verify_attn + owl_tree_accept) over one batch
+of seeded synthetic input.  Prints ONE JSON line.  `value` is algorithmic HBM bytes of a step
+(K/V of every visible position + Q + out + LSE + logits) divided by the device time of a step,
+summed over ranks: the "achieved HBM GB/s" half of the headline metric; `verify_step_us` is the
+other half.  Inputs are resident in HBM when the timed region starts and rotate over enough
+copies that no step finds its inputs in L2.  `e2e` is the same metric through the host-buffer
+C-ABI call, host<->device copies inside the timed region.  `--impl reference` times the CPU
+oracle on bounded samples of the same workload instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+L2_BYTES = 126 * 1024 * 1024
+METRIC = "verify_step_hbm_gbs"
+
+
+# ----------------------------------------------------------------------------- helpers
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            pk = json.load(f)
+        return float(pk["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+def algorithmic_bytes(wl):
+    """Bytes a step must move: K and V of every visible position, Q, out, LSE, block table, logits."""
+    sp = wl.spec
+    N, Hq, D = wl.q.shape
+    kv = sp.kv_bytes()
+    qo = 2 * N * Hq * D * 2 + N * Hq * 4
+    tab = int(sum((int(l) + n + sp.page_size - 1) // sp.page_size for l, n in zip(sp.ctx_lens, sp.node_counts()))) * 4 * sp.num_kv_heads
+    attn = kv + qo + tab
+    logits = sp.logits_bytes()
+    return attn, logits
+
+
+def ncu_traffic(workload_name):
+    """DRAM bytes per launch of the attention kernel from the committed ncu summary, if present."""
+    path = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            t = json.load(f)
+        return t.get(workload_name)
+    return None
+
+
+class ClockSampler(threading.Thread):
+    """Polls SM clock and throttle reasons through NVML (read-only) while the timed region runs."""
+
+    def __init__(self, index: int, period: float = 0.02):
+        super().__init__(daemon=True)
+        self.index, self.period = index, period
+        self.samples, self.reasons = [], set()
+        self.max_mhz = None
+        self._stop_evt = threading.Event()
+        self.active = threading.Event()
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.nv = None
+
+    def run(self):
+        if self.nv is None:
+            return
+        nv = self.nv
+        names = {nv.nvmlClocksEventReasonHwSlowdown: "hw_slowdown",
+                 nv.nvmlClocksEventReasonHwThermalSlowdown: "hw_thermal_slowdown",
+                 nv.nvmlClocksEventReasonSwThermalSlowdown: "sw_thermal_slowdown",
+                 nv.nvmlClocksEventReasonSwPowerCap: "sw_power_cap"}
+        while not self._stop_evt.is_set():
+            if self.active.is_set():
+                try:
+                    self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                    r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                    for bit, name in names.items():
+                        if r & bit:
+                            self.reasons.add(name)
+                except Exception:
+                    pass
+            time.sleep(self.period)
+
+    def stop(self):
+        self._stop_evt.set()
+
+    def summary(self):
+        med = int(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def physical_gpu_index(local_rank: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_rank])
+        except Exception:
+            return local_rank
+    return local_rank
+
+
+# ----------------------------------------------------------------------------- CPU oracle timing
+
+class OracleTimer:
+    """Times the CPU oracle, as it stands, on bounded samples of the workload's rows.
+
+    A sample is a set of (node, head) attention rows drawn without replacement plus the arg-max and
+    acceptance walk of a few logits rows; its per-row cost is scaled to the whole step.
+    """
+
+    def __init__(self, wl):
+        import oracle
+        self.oracle, self.wl = oracle, wl
+        self.N, self.Hq, _ = wl.q.shape
+        self.total_rows = self.N * self.Hq
+        self.threads = oracle.num_threads()
+        self.rng = np.random.default_rng(0)
+        self.row_cost = None
+
+    def _attn(self, nrows):
+        wl = self.wl
+        idx = self.rng.choice(self.total_rows, size=min(nrows, self.total_rows), replace=False)
+        rn, rh = (idx // self.Hq).astype(np.int32), (idx % self.Hq).astype(np.int32)
+        t0 = time.perf_counter()
+        self.oracle.verify_attn(wl.q, wl.k_cache, wl.v_cache, wl.block_table, wl.ctx_lens, wl.node_offsets,
+                                wl.tree_parent, wl.sm_scale, rows=(rn, rh))
+        return time.perf_counter() - t0, len(idx)
+
+    def sample(self, budget_s: float):
+        """Returns (estimated seconds of a whole step, seconds actually spent, description)."""
+        wl = self.wl
+        if self.row_cost is None:                     # untimed calibration: one row per thread
+            t, n = self._attn(self.threads)
+            self.row_cost = t / n
+        n_rows = int(min(self.total_rows, max(self.threads, budget_s * 0.8 / max(self.row_cost, 1e-9))))
+        n_rows = max(self.threads, (n_rows // self.threads) * self.threads)
+        t_attn, n_attn = self._attn(n_rows)
+        n_lg = min(self.N, self.threads)
+        t0 = time.perf_counter()
+        self.oracle.tree_accept(wl.logits[:n_lg], wl.draft_tokens[:n_lg], np.arange(n_lg + 1, dtype=np.int32),
+                                np.full(n_lg, -1, np.int32), 64)
+        t_acc = time.perf_counter() - t0
+        est = t_attn * self.total_rows / n_attn + t_acc * self.N / n_lg
+        desc = (f"{n_attn} of {self.total_rows} (node, head) attention rows + arg-max/accept of {n_lg} of {self.N} "
+                f"logits rows, cost scaled to the whole step")
+        return est, t_attn + t_acc, desc
+
+
+# ----------------------------------------------------------------------------- main arms
+
+def run_reference(args, rank, world):
+    from paper_2510_07535_b200 import workloads as W
+    if rank != 0:
+        return
+    spec = W.config_spec(args.workload)
+    wl = W.generate(spec)
+    attn_b, logit_b = algorithmic_bytes(wl)
+    timer = OracleTimer(wl)
+    # bounded samples: the whole --steps/--warmup run stays within a few minutes
+    budget = min(args.cpu_budget, max(0.05, 150.0 / max(1, args.steps + args.warmup)))
+    for _ in range(args.warmup):
+        timer.sample(budget)
+    ests, desc = [], ""
+    for _ in range(args.steps):
+        est, _, desc = timer.sample(budget)
+        ests.append(est)
+    threads = timer.threads
+    est = float(np.mean(ests))
+    value = (attn_b + logit_b) / est / 1e9
+    line = {
+        "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": est * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic", "impl": "reference",
+        "config": {"workload": spec.name, "note": "CPU oracle (plain fp64 C, OpenMP) on sampled rows of the same workload"},
+        "cpu_baseline": {"value": value, "unit": "GB/s", "cores": threads, "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "verify_step_us": est * 1e6, "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def run_gpu(args, rank, world, local_rank):
+    import torch
+    import torch.distributed as dist
+    from paper_2510_07535_b200 import OwlContext, workloads as W
+    from paper_2510_07535_b200.runner import DeviceWorkload, dims_of
+
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    def max_over_ranks(x: float) -> float:
+        if world == 1:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    spec = W.config_spec(args.workload)
+    if world > 1:
+        spec.seed += 1000 * rank       # replicas: every rank verifies its own batch
+    wl = W.generate(spec)
+    attn_b, logit_b = algorithmic_bytes(wl)
+    step_bytes = attn_b + logit_b
+    # rotate over enough input copies that a step never finds its K/V or logits in L2
+    copies = max(2, int(np.ceil(4 * L2_BYTES / step_bytes)) + 1) if step_bytes < 8 * L2_BYTES else 2
+    reps = [DeviceWorkload.upload(wl, dev) for _ in range(copies)]
+    ctx = OwlContext(dims_of(wl), dev)
+
+    sampler = ClockSampler(physical_gpu_index(local_rank))
+    sampler.start()
+
+    def run_steps(k, first=0):
+        for i in range(k):
+            reps[(first + i) % copies].step(ctx)
+
+    # ---- device-resident timing
+    run_steps(args.warmup)
+    assert ctx.owl_get_status() == 0
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches0 = ctx.launch_count()
+    barrier()
+    sampler.active.set()
+    ev0.record()
+    run_steps(args.steps, args.warmup)
+    ev1.record()
+    barrier()
+    sampler.active.clear()
+    launches = ctx.launch_count() - launches0
+    assert ctx.owl_get_status() == 0
+    sec = max_over_ranks(ev0.elapsed_time(ev1) * 1e-3)
+    step_s = sec / args.steps
+
+    # ---- per-kernel device times of the same steps (events between the kernels, same stream)
+    ctx.set_profiling(True)
+    kt = np.zeros(4)
+    kn = min(args.steps, 200)
+    for i in range(kn):
+        reps[i % copies].step(ctx)
+        kt += np.array(ctx.last_kernel_times())
+    ctx.set_profiling(False)
+    kt /= kn
+
+    # ---- end to end through the host-buffer C-ABI call (pinned host memory)
+    pin = lambda a, dt=None: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+    bf = lambda a: torch.from_numpy(a.view(np.int16)).view(torch.bfloat16).pin_memory()
+    N, Hq, D = wl.q.shape
+    B = spec.batch
+    h_in = dict(q=bf(wl.q), k=bf(wl.k_cache), v=bf(wl.v_cache), bt=pin(wl.block_table), cl=pin(wl.ctx_lens),
+                no=pin(wl.node_offsets), tp=pin(wl.tree_parent), lg=pin(wl.logits), dt=pin(wl.draft_tokens))
+    h_out = dict(out=torch.empty((N, Hq, D), dtype=torch.bfloat16).pin_memory(),
+                 lse=torch.empty((N, Hq), dtype=torch.float32).pin_memory(),
+                 alen=torch.empty(B, dtype=torch.int32).pin_memory(),
+                 path=torch.empty((B, 64), dtype=torch.int32).pin_memory(),
+                 bonus=torch.empty(B, dtype=torch.int32).pin_memory())
+    h2d = sum(t.numel() * t.element_size() for t in h_in.values())
+    d2h = sum(t.numel() * t.element_size() for t in h_out.values())
+
+    def host_step():
+        return ctx.owl_verify_step_host(reps[0].dims, h_in["q"], h_in["k"], h_in["v"], h_in["bt"], h_in["cl"], h_in["no"],
+                                        h_in["tp"], h_in["lg"], h_in["dt"], h_out["out"], h_out["lse"], h_out["alen"],
+                                        h_out["path"], h_out["bonus"])
+    e2e_steps = max(3, min(args.steps, int(2.0 / max(h2d / 20e9, 1e-4))))
+    for _ in range(3):
+        assert host_step() == 0
+    barrier()
+    ev0.record()
+    for _ in range(e2e_steps):
+        host_step()
+    ev1.record()
+    barrier()
+    e2e_s = max_over_ranks(ev0.elapsed_time(ev1) * 1e-3) / e2e_steps
+    sampler.stop()
+
+    # ---- CPU oracle beside it (rank 0, N=1 only)
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        timer = OracleTimer(wl)
+        est, _, desc = timer.sample(args.cpu_budget)
+        cpu = {"value": step_bytes / est / 1e9, "unit": "GB/s", "cores": timer.threads, "kind": "oracle", "sample": desc,
+               "est_step_s": est}
+
+    if rank == 0:
+        peak, peak_kind = measured_peaks()
+        achieved = attn_b / kt[0] / 1e9 if kt[0] > 0 else None
+        line = {
+            "metric": METRIC, "value": world * step_bytes / step_s / 1e9, "unit": "GB/s", "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": step_s * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": spec.name, "batch": B, "ctx_lens": [int(min(spec.ctx_lens)), int(max(spec.ctx_lens))],
+                       "nodes": int(wl.total_nodes), "q_heads": spec.num_q_heads, "kv_heads": spec.num_kv_heads,
+                       "vocab": spec.vocab, "parallelism": "replicas only" if world > 1 else "single GPU",
+                       "l2": f"rotating {copies} input copies ({copies * step_bytes / 1e6:.0f} MB > L2)"},
+            "verify_step_us": step_s * 1e6,
+            "frac_of_hbm_peak": step_bytes / step_s / 1e9 / peak,
+            "kernel_us": {"verify_attn": kt[0] * 1e6, "combine": kt[1] * 1e6, "argmax": kt[2] * 1e6, "accept_walk": kt[3] * 1e6},
+            "bytes_per_step": {"attention": attn_b, "logits": logit_b},
+            "roofline": {"bound": "hbm", "kernel": "verify_attn", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                         "frac": achieved / peak if achieved else None, "peak_kind": f"of {peak_kind}",
+                         "traffic": ncu_traffic(spec.name)},
+            "accept_gbs": logit_b / (kt[2] + kt[3]) / 1e9 if kt[2] > 0 else None,
+            "e2e": {"value": world * step_bytes / e2e_s / 1e9, "unit": "GB/s", "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h, "us_per_step": e2e_s * 1e6, "steps": e2e_steps},
+            "gpu_launches": launches,
+            "clocks": sampler.summary(),
+        }
+        if cpu:
+            line["cpu_baseline"] = cpu
+        print(json.dumps(line), flush=True)
+    ctx.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=500)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--workload", type=int, default=1, help="benchmark configuration 0..4 (default 1: 8B shape, 32K context, 32-node tree)")
+    ap.add_argument("--impl", default="owl", choices=["owl", "reference"])
+    ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of CPU oracle work per sample")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "owl" else args.warmup
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+    else:
+        run_gpu(args, rank, world, local_rank)
+
+
+if __name__ == "__main__":
+    main()

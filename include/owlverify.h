@@ -88,7 +88,7 @@ typedef struct owl_dims {
     int32_t max_pages_per_seq; /* row stride of block_table                                     */
     int32_t num_pages;         /* pages in k_cache / v_cache; block_table entries are checked   */
     int32_t vocab;             /* V (owl_tree_accept only; may be 0 for attention-only use)     */
-    int32_t path_stride;       /* row stride of accept_path, >= deepest path + 1 (64 always is) */
+    int32_t path_stride;       /* row stride of accept_path, >= max_nodes (64 always is)        */
     float sm_scale;            /* multiplies q.k before the softmax; always explicit            */
 } owl_dims;
 
@@ -139,6 +139,23 @@ int owl_tree_accept(owl_ctx* ctx, const owl_dims* dims, const float* logits,
                     const int32_t* draft_tokens, const int32_t* node_offsets,
                     const int32_t* tree_parent, int32_t* accept_len, int32_t* accept_path,
                     int32_t* bonus_token, int32_t* node_argmax, void* stream);
+
+/*
+ * One whole verify step from HOST memory: copies every input to device staging buffers owned by
+ * the context (grown on demand, so the first call at a given size allocates), runs
+ * owl_verify_attn and owl_tree_accept, copies the results back and synchronises `stream`.
+ * Every tensor pointer here is a HOST pointer (page-locked memory makes the copies asynchronous
+ * and fast; pageable memory works).  Shapes and meanings are those of the two calls above;
+ * lse_h may be NULL.  Returns a host-detected error, else the device status word (as
+ * owl_get_status, which it clears).  Meant for callers without device buffers of their own and
+ * for end-to-end timing; a serving loop keeps the KV cache resident and uses the device calls.
+ */
+int owl_verify_step_host(owl_ctx* ctx, const owl_dims* dims, const void* q_h, const void* k_cache_h,
+                         const void* v_cache_h, const int32_t* block_table_h, const int32_t* ctx_lens_h,
+                         const int32_t* node_offsets_h, const int32_t* tree_parent_h,
+                         const float* logits_h, const int32_t* draft_tokens_h, void* out_h, float* lse_h,
+                         int32_t* accept_len_h, int32_t* accept_path_h, int32_t* bonus_token_h,
+                         void* stream);
 
 /* Synchronise `stream`, return the device status word of the calls issued on this
  * context since the last owl_get_status (OWL_OK, OWL_ERR_BAD_TREE, OWL_ERR_BAD_PAGE,

@@ -50,6 +50,8 @@ def load_library() -> ctypes.CDLL:
     lib.owl_verify_attn.argtypes = [vp, dp] + [vp] * 10
     lib.owl_tree_accept.restype = i32
     lib.owl_tree_accept.argtypes = [vp, dp] + [vp] * 9
+    lib.owl_verify_step_host.restype = i32
+    lib.owl_verify_step_host.argtypes = [vp, dp] + [vp] * 15
     lib.owl_get_status.restype = i32
     lib.owl_get_status.argtypes = [vp, vp]
     lib.owl_status_string.restype = ctypes.c_char_p
@@ -134,6 +136,20 @@ class OwlContext:
             _ptr(node_argmax, torch.int32, dev, "node_argmax"), _stream(dev))
         if check and rc != OWL_OK:
             raise OwlError(rc, "owl_tree_accept", self.last_error())
+        return rc
+
+    def owl_verify_step_host(self, dims: OwlDims, q, k_cache, v_cache, block_table, ctx_lens, node_offsets,
+                             tree_parent, logits, draft_tokens, out, lse, accept_len, accept_path, bonus_token) -> int:
+        """All tensors are HOST (CPU, ideally pinned) torch tensors; returns the device status word."""
+        cpu = torch.device("cpu")
+        args = [(q, torch.bfloat16), (k_cache, torch.bfloat16), (v_cache, torch.bfloat16), (block_table, torch.int32),
+                (ctx_lens, torch.int32), (node_offsets, torch.int32), (tree_parent, torch.int32),
+                (logits, torch.float32), (draft_tokens, torch.int32), (out, torch.bfloat16), (lse, torch.float32),
+                (accept_len, torch.int32), (accept_path, torch.int32), (bonus_token, torch.int32)]
+        ptrs = [_ptr(t, dt, cpu, f"arg{i}") for i, (t, dt) in enumerate(args)]
+        rc = self.lib.owl_verify_step_host(self._h, ctypes.byref(dims), *ptrs, _stream(self.device))
+        if rc in (-1, -2, -3, -7):
+            raise OwlError(rc, "owl_verify_step_host", self.last_error())
         return rc
 
     def owl_get_status(self) -> int:

@@ -33,6 +33,8 @@ struct owl_ctx {
     cudaEvent_t ev[6] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
     bool ev_attn_valid = false, ev_accept_valid = false;
     char err[256] = {0};
+    // device staging of owl_verify_step_host (grown on demand)
+    struct Staging { void* p = nullptr; size_t cap = 0; } stg[16];
 };
 
 namespace {
@@ -166,6 +168,7 @@ int owl_destroy(owl_ctx* ctx) {
     cudaFree(ctx->status);
     cudaFree(ctx->seq_bad);
     cudaFree(ctx->part_keys);
+    for (auto& s : ctx->stg) cudaFree(s.p);
     for (auto& ev : ctx->ev)
         if (ev) cudaEventDestroy(ev);
     delete ctx;
@@ -279,6 +282,56 @@ int owl_tree_accept(owl_ctx* ctx, const owl_dims* d, const float* logits, const 
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(ctx, e, "owl_tree_accept launch");
     return OWL_OK;
+}
+
+int owl_verify_step_host(owl_ctx* ctx, const owl_dims* d, const void* q_h, const void* k_h, const void* v_h,
+                         const int32_t* bt_h, const int32_t* cl_h, const int32_t* no_h, const int32_t* tp_h,
+                         const float* logits_h, const int32_t* dt_h, void* out_h, float* lse_h, int32_t* alen_h,
+                         int32_t* apath_h, int32_t* bonus_h, void* stream_) {
+    if (!ctx) return OWL_ERR_INVALID_ARG;
+    int rc = check_dims(d, true, true);
+    if (rc != OWL_OK) return rc;
+    if (!q_h || !k_h || !v_h || !bt_h || !cl_h || !tp_h || !logits_h || !dt_h || !out_h || !alen_h || !apath_h || !bonus_h)
+        return OWL_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const size_t N = d->total_nodes, B = d->batch;
+    const size_t q_bytes = N * d->num_q_heads * kHeadDim * 2;
+    const size_t kv_bytes = (size_t)d->num_pages * d->num_kv_heads * d->page_size * kHeadDim * 2;
+    const size_t sizes[16] = {q_bytes, kv_bytes, kv_bytes, B * d->max_pages_per_seq * 4, B * 4, (B + 1) * 4, N * 4,
+                              N * (size_t)d->vocab * 4, N * 4,
+                              /* outputs */ q_bytes, N * d->num_q_heads * 4, B * 4, B * (size_t)d->path_stride * 4, B * 4, 0, 0};
+    for (int i = 0; i < 14; ++i) {
+        if (ctx->stg[i].cap < sizes[i]) {
+            cudaError_t e = cudaStreamSynchronize(stream);
+            if (e == cudaSuccess) { cudaFree(ctx->stg[i].p); ctx->stg[i].p = nullptr; ctx->stg[i].cap = 0; e = cudaMalloc(&ctx->stg[i].p, sizes[i]); }
+            if (e != cudaSuccess) return cuda_fail(ctx, e, "owl_verify_step_host staging");
+            ctx->stg[i].cap = sizes[i];
+        }
+    }
+    const void* src[9] = {q_h, k_h, v_h, bt_h, cl_h, no_h, tp_h, logits_h, dt_h};
+    for (int i = 0; i < 9; ++i) {
+        if (!src[i]) continue;  // node_offsets may be NULL
+        cudaError_t e = cudaMemcpyAsync(ctx->stg[i].p, src[i], sizes[i], cudaMemcpyHostToDevice, stream);
+        if (e != cudaSuccess) return cuda_fail(ctx, e, "owl_verify_step_host H2D");
+    }
+    auto dev = [&](int i) { return ctx->stg[i].p; };
+    const int32_t* no_d = no_h ? static_cast<const int32_t*>(dev(5)) : nullptr;
+    rc = owl_verify_attn(ctx, d, dev(0), dev(1), dev(2), static_cast<const int32_t*>(dev(3)),
+                         static_cast<const int32_t*>(dev(4)), no_d, static_cast<const int32_t*>(dev(6)), dev(9),
+                         static_cast<float*>(dev(10)), stream_);
+    if (rc != OWL_OK) return rc;
+    rc = owl_tree_accept(ctx, d, static_cast<const float*>(dev(7)), static_cast<const int32_t*>(dev(8)), no_d,
+                         static_cast<const int32_t*>(dev(6)), static_cast<int32_t*>(dev(11)),
+                         static_cast<int32_t*>(dev(12)), static_cast<int32_t*>(dev(13)), nullptr, stream_);
+    if (rc != OWL_OK) return rc;
+    void* dst[5] = {out_h, lse_h, alen_h, apath_h, bonus_h};
+    for (int i = 0; i < 5; ++i) {
+        if (!dst[i]) continue;
+        cudaError_t e = cudaMemcpyAsync(dst[i], dev(9 + i), sizes[9 + i], cudaMemcpyDeviceToHost, stream);
+        if (e != cudaSuccess) return cuda_fail(ctx, e, "owl_verify_step_host D2H");
+    }
+    return owl_get_status(ctx, stream_);
 }
 
 int owl_get_status(owl_ctx* ctx, void* stream_) {
