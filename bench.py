@@ -204,7 +204,7 @@ def run_reference(args, rank, world):
 def run_gpu(args, rank, world, local_rank):
     import torch
     import torch.distributed as dist
-    from paper_2510_07535_b200 import OwlContext, workloads as W
+    from paper_2510_07535_b200 import OwlContext, replicas, workloads as W
     from paper_2510_07535_b200.runner import DeviceWorkload, dims_of
 
     torch.cuda.set_device(local_rank)
@@ -218,15 +218,11 @@ def run_gpu(args, rank, world, local_rank):
         torch.cuda.synchronize(dev)
 
     def max_over_ranks(x: float) -> float:
-        if world == 1:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return replicas.aggregate(0.0, x, dev)[1]
 
     spec = W.config_spec(args.workload)
     if world > 1:
-        spec.seed += 1000 * rank       # replicas: every rank verifies its own batch
+        spec.seed = replicas.replica_seed(spec.seed, rank)   # replicas: every rank verifies its own batch
     wl = W.generate(spec)
     attn_b, logit_b = algorithmic_bytes(wl)
     step_bytes = attn_b + logit_b
