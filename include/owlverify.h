@@ -157,6 +157,43 @@ int owl_verify_step_host(owl_ctx* ctx, const owl_dims* dims, const void* q_h, co
                          int32_t* accept_len_h, int32_t* accept_path_h, int32_t* bonus_token_h,
                          void* stream);
 
+/*
+ * Greedy tree acceptance for callers that cannot allocate device memory.  (The paper has no
+ * counterpart to this call: it computes exactly what owl_tree_accept computes and exists only
+ * because of how some programs manage memory.)
+ *
+ * Who needs it: an inference server that gave the whole GPU to its own pool at start-up, a
+ * plug-in that must stay inside its host's memory budget, or any code on a path where
+ * cudaMalloc - and the device-wide synchronisation it can imply - is forbidden.  Such callers
+ * cannot use owl_create, which allocates a workspace.  This call takes no context and allocates
+ * nothing, neither with cudaMalloc nor through any library: its scratch (one 64-bit arg-max key
+ * per logits row and 8192-float vocabulary chunk, plus the status word) is a fixed array inside
+ * the library image.  The price: every GPU on which the library is loaded holds that array,
+ * (OWL_STATIC_MAX_KEYS + 32) * 8 bytes = 128.25 KiB, until the process exits.
+ *
+ * Limit: total_nodes * ceil(vocab / 8192) <= OWL_STATIC_MAX_KEYS (e.g. 1024 nodes at a 128256-entry
+ * vocabulary); anything larger returns OWL_ERR_TOO_LARGE and launches nothing.
+ *
+ * Arguments are those of owl_tree_accept (device pointers, caller-owned), without the context, plus
+ * device_status: a device int32 the call first clears and the kernels then set to OWL_ERR_BAD_TREE
+ * if a tree is malformed (that sequence's outputs stay unwritten).  NULL keeps the status in the
+ * library's own array, where nobody can read it.  The work runs on the CURRENT device, on `stream`,
+ * asynchronously.
+ *
+ * Sharing: all calls on a device use the same array.  Calls queued on one stream are safe one after
+ * another (a call overwrites every key before it reads it, so stale contents never matter); calls
+ * that can overlap on the GPU - different streams, different threads - race on it and must be
+ * serialised by the caller.
+ *
+ * First call: the first call made on each device looks up the array's device address
+ * (cudaGetSymbolAddress).  Make that first call outside any stream capture.
+ */
+#define OWL_STATIC_MAX_KEYS 16384
+int owl_tree_accept_static(const owl_dims* dims, const float* logits, const int32_t* draft_tokens,
+                           const int32_t* node_offsets, const int32_t* tree_parent, int32_t* accept_len,
+                           int32_t* accept_path, int32_t* bonus_token, int32_t* node_argmax,
+                           int32_t* device_status, void* stream);
+
 /* Synchronise `stream`, return the device status word of the calls issued on this
  * context since the last owl_get_status (OWL_OK, OWL_ERR_BAD_TREE, OWL_ERR_BAD_PAGE,
  * OWL_ERR_TIMEOUT; the first error wins) and clear it. */

@@ -6,4 +6,5 @@ acceptance, as hand-written sm_100a CUDA kernels behind the C ABI of ``include/o
 ``build`` compiles the library.  Nothing here computes on the CPU.
 """
 from . import workloads  # noqa: F401
-from .binding import OwlContext, OwlDims, OwlError, load_library, make_dims, status_string  # noqa: F401
+from .binding import (OwlContext, OwlDims, OwlError, load_library, make_dims, owl_tree_accept_static,  # noqa: F401
+                      status_string)

@@ -50,6 +50,8 @@ def load_library() -> ctypes.CDLL:
     lib.owl_verify_attn.argtypes = [vp, dp] + [vp] * 10
     lib.owl_tree_accept.restype = i32
     lib.owl_tree_accept.argtypes = [vp, dp] + [vp] * 9
+    lib.owl_tree_accept_static.restype = i32
+    lib.owl_tree_accept_static.argtypes = [dp] + [vp] * 10
     lib.owl_verify_step_host.restype = i32
     lib.owl_verify_step_host.argtypes = [vp, dp] + [vp] * 15
     lib.owl_get_status.restype = i32
@@ -170,6 +172,30 @@ class OwlContext:
         if rc != OWL_OK:
             raise OwlError(rc, "owl_last_kernel_times")
         return list(t)
+
+
+STATIC_MAX_KEYS = 16384   # OWL_STATIC_MAX_KEYS of owlverify.h
+
+
+def owl_tree_accept_static(dims: OwlDims, logits, draft_tokens, node_offsets, tree_parent, accept_len, accept_path,
+                           bonus_token, node_argmax=None, device_status=None, check: bool = True) -> int:
+    """Acceptance without a context and without any device allocation inside the library: for callers
+    whose memory is managed elsewhere and who therefore cannot create an ``OwlContext``.  The tensors
+    (allocated by the caller, as always) must live on the current CUDA device; scratch is the library's
+    fixed array, shared by every call on that device, so overlapping calls must be serialised by the
+    caller.  ``device_status`` (optional int32[1] on the device) receives 0 or OWL_ERR_BAD_TREE."""
+    lib = load_library()
+    dev = torch.device("cuda", torch.cuda.current_device())
+    rc = lib.owl_tree_accept_static(
+        ctypes.byref(dims), _ptr(logits, torch.float32, dev, "logits"),
+        _ptr(draft_tokens, torch.int32, dev, "draft_tokens"), _ptr(node_offsets, torch.int32, dev, "node_offsets"),
+        _ptr(tree_parent, torch.int32, dev, "tree_parent"), _ptr(accept_len, torch.int32, dev, "accept_len"),
+        _ptr(accept_path, torch.int32, dev, "accept_path"), _ptr(bonus_token, torch.int32, dev, "bonus_token"),
+        _ptr(node_argmax, torch.int32, dev, "node_argmax"), _ptr(device_status, torch.int32, dev, "device_status"),
+        _stream(dev))
+    if check and rc != OWL_OK:
+        raise OwlError(rc, "owl_tree_accept_static")
+    return rc
 
 
 def status_string(code: int) -> str:

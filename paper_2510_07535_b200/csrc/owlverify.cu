@@ -5,6 +5,7 @@
 
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 
 #include "accept.cuh"
@@ -372,3 +373,92 @@ int owl_last_kernel_times(owl_ctx* ctx, void* stream_, double t[4]) {
 }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------------------------
+// owl_tree_accept_static: greedy tree acceptance for callers that must not allocate.
+//
+// Some hosts of this library cannot call cudaMalloc at the point where they verify a draft: a
+// serving engine that handed the whole device to its own pool allocator at start-up, a plug-in
+// running inside someone else's memory budget, code on a latency path where an allocation (and
+// the implicit device synchronisation it may bring) is not allowed.  owl_create allocates, so
+// those callers cannot own an owl_ctx.  For them the arg-max scratch (one 64-bit key per logits
+// row and 8192-float vocabulary chunk) and the device status word live in the fixed array below,
+// which is part of the loaded library image: every device that loads the library holds its
+// (OWL_STATIC_MAX_KEYS + 32) * 8 bytes until the process exits, whether or not this entry point is ever called.
+//
+// The array's name is only a host-side handle here; the device address handed to the kernels
+// comes from cudaGetSymbolAddress, looked up once per device with that device current.
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+constexpr int kStaticMaxKeys = OWL_STATIC_MAX_KEYS;            // (row, chunk) keys
+constexpr int kStaticStatusWords = 32;                         // one 256-byte line for the status word
+constexpr int kStaticMaxDevices = 64;
+
+static __device__ __align__(256) unsigned long long g_accept_scratch[kStaticMaxKeys + kStaticStatusWords];
+
+unsigned long long* g_static_addr[kStaticMaxDevices] = {nullptr};
+bool g_static_ready[kStaticMaxDevices] = {false};
+std::mutex g_static_mutex;
+
+// Device address of g_accept_scratch on the current device `dev`; looked up on first use.
+cudaError_t static_scratch(int dev, unsigned long long** out) {
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_ready[dev]) {
+        void* p = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(&p, g_accept_scratch);
+        if (e != cudaSuccess) return e;
+        g_static_addr[dev] = static_cast<unsigned long long*>(p);
+        g_static_ready[dev] = true;
+    }
+    *out = g_static_addr[dev];
+    return cudaSuccess;
+}
+
+}  // namespace
+
+extern "C" int owl_tree_accept_static(const owl_dims* d, const float* logits, const int32_t* draft_tokens,
+                                      const int32_t* node_offsets, const int32_t* tree_parent, int32_t* accept_len,
+                                      int32_t* accept_path, int32_t* bonus_token, int32_t* node_argmax,
+                                      int32_t* device_status, void* stream_) {
+    int rc = check_dims(d, false, true);
+    if (rc != OWL_OK) return rc;
+    if (!logits || !draft_tokens || !tree_parent || !accept_len || !accept_path || !bonus_token) return OWL_ERR_INVALID_ARG;
+    if (!node_offsets && d->total_nodes % d->batch != 0) return OWL_ERR_INVALID_ARG;
+    if (d->total_nodes > 65535) return OWL_ERR_UNSUPPORTED;
+    const int chunks = (d->vocab + kArgmaxChunk - 1) / kArgmaxChunk;
+    if ((long long)d->total_nodes * chunks > kStaticMaxKeys) return OWL_ERR_TOO_LARGE;   // beyond the fixed scratch
+
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kStaticMaxDevices) return OWL_ERR_CUDA;
+    unsigned long long* scratch = nullptr;
+    if (static_scratch(dev, &scratch) != cudaSuccess) { cudaGetLastError(); return OWL_ERR_CUDA; }
+    int32_t* status = device_status ? device_status : reinterpret_cast<int32_t*>(scratch + kStaticMaxKeys);
+
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    // The keys need no clearing (every key a call reads it has written first); the status word does.
+    if (cudaMemsetAsync(status, 0, sizeof(int32_t), stream) != cudaSuccess) { cudaGetLastError(); return OWL_ERR_CUDA; }
+    AcceptParams p{};
+    p.logits = logits;
+    p.draft_tokens = draft_tokens;
+    p.node_offsets = node_offsets;
+    p.tree_parent = tree_parent;
+    p.accept_len = accept_len;
+    p.accept_path = accept_path;
+    p.bonus_token = bonus_token;
+    p.node_argmax = node_argmax;
+    p.part_keys = scratch;
+    p.chunks = chunks;
+    p.status = status;
+    p.batch = d->batch;
+    p.total_nodes = d->total_nodes;
+    p.nodes_uniform = d->total_nodes / d->batch;
+    p.max_nodes = d->max_nodes;
+    p.vocab = d->vocab;
+    p.path_stride = d->path_stride;
+    dim3 grid((unsigned)chunks, (unsigned)d->total_nodes);
+    argmax_partial_kernel<<<grid, kArgmaxThreads, 0, stream>>>(p);
+    accept_walk_kernel<<<d->batch, kMaxNodes, 0, stream>>>(p);
+    if (cudaGetLastError() != cudaSuccess) return OWL_ERR_CUDA;
+    return OWL_OK;
+}
