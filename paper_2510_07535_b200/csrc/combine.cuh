@@ -9,7 +9,10 @@ namespace owl {
 
 constexpr int kCombineWarps = 8;
 
-template <int TileKeys, int RowsPerBlock>
+// kTwoSlots = false: the partial of (CTA c, unit u) sits in slot c + u.
+// kTwoSlots = true:  a CTA stores at most two partials (only the first and the last unit of its
+//                    piece can be cut): slot 2c if its piece starts inside the unit, else 2c + 1.
+template <int TileKeys, int RowsPerBlock, bool kTwoSlots = false>
 __global__ void __launch_bounds__(kCombineWarps * 32) combine_kernel(const AttnParams p) {
     __shared__ long long s_tile[kMaxBatch + 1];
     __shared__ int s_unit[kMaxBatch + 1];
@@ -42,9 +45,12 @@ __global__ void __launch_bounds__(kCombineWarps * 32) combine_kernel(const AttnP
     const int c0 = part.owner(t0), c1 = part.owner(t0 + s.tiles - 1);
     if (c0 == c1) return;  // a single CTA saw every key of this unit and wrote the result itself
 
+    auto slot_of = [&](int c) -> long long {
+        return kTwoSlots ? 2ll * c + (part.begin(c) < t0 ? 1 : 0) : (long long)c + unit;
+    };
     float mx = -INFINITY;
     for (int c = c0 + lane; c <= c1; c += 32)
-        mx = fmaxf(mx, p.part_lse[((long long)c + unit) * p.rows_per_slot + lrow]);
+        mx = fmaxf(mx, p.part_lse[slot_of(c) * p.rows_per_slot + lrow]);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
 
@@ -52,7 +58,7 @@ __global__ void __launch_bounds__(kCombineWarps * 32) combine_kernel(const AttnP
     float sum = 0.f;
     if (mx > -INFINITY) {
         for (int c = c0; c <= c1; ++c) {
-            const long long prow = ((long long)c + unit) * p.rows_per_slot + lrow;
+            const long long prow = slot_of(c) * p.rows_per_slot + lrow;
             const float w = __expf(p.part_lse[prow] - mx);
             const float4 v = *reinterpret_cast<const float4*>(p.part_o + prow * kHeadDim + lane * 4);
             acc.x += w * v.x; acc.y += w * v.y; acc.z += w * v.z; acc.w += w * v.w;

@@ -4,6 +4,7 @@
 #include <cuda_runtime.h>
 
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <mutex>
 #include <new>
@@ -12,6 +13,7 @@
 #include "combine.cuh"
 #include "owl_common.cuh"
 #include "verify_attn_mma.cuh"
+#include "verify_attn_umma.cuh"
 
 using namespace owl;
 
@@ -28,6 +30,13 @@ struct owl_ctx {
     int32_t* seq_bad = nullptr;
     unsigned long long* part_keys = nullptr;
     long long part_keys_len = 0;
+    // tcgen05 path: tensor maps over the caller's K and V caches, re-encoded when the cache changes
+    bool use_umma = true;
+    EncodeTiledFn encode = nullptr;
+    CUtensorMap kmap{}, vmap{};
+    const void* map_k = nullptr;
+    const void* map_v = nullptr;
+    int map_pages = 0, map_heads = 0, map_page_size = 0;
     int32_t epoch = 0;
     int64_t launches = 0;
     bool profiling = false;
@@ -69,7 +78,7 @@ int check_dims(const owl_dims* d, bool for_attn, bool for_accept) {
     if (for_attn) {
         if (d->num_q_heads < 1 || d->num_kv_heads < 1 || d->num_q_heads % d->num_kv_heads != 0) return OWL_ERR_INVALID_ARG;
         if (d->max_pages_per_seq < 1 || d->num_pages < 1) return OWL_ERR_INVALID_ARG;
-        if (!(d->sm_scale == d->sm_scale)) return OWL_ERR_INVALID_ARG;
+        if (!(d->sm_scale == d->sm_scale) || d->sm_scale == 0.f || d->sm_scale - d->sm_scale != 0.f) return OWL_ERR_INVALID_ARG;
         if (d->head_dim != kHeadDim) return OWL_ERR_UNSUPPORTED;
         if ((d->num_q_heads / d->num_kv_heads) * d->max_nodes > kMaxRows) return OWL_ERR_UNSUPPORTED;
         if (!(d->page_size == 16 || d->page_size == 32 || d->page_size == 64 || d->page_size == 128)) return OWL_ERR_UNSUPPORTED;
@@ -124,6 +133,13 @@ int owl_create(owl_ctx** out, int device, const owl_dims* max_dims) {
     ctx->sm_count = prop.multiProcessorCount;
     ctx->num_ctas = ctx->sm_count;
 
+    const char* path_env = getenv("OWL_ATTN_PATH");     // "mma" selects the warp-level MMA kernel (for comparison)
+    ctx->use_umma = !(path_env && strcmp(path_env, "mma") == 0);
+    if (ctx->use_umma && attn) {
+        ctx->encode = load_encode_tiled();
+        if (!ctx->encode) { delete ctx; return OWL_ERR_CUDA; }
+    }
+
     bool ok = true;
     auto alloc = [&](void** p, size_t bytes) {
         if (ok && (e = cudaMalloc(p, bytes ? bytes : 16)) != cudaSuccess) ok = false;
@@ -132,8 +148,13 @@ int owl_create(owl_ctx** out, int device, const owl_dims* max_dims) {
         const int G = max_dims->num_q_heads / max_dims->num_kv_heads;
         const int M = G * max_dims->max_nodes;
         const int row_blocks = (M + mma_path::kRows - 1) / mma_path::kRows;
-        ctx->rows_per_slot = mma_path::kRows;
-        ctx->slots = (long long)ctx->num_ctas + (long long)max_dims->batch * max_dims->num_kv_heads * row_blocks;
+        if (ctx->use_umma) {
+            ctx->rows_per_slot = umma_path::kRows;
+            ctx->slots = 2ll * ctx->num_ctas;      // a CTA stores at most two partials per call
+        } else {
+            ctx->rows_per_slot = mma_path::kRows;
+            ctx->slots = (long long)ctx->num_ctas + (long long)max_dims->batch * max_dims->num_kv_heads * row_blocks;
+        }
         alloc((void**)&ctx->part_o, (size_t)ctx->slots * ctx->rows_per_slot * kHeadDim * sizeof(float));
         alloc((void**)&ctx->part_lse, (size_t)ctx->slots * ctx->rows_per_slot * sizeof(float));
     }
@@ -150,7 +171,9 @@ int owl_create(owl_ctx** out, int device, const owl_dims* max_dims) {
     for (int i = 0; ok && i < 6; ++i) ok = cudaEventCreate(&ctx->ev[i]) == cudaSuccess;
     if (ok && attn) {
         ok = cudaFuncSetAttribute(mma_path::verify_attn_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                  mma_path::kSmemBytes) == cudaSuccess;
+                                  mma_path::kSmemBytes) == cudaSuccess &&
+             cudaFuncSetAttribute(umma_path::verify_attn_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  umma_path::kSmemBytes) == cudaSuccess;
     }
     if (!ok || cudaDeviceSynchronize() != cudaSuccess) {
         cudaGetLastError();
@@ -189,7 +212,7 @@ int owl_verify_attn(owl_ctx* ctx, const owl_dims* d, const void* q, const void* 
     const int G = d->num_q_heads / d->num_kv_heads;
     const int row_blocks = (G * d->max_nodes + mma_path::kRows - 1) / mma_path::kRows;
     if (d->batch > mx.batch || d->total_nodes > mx.total_nodes ||
-        (long long)ctx->num_ctas + (long long)d->batch * d->num_kv_heads * row_blocks > ctx->slots)
+        (!ctx->use_umma && (long long)ctx->num_ctas + (long long)d->batch * d->num_kv_heads * row_blocks > ctx->slots))
         return OWL_ERR_TOO_LARGE;
 
     DeviceGuard guard(ctx->device);
@@ -224,13 +247,34 @@ int owl_verify_attn(owl_ctx* ctx, const owl_dims* d, const void* q, const void* 
     p.num_ctas = ctx->num_ctas;
     p.sm_scale = d->sm_scale;
 
+    if (ctx->use_umma && (ctx->map_k != k_cache || ctx->map_v != v_cache || ctx->map_pages != d->num_pages ||
+                          ctx->map_heads != d->num_kv_heads || ctx->map_page_size != d->page_size)) {
+        const int rk = make_kv_tensor_map(ctx->encode, &ctx->kmap, k_cache, d->num_pages, d->num_kv_heads, d->page_size);
+        const int rv = make_kv_tensor_map(ctx->encode, &ctx->vmap, v_cache, d->num_pages, d->num_kv_heads, d->page_size);
+        if (rk != 0 || rv != 0) {
+            ctx->map_k = ctx->map_v = nullptr;
+            snprintf(ctx->err, sizeof ctx->err, "cuTensorMapEncodeTiled failed (%d, %d): caches must be 16-byte aligned", rk, rv);
+            return OWL_ERR_CUDA;
+        }
+        ctx->map_k = k_cache; ctx->map_v = v_cache;
+        ctx->map_pages = d->num_pages; ctx->map_heads = d->num_kv_heads; ctx->map_page_size = d->page_size;
+    }
+
     if (ctx->profiling) cudaEventRecord(ctx->ev[0], stream);
-    mma_path::verify_attn_mma_kernel<<<ctx->num_ctas, mma_path::kThreads, mma_path::kSmemBytes, stream>>>(p);
-    ++ctx->launches;
-    if (ctx->profiling) cudaEventRecord(ctx->ev[1], stream);
     const long long rows = (long long)d->total_nodes * d->num_q_heads;
     const unsigned grid = (unsigned)((rows + kCombineWarps - 1) / kCombineWarps);
-    combine_kernel<mma_path::kTileKeys, mma_path::kRows><<<grid, kCombineWarps * 32, 0, stream>>>(p);
+    if (ctx->use_umma) {
+        umma_path::verify_attn_umma_kernel<<<ctx->num_ctas, umma_path::kThreads, umma_path::kSmemBytes, stream>>>(
+            p, ctx->kmap, ctx->vmap);
+        ++ctx->launches;
+        if (ctx->profiling) cudaEventRecord(ctx->ev[1], stream);
+        combine_kernel<umma_path::kTileKeys, umma_path::kRows, true><<<grid, kCombineWarps * 32, 0, stream>>>(p);
+    } else {
+        mma_path::verify_attn_mma_kernel<<<ctx->num_ctas, mma_path::kThreads, mma_path::kSmemBytes, stream>>>(p);
+        ++ctx->launches;
+        if (ctx->profiling) cudaEventRecord(ctx->ev[1], stream);
+        combine_kernel<mma_path::kTileKeys, mma_path::kRows><<<grid, kCombineWarps * 32, 0, stream>>>(p);
+    }
     ++ctx->launches;
     if (ctx->profiling) { cudaEventRecord(ctx->ev[2], stream); ctx->ev_attn_valid = true; }
     cudaError_t e = cudaGetLastError();

@@ -1,0 +1,618 @@
+// Split-KV verify attention on the 5th-generation tensor cores (tcgen05.mma, accumulators in
+// tensor memory), K/V tiles staged by TMA.
+//
+// One persistent CTA per SM, 12 warps:
+//   warp 0        TMA producer: per 128-key tile, one box per (page, head) for K and for V into a
+//                 ring of 32 KB shared-memory slots (layout in kv_tensor_map.cuh)
+//   warp 1        issues every tcgen05.mma (one lane) and the commits that signal their completion
+//   warps 4-7     softmax warpgroup of stream 0   (one thread per packed row)
+//   warps 8-11    softmax warpgroup of stream 1
+// A unit is one (sequence, KV head) with M = G * n packed rows (row = node * G + head in group).
+// The two streams are two independent online-softmax pipelines, each with its own score tile S
+// (128 x 128 fp32, columns of tensor memory), its own bf16 probabilities P (written over S) and its
+// own output accumulator O (128 x 128 fp32):
+//   M > 128  ("shared"): stream s owns rows [128 s, 128 s + 128); both streams consume every K/V tile,
+//            which is therefore read from HBM and staged once for all 256 rows;
+//   M <= 128 ("split"):  both streams hold the same rows; stream s consumes the key tiles of parity s,
+//            and the two partial results are merged by their log-sum-exp when the segment ends.
+// Either way the tensor pipe always has the other stream's products to run while one stream's
+// warpgroup is in its softmax.  Per tile and stream: S = Q K^T (8 MMAs of K = 16 over the head
+// dimension), softmax warpgroup reads S, applies the tree mask on the few tiles that reach drafted
+// positions, updates the running maximum lazily (O is rescaled only when the maximum grew by more
+// than 2^8), writes P, then O += P V (8 MMAs over the keys, A operand from tensor memory, V as an
+// MN-major B operand).
+//
+// Work is cut as in owl_common.cuh (flat range of 128-key tiles over all units, equal pieces per
+// CTA); a CTA whose piece covers a whole unit writes the final bf16 output, otherwise a normalised
+// fp32 partial and its LSE for the combine kernel.
+//
+// Every mbarrier wait is bounded (sm100_ptx.cuh).  When a wait gives up, the CTA's abort flag makes
+// all later waits return at once, MMA issue and output writes stop, the loops run out (they are
+// finite), the producer waits - bounded - for its TMA copies in flight, tensor memory is freed and
+// the status word reports OWL_ERR_TIMEOUT.
+#pragma once
+
+#include "kv_tensor_map.cuh"
+#include "owl_common.cuh"
+#include "sm100_ptx.cuh"
+
+namespace owl {
+namespace umma_path {
+
+using namespace sm100;
+
+constexpr int kTileKeys = 128;
+constexpr int kRows = 256;                 // packed rows per unit (two streams of 128)
+constexpr int kThreads = 384;
+constexpr int kSlots = 5;                  // ring of K / V tiles
+constexpr int kSlotBytes = kTileKeys * kHeadDim * 2;     // 32 KB
+constexpr int kQBytes = 128 * kHeadDim * 2;              // 32 KB per 128-row block
+constexpr int kRingOff = 2 * kQBytes;
+constexpr int kAuxOff = kRingOff + kSlots * kSlotBytes;  // 224 KB
+constexpr int kAuxBytes = 3072;
+constexpr int kSmemBytes = kAuxOff + kAuxBytes;          // 232448 = 227 KB
+constexpr uint32_t kTmemCols = 512;
+constexpr float kLazyRescale = 8.0f;       // log2 units
+
+struct Aux {
+    uint64_t full[kSlots];
+    uint64_t empty[kSlots];
+    uint64_t s_full[2], p_full[2], o_done[2];
+    uint64_t q_full;
+    uint32_t tmem_base;
+    int abort_flag;
+    int seg_bad_tree;
+    int sched_b0;
+    long long sched_tile_begin;
+    long long scan_tiles[12];
+    long long total_tiles;
+    int scan_units[12];
+    int sched_unit_begin;
+    short parent[kMaxNodes];
+    unsigned long long anc[kMaxNodes];
+};
+static_assert(sizeof(Aux) <= kAuxBytes, "aux area too small");
+
+struct Segment {
+    int b, h, unit, n, L, node_base, M;
+    int tiles, tile0, tile1;
+    bool shared;
+    __device__ __forceinline__ int iters(int s) const {
+        const int T = tile1 - tile0;
+        return shared ? T : (s == 0 ? (T + 1) >> 1 : T >> 1);
+    }
+    __device__ __forceinline__ int tile(int s, int i) const { return tile0 + (shared ? i : 2 * i + s); }
+    __device__ __forceinline__ bool whole() const { return tile0 == 0 && tile1 == tiles; }
+};
+
+// Walks the CTA's piece [t, t_end) of the flat tile range unit by unit.  Every role runs its own
+// copy; all copies see the same sequence of segments.
+struct Walker {
+    int b, unit_begin;
+    long long seq_begin, t, t_end;
+    __device__ __forceinline__ bool next(const AttnParams& p, Segment& g) {
+        if (t >= t_end) return false;
+        int n = 0, L = 0, tiles = 0;
+        while (b < p.batch) {
+            n = seq_nodes(p, b);
+            L = p.ctx_lens[b];
+            const bool ok = seq_shape_ok(p, b, n, L);
+            tiles = ok ? (L + n + kTileKeys - 1) / kTileKeys : 0;
+            const long long flat = (long long)tiles * p.num_kv_heads;
+            if (t < seq_begin + flat) break;
+            seq_begin += flat;
+            unit_begin += ok ? p.num_kv_heads : 0;
+            ++b;
+        }
+        if (b >= p.batch) { t = t_end; return false; }
+        const long long local = t - seq_begin;
+        g.b = b; g.n = n; g.L = L; g.tiles = tiles;
+        g.h = (int)(local / tiles);
+        g.tile0 = (int)(local % tiles);
+        const long long left = t_end - t;
+        g.tile1 = (int)(g.tile0 + left < tiles ? g.tile0 + left : tiles);
+        g.unit = unit_begin + g.h;
+        g.node_base = seq_node_base(p, b);
+        g.M = n * p.group;
+        g.shared = g.M > 128;
+        t += g.tile1 - g.tile0;
+        return true;
+    }
+};
+
+// Block-wide: totals of the flat tile range and the first sequence of this CTA's piece.
+__device__ __forceinline__ void build_walk(const AttnParams& p, Aux* aux, Walker& w) {
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int per = (p.batch + kThreads - 1) / kThreads;
+    const int b_lo = tid * per, b_hi = min(p.batch, b_lo + per);
+    long long my_tiles = 0;
+    int my_units = 0;
+    for (int b = b_lo; b < b_hi; ++b) {
+        const int n = seq_nodes(p, b), L = p.ctx_lens[b];
+        if (seq_shape_ok(p, b, n, L)) {
+            my_tiles += (long long)((L + n + kTileKeys - 1) / kTileKeys) * p.num_kv_heads;
+            my_units += p.num_kv_heads;
+        } else {
+            report(p.status, seq_tree_shape_ok(p, b, n) ? kErrBadPage : kErrBadTree);
+            p.seq_bad[b] = p.epoch;
+        }
+    }
+    long long inc_t = my_tiles;
+    int inc_u = my_units;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const long long vt = __shfl_up_sync(0xffffffffu, inc_t, o);
+        const int vu = __shfl_up_sync(0xffffffffu, inc_u, o);
+        if (lane >= o) { inc_t += vt; inc_u += vu; }
+    }
+    if (lane == 31) { aux->scan_tiles[warp] = inc_t; aux->scan_units[warp] = inc_u; }
+    __syncthreads();
+    long long off_t = 0;
+    int off_u = 0;
+    for (int w2 = 0; w2 < warp; ++w2) { off_t += aux->scan_tiles[w2]; off_u += aux->scan_units[w2]; }
+    const long long excl_t = off_t + inc_t - my_tiles;
+    const int excl_u = off_u + inc_u - my_units;
+    if (tid == kThreads - 1) aux->total_tiles = off_t + inc_t;
+    __syncthreads();
+    Partition part;
+    part.init(aux->total_tiles, gridDim.x);
+    const long long t_begin = part.begin(blockIdx.x), t_end = part.begin(blockIdx.x + 1);
+    if (t_begin < t_end && my_tiles > 0 && t_begin >= excl_t && t_begin < excl_t + my_tiles) {
+        aux->sched_b0 = b_lo;                 // the walker skips ahead from the first sequence of this thread
+        aux->sched_tile_begin = excl_t;
+        aux->sched_unit_begin = excl_u;
+    }
+    __syncthreads();
+    w.t = t_begin;
+    w.t_end = t_end;
+    w.b = aux->sched_b0;
+    w.seq_begin = aux->sched_tile_begin;
+    w.unit_begin = aux->sched_unit_begin;
+}
+
+// ------------------------------------------------------------------------------------------ producer
+__device__ __forceinline__ void producer_loop(const AttnParams& p, const CUtensorMap* kmap, const CUtensorMap* vmap,
+                                              Aux* aux, uint32_t ring, Walker w, uint32_t& items_out) {
+    const int lane = threadIdx.x & 31;
+    volatile int* abort_flag = &aux->abort_flag;
+    const int ppt = kTileKeys >> p.page_shift;               // pages (= TMA boxes) per tile
+    const uint32_t box_bytes = (uint32_t)p.page_size * 256u;
+    const int oob = p.num_pages * p.num_kv_heads;            // a coordinate past the end: the box reads zeros
+    uint32_t item = 0;
+    Segment g;
+    while (w.next(p, g)) {
+        const int keys = g.L + g.n;
+        const int pages_valid = (keys + p.page_size - 1) >> p.page_shift;
+        const int32_t* table = p.block_table + (long long)g.b * p.max_pages_per_seq;
+        auto coord_of = [&](int t) {
+            int c = oob;
+            const int lp = t * ppt + lane;
+            if (lane < ppt && lp < pages_valid) {
+                const int pg = table[lp];
+                if ((unsigned)pg < (unsigned)p.num_pages) c = pg * p.num_kv_heads + g.h;
+                else { report(p.status, kErrBadPage); p.seq_bad[g.b] = p.epoch; }
+            }
+            return c;
+        };
+        int c_next = coord_of(g.tile0);
+        for (int t = g.tile0; t < g.tile1; ++t) {
+            const int c_cur = c_next;
+            if (t + 1 < g.tile1) c_next = coord_of(t + 1);
+#pragma unroll
+            for (int kv = 0; kv < 2; ++kv) {
+                const uint32_t slot = item % kSlots, ph = (item / kSlots) & 1u;
+                const uint32_t full = smem_u32(&aux->full[slot]);
+                const bool ok = mbar_wait(smem_u32(&aux->empty[slot]), ph ^ 1u, abort_flag);
+                if (ok) {
+                    if (lane == 0) mbar_arrive_expect_tx(full, (uint32_t)kSlotBytes);
+                    __syncwarp();
+                    if (lane < ppt)
+                        tma_load_5d(ring + slot * kSlotBytes + lane * box_bytes, kv ? vmap : kmap, full, 0, 0, 0, 0, c_cur);
+                    ++item;
+                }
+                __syncwarp();
+            }
+        }
+    }
+    items_out = item;
+}
+
+// ------------------------------------------------------------------------------------------ MMA issuer
+__device__ __forceinline__ void mma_loop(const AttnParams& p, Aux* aux, uint32_t smem_base, uint32_t tmem, Walker w) {
+    const int lane = threadIdx.x & 31;
+    volatile int* abort_flag = &aux->abort_flag;
+    constexpr uint32_t idesc_qk = umma_idesc_bf16(128, kTileKeys, 0, 0);
+    constexpr uint32_t idesc_pv = umma_idesc_bf16(128, kHeadDim, 0, 1);
+    const uint32_t ring = smem_base + kRingOff;
+    uint32_t it[2] = {0, 0};
+    uint32_t seg_no = 0, item_base = 0;
+    Segment g;
+
+    while (w.next(p, g)) {
+        bool ok = mbar_wait(smem_u32(&aux->q_full), seg_no & 1u, abort_flag);
+        tc_fence_after();
+        const int n_it[2] = {g.iters(0), g.iters(1)};
+
+        auto issue_qk = [&](int s, int t) {
+            const uint32_t item = item_base + 2u * (uint32_t)(t - g.tile0);
+            const uint32_t slot = item % kSlots, ph = (item / kSlots) & 1u;
+            ok = mbar_wait(smem_u32(&aux->full[slot]), ph, abort_flag) && ok;
+            tc_fence_after();
+            if (lane == 0 && ok) {
+                const uint32_t qa = smem_base + (g.shared ? s : 0) * kQBytes;
+                const uint32_t ka = ring + slot * kSlotBytes;
+#pragma unroll
+                for (int hf = 0; hf < 2; ++hf)
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks)
+                        umma_ss(tmem + s * 128, umma_smem_desc_sw128(qa + hf * 16384 + ks * 32, 16, 1024),
+                                umma_smem_desc_sw128(ka + hf * 1024 + ks * 32, 16, 2048), idesc_qk, (hf | ks) ? 1u : 0u);
+                umma_commit(smem_u32(&aux->s_full[s]));
+                if (!g.shared || s == 1) umma_commit(smem_u32(&aux->empty[slot]));
+            }
+            __syncwarp();
+        };
+
+        for (int s = 0; s < 2; ++s)
+            if (n_it[s] > 0) issue_qk(s, g.tile(s, 0));
+        for (int i = 0; i < n_it[0]; ++i) {
+            for (int s = 0; s < 2; ++s) {
+                if (i >= n_it[s]) continue;
+                const int t = g.tile(s, i);
+                const uint32_t item = item_base + 2u * (uint32_t)(t - g.tile0) + 1u;
+                const uint32_t slot = item % kSlots, ph = (item / kSlots) & 1u;
+                ok = mbar_wait(smem_u32(&aux->p_full[s]), it[s] & 1u, abort_flag) && ok;
+                ok = mbar_wait(smem_u32(&aux->full[slot]), ph, abort_flag) && ok;
+                tc_fence_after();
+                if (lane == 0 && ok) {
+                    const uint32_t va = ring + slot * kSlotBytes;
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks)
+                        umma_ts(tmem + 256 + s * 128, tmem + s * 128 + ks * 8,
+                                umma_smem_desc_sw128(va + ks * 4096, 1024, 2048), idesc_pv, (i | ks) ? 1u : 0u);
+                    umma_commit(smem_u32(&aux->o_done[s]));
+                    if (!g.shared || s == 1) umma_commit(smem_u32(&aux->empty[slot]));
+                }
+                __syncwarp();
+                ++it[s];
+                if (i + 1 < n_it[s]) issue_qk(s, g.tile(s, i + 1));
+            }
+        }
+        item_base += 2u * (uint32_t)(g.tile1 - g.tile0);
+        ++seg_no;
+    }
+}
+
+// ------------------------------------------------------------------------------------------ softmax warpgroups
+__device__ __forceinline__ void named_barrier(int id, int count) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
+}
+
+__device__ __forceinline__ float max3(float a, float b, float c) { return fmaxf(fmaxf(a, b), c); }
+
+template <bool kFinal>
+__device__ __forceinline__ void store_row32(const AttnParams& p, long long out_row, long long part_row, int col,
+                                            const float (&v)[32]) {
+    if (kFinal) {
+        uint4* dst = reinterpret_cast<uint4*>(p.out + out_row * kHeadDim + col);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            __nv_bfloat162 a = __floats2bfloat162_rn(v[8 * j], v[8 * j + 1]), b = __floats2bfloat162_rn(v[8 * j + 2], v[8 * j + 3]);
+            __nv_bfloat162 c = __floats2bfloat162_rn(v[8 * j + 4], v[8 * j + 5]), d = __floats2bfloat162_rn(v[8 * j + 6], v[8 * j + 7]);
+            uint4 u;
+            u.x = *reinterpret_cast<uint32_t*>(&a); u.y = *reinterpret_cast<uint32_t*>(&b);
+            u.z = *reinterpret_cast<uint32_t*>(&c); u.w = *reinterpret_cast<uint32_t*>(&d);
+            dst[j] = u;
+        }
+    } else {
+        float4* dst = reinterpret_cast<float4*>(p.part_o + part_row * kHeadDim + col);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) dst[j] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+    }
+}
+
+__device__ __forceinline__ void softmax_loop(const AttnParams& p, Aux* aux, unsigned char* smem, uint32_t tmem, Walker w,
+                                             const int s /*stream*/) {
+    const int wtid = threadIdx.x - 128 - s * 128;          // 0..127 inside the warpgroup
+    const int row_local = wtid;                             // TMEM lane = (warp % 4) * 32 + lane
+    volatile int* abort_flag = &aux->abort_flag;
+    const uint32_t lane_sel = (uint32_t)(((threadIdx.x >> 5) & 3) * 32) << 16;
+    const uint32_t tS = tmem + lane_sel + s * 128;
+    const float scale2 = fabsf(p.sm_scale) * 1.4426950408889634f;
+    const uint32_t q_flip = p.sm_scale < 0.f ? 0x80008000u : 0u;   // a negative scale is folded into Q (exact)
+    const int G = p.group;
+    uint32_t it = 0, seg_no = 0;
+    Segment g;
+
+    while (w.next(p, g)) {
+        // ---- ancestor masks (stream 0's warpgroup) and Q
+        if (s == 0) {
+            if (wtid == 0) aux->seg_bad_tree = 0;
+            named_barrier(2, 128);
+            if (wtid < g.n) {
+                const int pi = p.tree_parent[g.node_base + wtid];
+                const bool bad = (wtid == 0 && pi != -1) || (wtid > 0 && (pi < 0 || pi >= wtid));
+                if (bad) {
+                    atomicExch(&aux->seg_bad_tree, 1);
+                    report(p.status, kErrBadTree);
+                    p.seq_bad[g.b] = p.epoch;
+                }
+                aux->parent[wtid] = bad ? (short)-1 : (short)pi;
+            }
+            named_barrier(2, 128);
+            if (wtid < g.n) {
+                unsigned long long m = 0;
+                if (!aux->seg_bad_tree)
+                    for (int j = wtid, guard = 0; j >= 0 && guard < kMaxNodes; j = aux->parent[j], ++guard) m |= 1ull << j;
+                aux->anc[wtid] = m;
+            }
+        }
+        {
+            // shared: this warpgroup loads its own 128-row block; split: rows [64 s, 64 s + 64) of block 0
+            const int blk = g.shared ? s : 0;
+            const int r_first = g.shared ? 0 : 64 * s;
+            const int chunks = (g.shared ? 128 : 64) * 16;
+            unsigned char* qs = smem + blk * kQBytes;
+            for (int base = 0; base < chunks; base += 128 * 8) {
+                uint4 v[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const int idx = base + j * 128 + wtid;
+                    const int r = r_first + (idx >> 4), c = idx & 15;
+                    const int rr = blk * 128 + r;
+                    v[j] = make_uint4(0u, 0u, 0u, 0u);
+                    if (idx < chunks && rr < g.M)
+                        v[j] = __ldg(reinterpret_cast<const uint4*>(
+                            p.q + ((long long)(g.node_base + rr / G) * p.num_q_heads + g.h * G + rr % G) * kHeadDim + c * 8));
+                }
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const int idx = base + j * 128 + wtid;
+                    if (idx < chunks) {
+                        const int r = r_first + (idx >> 4), c = idx & 15;
+                        uint4 u = v[j];
+                        u.x ^= q_flip; u.y ^= q_flip; u.z ^= q_flip; u.w ^= q_flip;
+                        *reinterpret_cast<uint4*>(qs + (c >> 3) * 16384 + r * 128 + (((c & 7) ^ (r & 7)) << 4)) = u;
+                    }
+                }
+            }
+        }
+        fence_proxy_async_smem();
+        named_barrier(1, 256);                 // masks and the tree verdict are visible to both warpgroups
+        mbar_arrive(smem_u32(&aux->q_full));
+
+        const int rr = (g.shared ? s * 128 : 0) + row_local;       // packed row of this thread
+        const unsigned long long anc_row = rr < g.M ? aux->anc[rr / G] : 0ull;
+        const bool bad_tree = aux->seg_bad_tree != 0;
+        const int n_it = g.iters(s);
+        float m = -INFINITY, l = 0.f, lx = 0.f;   // l: sum of the bf16 weights (normaliser); lx: exact sum (LSE)
+
+        for (int i = 0; i < n_it; ++i) {
+            const int t = g.tile(s, i);
+            mbar_wait(smem_u32(&aux->s_full[s]), it & 1u, abort_flag);
+            tc_fence_after();
+            float sv[128];
+            {
+                uint32_t (&raw)[128] = reinterpret_cast<uint32_t(&)[128]>(sv);
+                tmem_ld32(tS, reinterpret_cast<uint32_t(&)[32]>(raw[0]));
+                tmem_ld32(tS + 32, reinterpret_cast<uint32_t(&)[32]>(raw[32]));
+                tmem_ld32(tS + 64, reinterpret_cast<uint32_t(&)[32]>(raw[64]));
+                tmem_ld32(tS + 96, reinterpret_cast<uint32_t(&)[32]>(raw[96]));
+                tmem_wait_ld();
+            }
+            if ((t + 1) * kTileKeys > g.L) {
+                // visibility of the tile's 128 keys for this row: prefix keys all, drafted key j iff ancestor-or-self
+                const int j0 = t * kTileKeys - g.L;
+                unsigned long long lo, hi;
+                if (j0 >= 0) {
+                    lo = j0 < 64 ? anc_row >> j0 : 0ull;
+                    hi = 0ull;
+                } else {
+                    const int k = -j0;   // 1..127 prefix keys at the front of the tile
+                    if (k >= 64) { lo = ~0ull; hi = (k == 64 ? 0ull : (~0ull >> (128 - k))) | (anc_row << (k - 64)); }
+                    else { lo = (~0ull >> (64 - k)) | (anc_row << k); hi = anc_row >> (64 - k); }
+                }
+#pragma unroll
+                for (int c = 0; c < 64; ++c) {
+                    if (!((lo >> c) & 1ull)) sv[c] = -INFINITY;
+                    if (!((hi >> c) & 1ull)) sv[64 + c] = -INFINITY;
+                }
+            }
+            float mx = max3(sv[0], sv[1], sv[2]);
+#pragma unroll
+            for (int c = 3; c + 1 < 128; c += 2) mx = max3(mx, sv[c], sv[c + 1]);
+            mx = fmaxf(mx, sv[127]);
+            const float m_new = fmaxf(m, mx * scale2);
+            const bool need = (m_new - m) > kLazyRescale;      // false when both are -inf (NaN compares false)
+            if (__any_sync(0xffffffffu, need)) {
+                const float alpha = (m_new == -INFINITY) ? 1.f : fast_exp2(m - m_new);
+                if (i > 0) {
+                    mbar_wait(smem_u32(&aux->o_done[s]), (it - 1u) & 1u, abort_flag);
+                    tc_fence_after();
+                    const uint32_t tO = tmem + lane_sel + 256 + s * 128;
+#pragma unroll
+                    for (int c4 = 0; c4 < 4; ++c4) {
+                        uint32_t o[32];
+                        tmem_ld32(tO + c4 * 32, o);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * alpha);
+                        tmem_st32(tO + c4 * 32, o);
+                    }
+                    l *= alpha;
+                    lx *= alpha;
+                }
+                m = m_new;
+            }
+            const float neg_m = (m == -INFINITY) ? 0.f : -m;
+            float sum0 = 0.f, sum1 = 0.f, ex0 = 0.f, ex1 = 0.f;
+#pragma unroll
+            for (int hf = 0; hf < 2; ++hf) {
+                uint32_t pk[32];
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    const float p0 = fast_exp2(fmaf(sv[hf * 64 + 2 * j], scale2, neg_m));
+                    const float p1 = fast_exp2(fmaf(sv[hf * 64 + 2 * j + 1], scale2, neg_m));
+                    __nv_bfloat162 b2 = __floats2bfloat162_rn(p0, p1);
+                    const uint32_t u = *reinterpret_cast<uint32_t*>(&b2);
+                    pk[j] = u;
+                    // the row sum takes the bf16-rounded weights, the very numbers P V multiplies by, so
+                    // that out = sum(p v) / sum(p) stays a true weighted mean (exact when one key dominates)
+                    sum0 += __uint_as_float(u << 16);
+                    sum1 += __uint_as_float(u & 0xffff0000u);
+                    ex0 += p0; ex1 += p1;              // the unrounded sum gives the LSE
+                }
+                tmem_st32(tS + hf * 32, pk);
+            }
+            l += sum0 + sum1;
+            lx += ex0 + ex1;
+            tmem_wait_st();
+            tc_fence_before();
+            mbar_arrive(smem_u32(&aux->p_full[s]));
+            ++it;
+        }
+
+        // ---- segment end: every product of this stream has completed
+        if (n_it > 0) mbar_wait(smem_u32(&aux->o_done[s]), (it - 1u) & 1u, abort_flag);
+        tc_fence_after();
+        // split mode: the streams exchange (m, l, lx) through the second Q block, which only the shared mode uses
+        float (*ml)[128][3] = reinterpret_cast<float (*)[128][3]>(smem + kQBytes);
+        if (!g.shared) { ml[s][row_local][0] = m; ml[s][row_local][1] = l; ml[s][row_local][2] = lx; }
+        named_barrier(1, 256);                 // both streams done: all MMAs of the segment have completed
+        const bool write_ok = !bad_tree && !*abort_flag && *reinterpret_cast<volatile int32_t*>(p.seq_bad + g.b) != p.epoch;
+        // only the first and the last unit of a CTA's piece can be cut: two partial slots per CTA
+        const long long part_row = (2ll * blockIdx.x + (seg_no > 0 ? 1 : 0)) * p.rows_per_slot + rr;
+        const long long out_row = rr < g.M ? (long long)(g.node_base + rr / G) * p.num_q_heads + g.h * G + rr % G : 0;
+        const bool row_ok = write_ok && rr < g.M;
+        const bool whole = g.whole();
+        if (g.shared) {
+            const float inv = l > 0.f ? 1.f / l : 0.f;
+            const uint32_t tO = tmem + lane_sel + 256 + s * 128;
+#pragma unroll
+            for (int c4 = 0; c4 < 4; ++c4) {
+                uint32_t o[32];
+                tmem_ld32(tO + c4 * 32, o);
+                tmem_wait_ld();
+                float v[32];
+#pragma unroll
+                for (int j = 0; j < 32; ++j) v[j] = l > 0.f ? __uint_as_float(o[j]) * inv : 0.f;
+                if (row_ok) {
+                    if (whole) store_row32<true>(p, out_row, part_row, c4 * 32, v);
+                    else store_row32<false>(p, out_row, part_row, c4 * 32, v);
+                }
+            }
+            if (row_ok) {
+                const float lse = lx > 0.f ? (m + __log2f(lx)) * 0.6931471805599453f : -INFINITY;
+                if (whole) { if (p.lse) p.lse[out_row] = lse; }
+                else p.part_lse[part_row] = lse;
+            }
+        } else {
+            // merge the two streams (same rows, disjoint key tiles); this warpgroup writes columns [64 s, 64 s + 64)
+            const float m0 = ml[0][row_local][0], l0 = ml[0][row_local][1];
+            const bool has1 = g.iters(1) > 0;
+            const float m1 = has1 ? ml[1][row_local][0] : -INFINITY, l1 = has1 ? ml[1][row_local][1] : 0.f;
+            const float x0 = ml[0][row_local][2], x1 = has1 ? ml[1][row_local][2] : 0.f;
+            const float mm = fmaxf(m0, m1);
+            const float a0 = (m0 == -INFINITY) ? 0.f : fast_exp2(m0 - mm);
+            const float a1 = (m1 == -INFINITY) ? 0.f : fast_exp2(m1 - mm);
+            const float lt = a0 * l0 + a1 * l1;
+            const float inv = lt > 0.f ? 1.f / lt : 0.f;
+            const float w0 = a0 * inv, w1 = a1 * inv;
+            const uint32_t tO0 = tmem + lane_sel + 256, tO1 = tmem + lane_sel + 384;
+#pragma unroll
+            for (int c2 = 0; c2 < 2; ++c2) {
+                const int col = s * 64 + c2 * 32;
+                uint32_t o0[32], o1[32];
+                tmem_ld32(tO0 + col, o0);
+                if (has1) tmem_ld32(tO1 + col, o1);
+                tmem_wait_ld();
+                float v[32];
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    float x = a0 > 0.f ? __uint_as_float(o0[j]) * w0 : 0.f;
+                    if (has1 && a1 > 0.f) x = fmaf(__uint_as_float(o1[j]), w1, x);
+                    v[j] = x;
+                }
+                if (row_ok) {
+                    if (whole) store_row32<true>(p, out_row, part_row, col, v);
+                    else store_row32<false>(p, out_row, part_row, col, v);
+                }
+            }
+            if (row_ok && s == 0) {
+                const float xt = a0 * x0 + a1 * x1;
+                const float lse = xt > 0.f ? (mm + __log2f(xt)) * 0.6931471805599453f : -INFINITY;
+                if (whole) { if (p.lse) p.lse[out_row] = lse; }
+                else p.part_lse[part_row] = lse;
+            }
+        }
+        tc_fence_before();
+        ++seg_no;
+    }
+}
+
+// ------------------------------------------------------------------------------------------ kernel
+__global__ void __launch_bounds__(kThreads, 1)
+verify_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap vmap) {
+    extern __shared__ __align__(1024) unsigned char smem[];
+    Aux* aux = reinterpret_cast<Aux*>(smem + kAuxOff);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t smem_base = smem_u32(smem);
+    if (smem_base & 1023u) {                       // operand tiles must sit on swizzle-atom boundaries
+        if (tid == 0) report(p.status, kErrTimeout);
+        return;
+    }
+    if (tid == 0) {
+        for (int i = 0; i < kSlots; ++i) { mbar_init(smem_u32(&aux->full[i]), 1); mbar_init(smem_u32(&aux->empty[i]), 1); }
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(smem_u32(&aux->s_full[s]), 1);
+            mbar_init(smem_u32(&aux->p_full[s]), 128);
+            mbar_init(smem_u32(&aux->o_done[s]), 1);
+        }
+        mbar_init(smem_u32(&aux->q_full), 256);
+        aux->abort_flag = 0;
+        aux->seg_bad_tree = 0;
+        aux->sched_b0 = 0; aux->sched_tile_begin = 0; aux->sched_unit_begin = 0;
+        fence_barrier_init();
+        tma_prefetch_desc(&kmap);
+        tma_prefetch_desc(&vmap);
+    }
+    if (warp == 0) { tmem_alloc(smem_u32(&aux->tmem_base), kTmemCols); tmem_relinquish(); }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = aux->tmem_base;
+
+    Walker w;
+    build_walk(p, aux, w);
+
+    // registers move from the warpgroup of the producer / MMA warps to the two softmax warpgroups,
+    // whose threads each hold a 128-column row of S: 128 x 56 + 256 x 224 = 384 x 168
+    uint32_t items = 0;
+    if (warp < 4) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+        if (warp == 0) producer_loop(p, &kmap, &vmap, aux, smem_base + kRingOff, w, items);
+        else if (warp == 1) mma_loop(p, aux, smem_base, tmem, w);
+    } else {
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
+        softmax_loop(p, aux, smem, tmem, w, warp >= 8 ? 1 : 0);
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) {
+        if (aux->abort_flag) {
+            // give the copies still in flight a bounded time to land before the CTA's shared memory is released
+            const uint32_t first = items > (uint32_t)kSlots ? items - kSlots : 0u;
+            for (uint32_t it = first; it < items; ++it) {
+                const uint32_t bar = smem_u32(&aux->full[it % kSlots]), ph = (it / kSlots) & 1u;
+                for (int polls = 0; polls < (1 << 20) && !mbar_try_wait(bar, ph); ++polls) {}
+            }
+            if (lane == 0) report(p.status, kErrTimeout);
+        }
+        tc_fence_after();
+        tmem_dealloc(tmem, kTmemCols);
+    }
+}
+
+}  // namespace umma_path
+}  // namespace owl
