@@ -82,14 +82,14 @@ typedef struct owl_dims {
     int32_t total_nodes;       /* N = sum of n_b >= B                                           */
     int32_t max_nodes;         /* T = max n_b, 1..64 (the paper's trees have 60 nodes)          */
     int32_t num_q_heads;       /* Hq                                                            */
-    int32_t num_kv_heads;      /* Hkv, divides Hq; G*T <= 256                                   */
+    int32_t num_kv_heads;      /* Hkv <= 128, divides Hq; G*T <= 256                            */
     int32_t head_dim;          /* must be 128                                                   */
     int32_t page_size;         /* tokens per page: 16 (also 32, 64, 128)                        */
     int32_t max_pages_per_seq; /* row stride of block_table                                     */
     int32_t num_pages;         /* pages in k_cache / v_cache; block_table entries are checked   */
     int32_t vocab;             /* V (owl_tree_accept only; may be 0 for attention-only use)     */
     int32_t path_stride;       /* row stride of accept_path, >= max_nodes (64 always is)        */
-    float sm_scale;            /* multiplies q.k before the softmax; always explicit            */
+    float sm_scale;            /* multiplies q.k before the softmax; explicit, finite, > 0      */
 } owl_dims;
 
 /* Create a context on `device` with workspace for any call whose dims do not exceed

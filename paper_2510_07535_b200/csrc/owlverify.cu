@@ -77,8 +77,9 @@ int check_dims(const owl_dims* d, bool for_attn, bool for_accept) {
     if ((long long)d->max_nodes * d->batch < d->total_nodes) return OWL_ERR_INVALID_ARG;
     if (for_attn) {
         if (d->num_q_heads < 1 || d->num_kv_heads < 1 || d->num_q_heads % d->num_kv_heads != 0) return OWL_ERR_INVALID_ARG;
+        if (d->num_kv_heads > 128) return OWL_ERR_UNSUPPORTED;
         if (d->max_pages_per_seq < 1 || d->num_pages < 1) return OWL_ERR_INVALID_ARG;
-        if (!(d->sm_scale == d->sm_scale) || d->sm_scale == 0.f || d->sm_scale - d->sm_scale != 0.f) return OWL_ERR_INVALID_ARG;
+        if (!(d->sm_scale > 0.f) || d->sm_scale - d->sm_scale != 0.f) return OWL_ERR_INVALID_ARG;   // finite, > 0
         if (d->head_dim != kHeadDim) return OWL_ERR_UNSUPPORTED;
         if ((d->num_q_heads / d->num_kv_heads) * d->max_nodes > kMaxRows) return OWL_ERR_UNSUPPORTED;
         if (!(d->page_size == 16 || d->page_size == 32 || d->page_size == 64 || d->page_size == 128)) return OWL_ERR_UNSUPPORTED;

@@ -90,30 +90,38 @@ struct Segment {
 struct Walker {
     int b, unit_begin;
     long long seq_begin, t, t_end;
+    // the sequence `b` as last loaded (most segments of a piece lie in the same sequence)
+    int cur_b = -1, cur_n = 0, cur_L = 0, cur_tiles = 0, cur_node_base = 0;
+    bool cur_ok = false;
+    __device__ __forceinline__ void load_seq(const AttnParams& p) {
+        cur_n = seq_nodes(p, b);
+        cur_L = p.ctx_lens[b];
+        cur_ok = seq_shape_ok(p, b, cur_n, cur_L);
+        cur_tiles = cur_ok ? (cur_L + cur_n + kTileKeys - 1) / kTileKeys : 0;
+        cur_node_base = seq_node_base(p, b);
+        cur_b = b;
+    }
     __device__ __forceinline__ bool next(const AttnParams& p, Segment& g) {
         if (t >= t_end) return false;
-        int n = 0, L = 0, tiles = 0;
         while (b < p.batch) {
-            n = seq_nodes(p, b);
-            L = p.ctx_lens[b];
-            const bool ok = seq_shape_ok(p, b, n, L);
-            tiles = ok ? (L + n + kTileKeys - 1) / kTileKeys : 0;
-            const long long flat = (long long)tiles * p.num_kv_heads;
+            if (cur_b != b) load_seq(p);
+            const long long flat = (long long)cur_tiles * p.num_kv_heads;
             if (t < seq_begin + flat) break;
             seq_begin += flat;
-            unit_begin += ok ? p.num_kv_heads : 0;
+            unit_begin += cur_ok ? p.num_kv_heads : 0;
             ++b;
         }
         if (b >= p.batch) { t = t_end; return false; }
-        const long long local = t - seq_begin;
-        g.b = b; g.n = n; g.L = L; g.tiles = tiles;
-        g.h = (int)(local / tiles);
-        g.tile0 = (int)(local % tiles);
+        const int tiles = cur_tiles;
+        const unsigned local = (unsigned)(t - seq_begin);   // < tiles * Hkv <= 2^24 * 2^7
+        g.b = b; g.n = cur_n; g.L = cur_L; g.tiles = tiles;
+        g.h = (int)(local / (unsigned)tiles);
+        g.tile0 = (int)(local - (unsigned)g.h * (unsigned)tiles);
         const long long left = t_end - t;
         g.tile1 = (int)(g.tile0 + left < tiles ? g.tile0 + left : tiles);
         g.unit = unit_begin + g.h;
-        g.node_base = seq_node_base(p, b);
-        g.M = n * p.group;
+        g.node_base = cur_node_base;
+        g.M = cur_n * p.group;
         g.shared = g.M > 128;
         t += g.tile1 - g.tile0;
         return true;
@@ -179,6 +187,8 @@ __device__ __forceinline__ void producer_loop(const AttnParams& p, const CUtenso
     const uint32_t box_bytes = (uint32_t)p.page_size * 256u;
     const int oob = p.num_pages * p.num_kv_heads;            // a coordinate past the end: the box reads zeros
     uint32_t item = 0;
+    // K/V are read once: let them leave L2 first, so that Q, the partials, the tables and the code stay
+    const uint64_t stream_policy = l2_policy_evict_first();
     Segment g;
     while (w.next(p, g)) {
         const int keys = g.L + g.n;
@@ -207,7 +217,8 @@ __device__ __forceinline__ void producer_loop(const AttnParams& p, const CUtenso
                     if (lane == 0) mbar_arrive_expect_tx(full, (uint32_t)kSlotBytes);
                     __syncwarp();
                     if (lane < ppt)
-                        tma_load_5d(ring + slot * kSlotBytes + lane * box_bytes, kv ? vmap : kmap, full, 0, 0, 0, 0, c_cur);
+                        tma_load_5d_hint(ring + slot * kSlotBytes + lane * box_bytes, kv ? vmap : kmap, full, 0, 0, 0, 0, c_cur,
+                                         stream_policy);
                     ++item;
                 }
                 __syncwarp();
@@ -233,49 +244,50 @@ __device__ __forceinline__ void mma_loop(const AttnParams& p, Aux* aux, uint32_t
         tc_fence_after();
         const int n_it[2] = {g.iters(0), g.iters(1)};
 
-        auto issue_qk = [&](int s, int t) {
-            const uint32_t item = item_base + 2u * (uint32_t)(t - g.tile0);
-            const uint32_t slot = item % kSlots, ph = (item / kSlots) & 1u;
-            ok = mbar_wait(smem_u32(&aux->full[slot]), ph, abort_flag) && ok;
-            tc_fence_after();
-            if (lane == 0 && ok) {
-                const uint32_t qa = smem_base + (g.shared ? s : 0) * kQBytes;
-                const uint32_t ka = ring + slot * kSlotBytes;
-#pragma unroll
-                for (int hf = 0; hf < 2; ++hf)
-#pragma unroll
-                    for (int ks = 0; ks < 4; ++ks)
-                        umma_ss(tmem + s * 128, umma_smem_desc_sw128(qa + hf * 16384 + ks * 32, 16, 1024),
-                                umma_smem_desc_sw128(ka + hf * 1024 + ks * 32, 16, 2048), idesc_qk, (hf | ks) ? 1u : 0u);
-                umma_commit(smem_u32(&aux->s_full[s]));
-                if (!g.shared || s == 1) umma_commit(smem_u32(&aux->empty[slot]));
-            }
-            __syncwarp();
-        };
-
-        for (int s = 0; s < 2; ++s)
-            if (n_it[s] > 0) issue_qk(s, g.tile(s, 0));
-        for (int i = 0; i < n_it[0]; ++i) {
+        // i = -1 issues the first S = Q K^T of both streams; afterwards, per stream: O += P V of tile i, then
+        // S = Q K^T of tile i + 1 (which overwrites the P just consumed; the tensor pipe runs them in order)
+#pragma unroll 1
+        for (int i = -1; i < n_it[0]; ++i) {
+#pragma unroll 1
             for (int s = 0; s < 2; ++s) {
-                if (i >= n_it[s]) continue;
-                const int t = g.tile(s, i);
-                const uint32_t item = item_base + 2u * (uint32_t)(t - g.tile0) + 1u;
-                const uint32_t slot = item % kSlots, ph = (item / kSlots) & 1u;
-                ok = mbar_wait(smem_u32(&aux->p_full[s]), it[s] & 1u, abort_flag) && ok;
-                ok = mbar_wait(smem_u32(&aux->full[slot]), ph, abort_flag) && ok;
-                tc_fence_after();
-                if (lane == 0 && ok) {
-                    const uint32_t va = ring + slot * kSlotBytes;
+                const bool last_reader = !g.shared || s == 1;
+                if (i >= 0 && i < n_it[s]) {
+                    const uint32_t item = item_base + 2u * (uint32_t)(g.tile(s, i) - g.tile0) + 1u;
+                    const uint32_t slot = item % kSlots, ph = (item / kSlots) & 1u;
+                    ok = mbar_wait(smem_u32(&aux->p_full[s]), it[s] & 1u, abort_flag) && ok;
+                    ok = mbar_wait(smem_u32(&aux->full[slot]), ph, abort_flag) && ok;
+                    tc_fence_after();
+                    if (lane == 0 && ok) {
+                        const uint32_t va = ring + slot * kSlotBytes;
 #pragma unroll
-                    for (int ks = 0; ks < 8; ++ks)
-                        umma_ts(tmem + 256 + s * 128, tmem + s * 128 + ks * 8,
-                                umma_smem_desc_sw128(va + ks * 4096, 1024, 2048), idesc_pv, (i | ks) ? 1u : 0u);
-                    umma_commit(smem_u32(&aux->o_done[s]));
-                    if (!g.shared || s == 1) umma_commit(smem_u32(&aux->empty[slot]));
+                        for (int ks = 0; ks < 8; ++ks)
+                            umma_ts(tmem + 256 + s * 128, tmem + s * 128 + ks * 8,
+                                    umma_smem_desc_sw128(va + ks * 4096, 1024, 2048), idesc_pv, (i | ks) ? 1u : 0u);
+                        umma_commit(smem_u32(&aux->o_done[s]));
+                        if (last_reader) umma_commit(smem_u32(&aux->empty[slot]));
+                    }
+                    __syncwarp();
+                    ++it[s];
                 }
-                __syncwarp();
-                ++it[s];
-                if (i + 1 < n_it[s]) issue_qk(s, g.tile(s, i + 1));
+                if (i + 1 < n_it[s]) {
+                    const uint32_t item = item_base + 2u * (uint32_t)(g.tile(s, i + 1) - g.tile0);
+                    const uint32_t slot = item % kSlots, ph = (item / kSlots) & 1u;
+                    ok = mbar_wait(smem_u32(&aux->full[slot]), ph, abort_flag) && ok;
+                    tc_fence_after();
+                    if (lane == 0 && ok) {
+                        const uint32_t qa = smem_base + (g.shared ? s : 0) * kQBytes;
+                        const uint32_t ka = ring + slot * kSlotBytes;
+#pragma unroll
+                        for (int hf = 0; hf < 2; ++hf)
+#pragma unroll
+                            for (int ks = 0; ks < 4; ++ks)
+                                umma_ss(tmem + s * 128, umma_smem_desc_sw128(qa + hf * 16384 + ks * 32, 16, 1024),
+                                        umma_smem_desc_sw128(ka + hf * 1024 + ks * 32, 16, 2048), idesc_qk, (hf | ks) ? 1u : 0u);
+                        umma_commit(smem_u32(&aux->s_full[s]));
+                        if (last_reader) umma_commit(smem_u32(&aux->empty[slot]));
+                    }
+                    __syncwarp();
+                }
             }
         }
         item_base += 2u * (uint32_t)(g.tile1 - g.tile0);
@@ -290,24 +302,45 @@ __device__ __forceinline__ void named_barrier(int id, int count) {
 
 __device__ __forceinline__ float max3(float a, float b, float c) { return fmaxf(fmaxf(a, b), c); }
 
+// Writes a warp's 32 rows x 32 columns (lane = row, v = its 32 fp32 values) to global memory through a
+// per-warp staging area in shared memory, so that every store instruction covers whole 64- or 128-byte
+// row segments instead of 32 scattered 16-byte pieces.  `out_row` / `row_ok` are the lane's own row;
+// the other rows' values come by shuffle.  kFinal: bf16 into `out`; else fp32 into the partial slot,
+// whose rows are consecutive (part_row0 = row of lane 0).
+constexpr int kStageStride = 36;                     // floats per staged row: 16-byte aligned, conflict-free
+constexpr int kStageBytesPerWarp = 32 * kStageStride * 4;
 template <bool kFinal>
-__device__ __forceinline__ void store_row32(const AttnParams& p, long long out_row, long long part_row, int col,
-                                            const float (&v)[32]) {
-    if (kFinal) {
-        uint4* dst = reinterpret_cast<uint4*>(p.out + out_row * kHeadDim + col);
+__device__ __forceinline__ void store_rows32(const AttnParams& p, float* stage, long long out_row, bool row_ok,
+                                             long long part_row0, int col, const float (&v)[32]) {
+    const int lane = threadIdx.x & 31;
+    __syncwarp();
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            __nv_bfloat162 a = __floats2bfloat162_rn(v[8 * j], v[8 * j + 1]), b = __floats2bfloat162_rn(v[8 * j + 2], v[8 * j + 3]);
-            __nv_bfloat162 c = __floats2bfloat162_rn(v[8 * j + 4], v[8 * j + 5]), d = __floats2bfloat162_rn(v[8 * j + 6], v[8 * j + 7]);
+    for (int j = 0; j < 8; ++j)
+        *reinterpret_cast<float4*>(stage + lane * kStageStride + 4 * j) = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+    __syncwarp();
+    if (kFinal) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {                 // 8 rows x 64 bytes per instruction
+            const int row = 8 * k + (lane >> 2), piece = lane & 3;
+            const long long orow = __shfl_sync(0xffffffffu, out_row, row);
+            const bool ok = __shfl_sync(0xffffffffu, row_ok ? 1 : 0, row) != 0;
+            const float4 a = *reinterpret_cast<const float4*>(stage + row * kStageStride + piece * 8);
+            const float4 b2 = *reinterpret_cast<const float4*>(stage + row * kStageStride + piece * 8 + 4);
+            __nv_bfloat162 w0 = __floats2bfloat162_rn(a.x, a.y), w1 = __floats2bfloat162_rn(a.z, a.w);
+            __nv_bfloat162 w2 = __floats2bfloat162_rn(b2.x, b2.y), w3 = __floats2bfloat162_rn(b2.z, b2.w);
             uint4 u;
-            u.x = *reinterpret_cast<uint32_t*>(&a); u.y = *reinterpret_cast<uint32_t*>(&b);
-            u.z = *reinterpret_cast<uint32_t*>(&c); u.w = *reinterpret_cast<uint32_t*>(&d);
-            dst[j] = u;
+            u.x = *reinterpret_cast<uint32_t*>(&w0); u.y = *reinterpret_cast<uint32_t*>(&w1);
+            u.z = *reinterpret_cast<uint32_t*>(&w2); u.w = *reinterpret_cast<uint32_t*>(&w3);
+            if (ok) *reinterpret_cast<uint4*>(p.out + orow * kHeadDim + col + piece * 8) = u;
         }
     } else {
-        float4* dst = reinterpret_cast<float4*>(p.part_o + part_row * kHeadDim + col);
 #pragma unroll
-        for (int j = 0; j < 8; ++j) dst[j] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+        for (int k = 0; k < 8; ++k) {                 // 4 rows x 128 bytes per instruction
+            const int row = 4 * k + (lane >> 3), piece = lane & 7;
+            const bool ok = __shfl_sync(0xffffffffu, row_ok ? 1 : 0, row) != 0;
+            const float4 a = *reinterpret_cast<const float4*>(stage + row * kStageStride + piece * 4);
+            if (ok) *reinterpret_cast<float4*>(p.part_o + (part_row0 + row) * kHeadDim + col + piece * 4) = a;
+        }
     }
 }
 
@@ -318,26 +351,48 @@ __device__ __forceinline__ void softmax_loop(const AttnParams& p, Aux* aux, unsi
     volatile int* abort_flag = &aux->abort_flag;
     const uint32_t lane_sel = (uint32_t)(((threadIdx.x >> 5) & 3) * 32) << 16;
     const uint32_t tS = tmem + lane_sel + s * 128;
-    const float scale2 = fabsf(p.sm_scale) * 1.4426950408889634f;
-    const uint32_t q_flip = p.sm_scale < 0.f ? 0x80008000u : 0u;   // a negative scale is folded into Q (exact)
+    const float scale2 = p.sm_scale * 1.4426950408889634f;   // > 0 (checked on the host)
     const int G = p.group;
     uint32_t it = 0, seg_no = 0;
     Segment g;
 
     while (w.next(p, g)) {
-        // ---- ancestor masks (stream 0's warpgroup) and Q
+        // ---- Q rows (16-byte asynchronous copies, rows beyond M zero-filled) and, in stream 0's warpgroup, the
+        // ancestor masks; every global read of the segment start is in flight at the same time
+        int parent_i = -1;
+        if (s == 0 && wtid < g.n) parent_i = p.tree_parent[g.node_base + wtid];
+        if (seg_no > 0) named_barrier(1, 256);   // the other warpgroup may still be reading its staging area in the Q blocks
+        {
+            // shared: this warpgroup loads its own 128-row block; split: rows [64 s, 64 s + 64) of block 0
+            const int blk = g.shared ? s : 0;
+            const int r_first = (g.shared ? 0 : 64 * s) + (wtid >> 4);
+            const int r_count = g.shared ? 16 : 8;                 // rows per thread, 8 apart
+            const int c = wtid & 15;                               // 16-byte chunk of the row
+            const uint32_t qs = smem_u32(smem) + blk * kQBytes + (c >> 3) * 16384;
+#pragma unroll 2
+            for (int j = 0; j < r_count; ++j) {
+                const int r = r_first + 8 * j;
+                const unsigned rr = (unsigned)(blk * 128 + r);
+                const bool valid = rr < (unsigned)g.M;
+                const unsigned node = rr / (unsigned)G, hg = rr - node * (unsigned)G;
+                const __nv_bfloat16* src =
+                    valid ? p.q + ((long long)(g.node_base + node) * p.num_q_heads + g.h * G + hg) * kHeadDim + c * 8 : p.q;
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(qs + r * 128 + (((c & 7) ^ (r & 7)) << 4)),
+                             "l"(src), "r"(valid ? 16 : 0) : "memory");
+            }
+            asm volatile("cp.async.commit_group;" ::: "memory");
+        }
         if (s == 0) {
             if (wtid == 0) aux->seg_bad_tree = 0;
             named_barrier(2, 128);
             if (wtid < g.n) {
-                const int pi = p.tree_parent[g.node_base + wtid];
-                const bool bad = (wtid == 0 && pi != -1) || (wtid > 0 && (pi < 0 || pi >= wtid));
+                const bool bad = (wtid == 0 && parent_i != -1) || (wtid > 0 && (parent_i < 0 || parent_i >= wtid));
                 if (bad) {
                     atomicExch(&aux->seg_bad_tree, 1);
                     report(p.status, kErrBadTree);
                     p.seq_bad[g.b] = p.epoch;
                 }
-                aux->parent[wtid] = bad ? (short)-1 : (short)pi;
+                aux->parent[wtid] = bad ? (short)-1 : (short)parent_i;
             }
             named_barrier(2, 128);
             if (wtid < g.n) {
@@ -347,36 +402,7 @@ __device__ __forceinline__ void softmax_loop(const AttnParams& p, Aux* aux, unsi
                 aux->anc[wtid] = m;
             }
         }
-        {
-            // shared: this warpgroup loads its own 128-row block; split: rows [64 s, 64 s + 64) of block 0
-            const int blk = g.shared ? s : 0;
-            const int r_first = g.shared ? 0 : 64 * s;
-            const int chunks = (g.shared ? 128 : 64) * 16;
-            unsigned char* qs = smem + blk * kQBytes;
-            for (int base = 0; base < chunks; base += 128 * 8) {
-                uint4 v[8];
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const int idx = base + j * 128 + wtid;
-                    const int r = r_first + (idx >> 4), c = idx & 15;
-                    const int rr = blk * 128 + r;
-                    v[j] = make_uint4(0u, 0u, 0u, 0u);
-                    if (idx < chunks && rr < g.M)
-                        v[j] = __ldg(reinterpret_cast<const uint4*>(
-                            p.q + ((long long)(g.node_base + rr / G) * p.num_q_heads + g.h * G + rr % G) * kHeadDim + c * 8));
-                }
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const int idx = base + j * 128 + wtid;
-                    if (idx < chunks) {
-                        const int r = r_first + (idx >> 4), c = idx & 15;
-                        uint4 u = v[j];
-                        u.x ^= q_flip; u.y ^= q_flip; u.z ^= q_flip; u.w ^= q_flip;
-                        *reinterpret_cast<uint4*>(qs + (c >> 3) * 16384 + r * 128 + (((c & 7) ^ (r & 7)) << 4)) = u;
-                    }
-                }
-            }
-        }
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
         fence_proxy_async_smem();
         named_barrier(1, 256);                 // masks and the tree verdict are visible to both warpgroups
         mbar_arrive(smem_u32(&aux->q_full));
@@ -391,17 +417,10 @@ __device__ __forceinline__ void softmax_loop(const AttnParams& p, Aux* aux, unsi
             const int t = g.tile(s, i);
             mbar_wait(smem_u32(&aux->s_full[s]), it & 1u, abort_flag);
             tc_fence_after();
-            float sv[128];
-            {
-                uint32_t (&raw)[128] = reinterpret_cast<uint32_t(&)[128]>(sv);
-                tmem_ld32(tS, reinterpret_cast<uint32_t(&)[32]>(raw[0]));
-                tmem_ld32(tS + 32, reinterpret_cast<uint32_t(&)[32]>(raw[32]));
-                tmem_ld32(tS + 64, reinterpret_cast<uint32_t(&)[32]>(raw[64]));
-                tmem_ld32(tS + 96, reinterpret_cast<uint32_t(&)[32]>(raw[96]));
-                tmem_wait_ld();
-            }
             if ((t + 1) * kTileKeys > g.L) {
-                // visibility of the tile's 128 keys for this row: prefix keys all, drafted key j iff ancestor-or-self
+                // The tile reaches drafted positions (or the end of the sequence): at most two tiles per unit.
+                // Visibility of its 128 keys for this row: prefix keys all, drafted key j iff ancestor-or-self.
+                // The mask is applied to S in tensor memory, 32 columns at a time, before the common path reads it.
                 const int j0 = t * kTileKeys - g.L;
                 unsigned long long lo, hi;
                 if (j0 >= 0) {
@@ -412,11 +431,25 @@ __device__ __forceinline__ void softmax_loop(const AttnParams& p, Aux* aux, unsi
                     if (k >= 64) { lo = ~0ull; hi = (k == 64 ? 0ull : (~0ull >> (128 - k))) | (anc_row << (k - 64)); }
                     else { lo = (~0ull >> (64 - k)) | (anc_row << k); hi = anc_row >> (64 - k); }
                 }
+#pragma unroll 1
+                for (int c4 = 0; c4 < 4; ++c4) {
+                    const uint32_t bits = (uint32_t)((c4 < 2 ? lo : hi) >> ((c4 & 1) * 32));
+                    uint32_t r[32];
+                    tmem_ld32(tS + c4 * 32, r);
+                    tmem_wait_ld();
 #pragma unroll
-                for (int c = 0; c < 64; ++c) {
-                    if (!((lo >> c) & 1ull)) sv[c] = -INFINITY;
-                    if (!((hi >> c) & 1ull)) sv[64 + c] = -INFINITY;
+                    for (int j = 0; j < 32; ++j)
+                        if (!((bits >> j) & 1u)) r[j] = 0xff800000u;   // -inf
+                    tmem_st32(tS + c4 * 32, r);
                 }
+                tmem_wait_st();
+            }
+            float sv[128];
+            {
+                uint32_t (&raw)[128] = reinterpret_cast<uint32_t(&)[128]>(sv);
+                tmem_ld64(tS, reinterpret_cast<uint32_t(&)[64]>(raw[0]));
+                tmem_ld64(tS + 64, reinterpret_cast<uint32_t(&)[64]>(raw[64]));
+                tmem_wait_ld();
             }
             float mx = max3(sv[0], sv[1], sv[2]);
 #pragma unroll
@@ -430,7 +463,7 @@ __device__ __forceinline__ void softmax_loop(const AttnParams& p, Aux* aux, unsi
                     mbar_wait(smem_u32(&aux->o_done[s]), (it - 1u) & 1u, abort_flag);
                     tc_fence_after();
                     const uint32_t tO = tmem + lane_sel + 256 + s * 128;
-#pragma unroll
+#pragma unroll 1
                     for (int c4 = 0; c4 < 4; ++c4) {
                         uint32_t o[32];
                         tmem_ld32(tO + c4 * 32, o);
@@ -439,33 +472,43 @@ __device__ __forceinline__ void softmax_loop(const AttnParams& p, Aux* aux, unsi
                         for (int j = 0; j < 32; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * alpha);
                         tmem_st32(tO + c4 * 32, o);
                     }
+                    tmem_wait_st();
                     l *= alpha;
                     lx *= alpha;
                 }
                 m = m_new;
             }
             const float neg_m = (m == -INFINITY) ? 0.f : -m;
-            float sum0 = 0.f, sum1 = 0.f, ex0 = 0.f, ex1 = 0.f;
+            const uint64_t scale2_x2 = pack_f32x2(scale2, scale2), neg_m_x2 = pack_f32x2(neg_m, neg_m);
+            // two packed accumulators each for the exact sum (LSE) and for the sum of the bf16-rounded weights:
+            // the normaliser takes the very numbers P V multiplies by, so that out = sum(p v) / sum(p) stays a
+            // true weighted mean (exact when one key dominates)
+            uint64_t ex_a = 0ull, ex_b = 0ull, rs_a = 0ull, rs_b = 0ull;
 #pragma unroll
             for (int hf = 0; hf < 2; ++hf) {
                 uint32_t pk[32];
 #pragma unroll
                 for (int j = 0; j < 32; ++j) {
-                    const float p0 = fast_exp2(fmaf(sv[hf * 64 + 2 * j], scale2, neg_m));
-                    const float p1 = fast_exp2(fmaf(sv[hf * 64 + 2 * j + 1], scale2, neg_m));
+                    float x0, x1;
+                    unpack_f32x2(fma_f32x2(pack_f32x2(sv[hf * 64 + 2 * j], sv[hf * 64 + 2 * j + 1]), scale2_x2, neg_m_x2), x0, x1);
+                    const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
                     __nv_bfloat162 b2 = __floats2bfloat162_rn(p0, p1);
                     const uint32_t u = *reinterpret_cast<uint32_t*>(&b2);
                     pk[j] = u;
-                    // the row sum takes the bf16-rounded weights, the very numbers P V multiplies by, so
-                    // that out = sum(p v) / sum(p) stays a true weighted mean (exact when one key dominates)
-                    sum0 += __uint_as_float(u << 16);
-                    sum1 += __uint_as_float(u & 0xffff0000u);
-                    ex0 += p0; ex1 += p1;              // the unrounded sum gives the LSE
+                    const uint64_t pe = pack_f32x2(p0, p1);
+                    const uint64_t pr = pack_f32x2(__uint_as_float(u << 16), __uint_as_float(u & 0xffff0000u));
+                    if (j & 1) { ex_b = add_f32x2(ex_b, pe); rs_b = add_f32x2(rs_b, pr); }
+                    else { ex_a = add_f32x2(ex_a, pe); rs_a = add_f32x2(rs_a, pr); }
                 }
                 tmem_st32(tS + hf * 32, pk);
             }
-            l += sum0 + sum1;
-            lx += ex0 + ex1;
+            {
+                float a0, a1, b0, b1;
+                unpack_f32x2(add_f32x2(rs_a, rs_b), a0, a1);
+                unpack_f32x2(add_f32x2(ex_a, ex_b), b0, b1);
+                l += a0 + a1;
+                lx += b0 + b1;
+            }
             tmem_wait_st();
             tc_fence_before();
             mbar_arrive(smem_u32(&aux->p_full[s]));
@@ -485,65 +528,54 @@ __device__ __forceinline__ void softmax_loop(const AttnParams& p, Aux* aux, unsi
         const long long out_row = rr < g.M ? (long long)(g.node_base + rr / G) * p.num_q_heads + g.h * G + rr % G : 0;
         const bool row_ok = write_ok && rr < g.M;
         const bool whole = g.whole();
+        // staging for coalesced stores: the Q blocks are idle now (every MMA of the segment is done); stream 1's
+        // area starts after the (m, l, lx) exchange
+        float* stage = reinterpret_cast<float*>(smem + s * (kQBytes + 4096) + ((threadIdx.x >> 5) & 3) * kStageBytesPerWarp);
+        const long long part_row0 = part_row - (threadIdx.x & 31);
+        // One loop writes both modes.  shared: this warpgroup's own rows, all 128 columns of its O, weight 1 / l.
+        // split: the two streams hold the same rows over disjoint key tiles; they are merged by their maxima and
+        // sums, and this warpgroup writes columns [64 s, 64 s + 64) of the merged rows.
+        float wa, wb = 0.f, lse;
+        uint32_t tOa = tmem + lane_sel + 256 + s * 128, tOb = tmem + lane_sel + 384;
+        bool use_b = false, write_lse = true;
+        int c_first = 0, c_count = 4;
         if (g.shared) {
-            const float inv = l > 0.f ? 1.f / l : 0.f;
-            const uint32_t tO = tmem + lane_sel + 256 + s * 128;
-#pragma unroll
-            for (int c4 = 0; c4 < 4; ++c4) {
-                uint32_t o[32];
-                tmem_ld32(tO + c4 * 32, o);
-                tmem_wait_ld();
-                float v[32];
-#pragma unroll
-                for (int j = 0; j < 32; ++j) v[j] = l > 0.f ? __uint_as_float(o[j]) * inv : 0.f;
-                if (row_ok) {
-                    if (whole) store_row32<true>(p, out_row, part_row, c4 * 32, v);
-                    else store_row32<false>(p, out_row, part_row, c4 * 32, v);
-                }
-            }
-            if (row_ok) {
-                const float lse = lx > 0.f ? (m + __log2f(lx)) * 0.6931471805599453f : -INFINITY;
-                if (whole) { if (p.lse) p.lse[out_row] = lse; }
-                else p.part_lse[part_row] = lse;
-            }
+            wa = l > 0.f ? 1.f / l : 0.f;
+            lse = lx > 0.f ? (m + __log2f(lx)) * 0.6931471805599453f : -INFINITY;
         } else {
-            // merge the two streams (same rows, disjoint key tiles); this warpgroup writes columns [64 s, 64 s + 64)
-            const float m0 = ml[0][row_local][0], l0 = ml[0][row_local][1];
-            const bool has1 = g.iters(1) > 0;
-            const float m1 = has1 ? ml[1][row_local][0] : -INFINITY, l1 = has1 ? ml[1][row_local][1] : 0.f;
-            const float x0 = ml[0][row_local][2], x1 = has1 ? ml[1][row_local][2] : 0.f;
+            const float m0 = ml[0][row_local][0], l0 = ml[0][row_local][1], x0 = ml[0][row_local][2];
+            use_b = g.iters(1) > 0;
+            const float m1 = use_b ? ml[1][row_local][0] : -INFINITY, l1 = use_b ? ml[1][row_local][1] : 0.f;
+            const float x1 = use_b ? ml[1][row_local][2] : 0.f;
             const float mm = fmaxf(m0, m1);
             const float a0 = (m0 == -INFINITY) ? 0.f : fast_exp2(m0 - mm);
             const float a1 = (m1 == -INFINITY) ? 0.f : fast_exp2(m1 - mm);
-            const float lt = a0 * l0 + a1 * l1;
+            const float lt = a0 * l0 + a1 * l1, xt = a0 * x0 + a1 * x1;
             const float inv = lt > 0.f ? 1.f / lt : 0.f;
-            const float w0 = a0 * inv, w1 = a1 * inv;
-            const uint32_t tO0 = tmem + lane_sel + 256, tO1 = tmem + lane_sel + 384;
+            wa = a0 * inv; wb = a1 * inv;
+            lse = xt > 0.f ? (mm + __log2f(xt)) * 0.6931471805599453f : -INFINITY;
+            tOa = tmem + lane_sel + 256;
+            write_lse = s == 0;
+            c_first = 2 * s; c_count = 2;
+        }
+#pragma unroll 1
+        for (int c4 = c_first; c4 < c_first + c_count; ++c4) {
+            uint32_t oa[32], ob[32];
+            tmem_ld32(tOa + c4 * 32, oa);
+            if (use_b) tmem_ld32(tOb + c4 * 32, ob);
+            tmem_wait_ld();
+            float v[32];
 #pragma unroll
-            for (int c2 = 0; c2 < 2; ++c2) {
-                const int col = s * 64 + c2 * 32;
-                uint32_t o0[32], o1[32];
-                tmem_ld32(tO0 + col, o0);
-                if (has1) tmem_ld32(tO1 + col, o1);
-                tmem_wait_ld();
-                float v[32];
-#pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    float x = a0 > 0.f ? __uint_as_float(o0[j]) * w0 : 0.f;
-                    if (has1 && a1 > 0.f) x = fmaf(__uint_as_float(o1[j]), w1, x);
-                    v[j] = x;
-                }
-                if (row_ok) {
-                    if (whole) store_row32<true>(p, out_row, part_row, col, v);
-                    else store_row32<false>(p, out_row, part_row, col, v);
-                }
+            for (int j = 0; j < 32; ++j) {
+                v[j] = __uint_as_float(oa[j]) * wa;           // rows that saw no key have O = 0 and weight 0
+                if (use_b) v[j] = fmaf(__uint_as_float(ob[j]), wb, v[j]);
             }
-            if (row_ok && s == 0) {
-                const float xt = a0 * x0 + a1 * x1;
-                const float lse = xt > 0.f ? (mm + __log2f(xt)) * 0.6931471805599453f : -INFINITY;
-                if (whole) { if (p.lse) p.lse[out_row] = lse; }
-                else p.part_lse[part_row] = lse;
-            }
+            if (whole) store_rows32<true>(p, stage, out_row, row_ok, part_row0, c4 * 32, v);
+            else store_rows32<false>(p, stage, out_row, row_ok, part_row0, c4 * 32, v);
+        }
+        if (row_ok && write_lse) {
+            if (whole) { if (p.lse) p.lse[out_row] = lse; }
+            else p.part_lse[part_row] = lse;
         }
         tc_fence_before();
         ++seg_no;
