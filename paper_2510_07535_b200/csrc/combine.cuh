@@ -9,10 +9,7 @@ namespace owl {
 
 constexpr int kCombineWarps = 8;
 
-// kTwoSlots = false: the partial of (CTA c, unit u) sits in slot c + u.
-// kTwoSlots = true:  a CTA stores at most two partials (only the first and the last unit of its
-//                    piece can be cut): slot 2c if its piece starts inside the unit, else 2c + 1.
-template <int TileKeys, int RowsPerBlock, bool kTwoSlots = false>
+template <int TileKeys, int RowsPerBlock>
 __global__ void __launch_bounds__(kCombineWarps * 32) combine_kernel(const AttnParams p) {
     __shared__ long long s_tile[kMaxBatch + 1];
     __shared__ int s_unit[kMaxBatch + 1];
@@ -46,7 +43,7 @@ __global__ void __launch_bounds__(kCombineWarps * 32) combine_kernel(const AttnP
     if (c0 == c1) return;  // a single CTA saw every key of this unit and wrote the result itself
 
     auto slot_of = [&](int c) -> long long {
-        return kTwoSlots ? 2ll * c + (part.begin(c) < t0 ? 1 : 0) : (long long)c + unit;
+        return (long long)c + unit;   // the partial of (CTA c, unit u) sits in slot c + u
     };
     float mx = -INFINITY;
     for (int c = c0 + lane; c <= c1; c += 32)
@@ -63,6 +60,73 @@ __global__ void __launch_bounds__(kCombineWarps * 32) combine_kernel(const AttnP
             const float4 v = *reinterpret_cast<const float4*>(p.part_o + prow * kHeadDim + lane * 4);
             acc.x += w * v.x; acc.y += w * v.y; acc.z += w * v.z; acc.w += w * v.w;
             sum += w;
+        }
+    }
+    const float inv = sum > 0.f ? 1.f / sum : 0.f;
+    __nv_bfloat162 lo2 = __floats2bfloat162_rn(acc.x * inv, acc.y * inv);
+    __nv_bfloat162 hi2 = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
+    uint2 pk;
+    pk.x = *reinterpret_cast<uint32_t*>(&lo2);
+    pk.y = *reinterpret_cast<uint32_t*>(&hi2);
+    *reinterpret_cast<uint2*>(p.out + row_id * kHeadDim + lane * 4) = pk;
+    if (p.lse && lane == 0) p.lse[row_id] = sum > 0.f ? mx + logf(sum) : -INFINITY;
+}
+
+
+// LSE merge for the tcgen05 split-KV pass.  That pass leaves its schedule in global memory (first flat
+// tile of every sequence, totals, choice of partition), so this kernel rebuilds nothing: one warp per
+// output row finds the CTAs whose pieces cut the row's unit and merges their partials in CTA order.
+// A CTA stores at most two partials: slot 2c if its piece starts inside the unit, else 2c + 1.
+__global__ void __launch_bounds__(kCombineWarps * 32) combine_sched_kernel(const AttnParams p) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const long long row_id = (long long)blockIdx.x * kCombineWarps + warp;
+    if (row_id >= (long long)p.total_nodes * p.num_q_heads) return;
+    const int n = (int)(row_id / p.num_q_heads), hq = (int)(row_id % p.num_q_heads);
+    int b;
+    if (p.node_offsets) {
+        int lo = 0, hi = p.batch;  // largest b with node_offsets[b] <= n
+        while (hi - lo > 1) { int mid = (lo + hi) >> 1; if (p.node_offsets[mid] <= n) lo = mid; else hi = mid; }
+        b = lo;
+    } else {
+        b = n / p.nodes_uniform;
+    }
+    if (p.seq_bad[b] == p.epoch) return;
+    const long long seq_begin = p.sched_seq_begin[b];
+    const int tiles = (int)((p.sched_seq_begin[b + 1] - seq_begin) / p.num_kv_heads);
+    if (tiles == 0) return;
+    const SchedHeader hdr = *p.sched_header;
+    Partition part;
+    part.init(hdr.total_tiles, p.num_ctas, hdr.units, hdr.uniform_tiles);
+    const int G = p.group;
+    const int lrow = (n - seq_node_base(p, b)) * G + hq % G;
+    const long long t0 = seq_begin + (long long)(hq / G) * tiles;
+    const int c0 = part.owner(t0), c1 = part.owner(t0 + tiles - 1);
+    if (c0 == c1) return;  // a single CTA saw every key of this unit and wrote the result itself
+    const int count = c1 - c0 + 1;
+
+    auto row_of = [&](int c) -> long long { return (2ll * c + (part.begin(c) < t0 ? 1 : 0)) * p.rows_per_slot + lrow; };
+    float mx = -INFINITY;
+    for (int i = lane; i < count; i += 32) mx = fmaxf(mx, p.part_lse[row_of(c0 + i)]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    float sum = 0.f;
+    if (mx > -INFINITY) {
+        for (int base = 0; base < count; base += 32) {
+            const int mine = base + lane;
+            long long prow = 0;
+            float w = 0.f;
+            if (mine < count) { prow = row_of(c0 + mine); w = __expf(p.part_lse[prow] - mx); }
+            const int m = min(32, count - base);
+#pragma unroll 4
+            for (int j = 0; j < m; ++j) {
+                const float wj = __shfl_sync(0xffffffffu, w, j);
+                const long long pj = __shfl_sync(0xffffffffu, prow, j);
+                const float4 v = *reinterpret_cast<const float4*>(p.part_o + pj * kHeadDim + lane * 4);
+                acc.x += wj * v.x; acc.y += wj * v.y; acc.z += wj * v.z; acc.w += wj * v.w;
+                sum += wj;
+            }
         }
     }
     const float inv = sum > 0.f ? 1.f / sum : 0.f;

@@ -18,6 +18,8 @@ constexpr int kErrBadTree = -4;
 constexpr int kErrBadPage = -5;
 constexpr int kErrTimeout = -6;
 
+struct SchedHeader;
+
 // Problem description handed to every kernel of the attention path.
 struct AttnParams {
     const __nv_bfloat16* q;
@@ -33,6 +35,8 @@ struct AttnParams {
     float* part_lse;              // [slots, rows_per_slot] fp32, natural-log partial LSE (-inf if empty)
     int32_t* status;              // device status word (0 = ok, first error wins)
     int32_t* seq_bad;             // [B] epoch of the call in which the sequence was found malformed
+    long long* sched_seq_begin;   // [B + 1] first flat tile of every sequence (tcgen05 path; written by its CTA 0)
+    SchedHeader* sched_header;    // (tcgen05 path)
     int32_t epoch;
     int32_t batch, total_nodes, nodes_uniform, max_nodes;
     int32_t num_q_heads, num_kv_heads, group;  // group = Hq / Hkv
@@ -69,17 +73,56 @@ struct SeqSched {
     int node_base;
 };
 
+// Cut of the flat tile range [0, total) into `ctas` pieces, one per CTA.
+//   flat:    contiguous, nearly equal pieces; a piece may start and end inside a unit.
+//   aligned: only when every unit has the same number of tiles (`unit_tiles`) and there are at least as
+//            many CTAs as units: unit u is cut into base + (u < urem) nearly equal pieces, so no piece
+//            crosses a unit boundary.  Chosen when its largest piece is smaller than the flat piece plus
+//            what a unit boundary costs a CTA (pipeline drain, epilogue, new Q), counted in tiles.
+constexpr int kBoundaryPenaltyTiles = 5;
 struct Partition {
     long long total, q;
     int rem, ctas;
+    int unit_tiles, base, urem;   // aligned mode iff unit_tiles > 0
     __device__ __host__ void init(long long total_, int ctas_) {
         total = total_; ctas = ctas_; q = total_ / ctas_; rem = (int)(total_ % ctas_);
+        unit_tiles = 0; base = 0; urem = 0;
     }
-    __device__ __host__ long long begin(int c) const { return (long long)c * q + (c < rem ? c : rem); }
+    __device__ __host__ void init(long long total_, int ctas_, int units, int uniform_tiles) {
+        init(total_, ctas_);
+        if (uniform_tiles > 0 && units > 1 && units <= ctas_) {
+            const int b = ctas_ / units;
+            const long long cost_aligned = (uniform_tiles + b - 1) / b;
+            const long long cost_flat = (total_ + ctas_ - 1) / ctas_ + kBoundaryPenaltyTiles;
+            if (cost_aligned < cost_flat) { unit_tiles = uniform_tiles; base = b; urem = ctas_ % units; }
+        }
+    }
+    __device__ __host__ long long begin(int c) const {
+        if (unit_tiles == 0) return (long long)c * q + (c < rem ? c : rem);
+        const int big = urem * (base + 1);
+        int u, k, cu;
+        if (c < big) { u = c / (base + 1); k = c - u * (base + 1); cu = base + 1; }
+        else { u = urem + (c - big) / base; k = (c - big) - (u - urem) * base; cu = base; }
+        const int qq = unit_tiles / cu, rr = unit_tiles % cu;
+        return (long long)u * unit_tiles + (long long)k * qq + (k < rr ? k : rr);
+    }
     __device__ __host__ int owner(long long t) const {
-        long long big = (long long)rem * (q + 1);
-        return t < big ? (int)(t / (q + 1)) : rem + (int)((t - big) / q);
+        if (unit_tiles == 0) {
+            long long big = (long long)rem * (q + 1);
+            return t < big ? (int)(t / (q + 1)) : rem + (int)((t - big) / q);
+        }
+        const int u = (int)(t / unit_tiles), local = (int)(t - (long long)u * unit_tiles);
+        const int cu = base + (u < urem ? 1 : 0), c0 = u * base + (u < urem ? u : urem);
+        const int qq = unit_tiles / cu, rr = unit_tiles % cu, bigl = rr * (qq + 1);
+        return c0 + (local < bigl ? local / (qq + 1) : rr + (local - bigl) / qq);
     }
+};
+
+// What the split-KV pass leaves for the combine kernel: totals and the choice of partition.
+struct SchedHeader {
+    long long total_tiles;
+    int uniform_tiles;   // tiles per unit if every schedulable sequence has the same count, else 0
+    int units;
 };
 
 __device__ __forceinline__ int seq_nodes(const AttnParams& p, int b) {

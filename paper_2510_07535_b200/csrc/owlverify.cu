@@ -28,6 +28,8 @@ struct owl_ctx {
     float* part_lse = nullptr;
     int32_t* status = nullptr;
     int32_t* seq_bad = nullptr;
+    long long* sched_seq_begin = nullptr;
+    SchedHeader* sched_header = nullptr;
     unsigned long long* part_keys = nullptr;
     long long part_keys_len = 0;
     // tcgen05 path: tensor maps over the caller's K and V caches, re-encoded when the cache changes
@@ -161,6 +163,8 @@ int owl_create(owl_ctx** out, int device, const owl_dims* max_dims) {
     }
     alloc((void**)&ctx->status, sizeof(int32_t));
     alloc((void**)&ctx->seq_bad, (size_t)max_dims->batch * sizeof(int32_t));
+    alloc((void**)&ctx->sched_seq_begin, ((size_t)max_dims->batch + 1) * sizeof(long long));
+    alloc((void**)&ctx->sched_header, sizeof(SchedHeader));
     if (acc) {
         ctx->part_keys_len = (long long)max_dims->total_nodes * ((max_dims->vocab + kArgmaxChunk - 1) / kArgmaxChunk);
         alloc((void**)&ctx->part_keys, (size_t)ctx->part_keys_len * sizeof(unsigned long long));
@@ -192,6 +196,8 @@ int owl_destroy(owl_ctx* ctx) {
     cudaFree(ctx->part_lse);
     cudaFree(ctx->status);
     cudaFree(ctx->seq_bad);
+    cudaFree(ctx->sched_seq_begin);
+    cudaFree(ctx->sched_header);
     cudaFree(ctx->part_keys);
     for (auto& s : ctx->stg) cudaFree(s.p);
     for (auto& ev : ctx->ev)
@@ -232,6 +238,8 @@ int owl_verify_attn(owl_ctx* ctx, const owl_dims* d, const void* q, const void* 
     p.part_lse = ctx->part_lse;
     p.status = ctx->status;
     p.seq_bad = ctx->seq_bad;
+    p.sched_seq_begin = ctx->sched_seq_begin;
+    p.sched_header = ctx->sched_header;
     p.epoch = ++ctx->epoch;
     p.batch = d->batch;
     p.total_nodes = d->total_nodes;
@@ -269,7 +277,7 @@ int owl_verify_attn(owl_ctx* ctx, const owl_dims* d, const void* q, const void* 
             p, ctx->kmap, ctx->vmap);
         ++ctx->launches;
         if (ctx->profiling) cudaEventRecord(ctx->ev[1], stream);
-        combine_kernel<umma_path::kTileKeys, umma_path::kRows, true><<<grid, kCombineWarps * 32, 0, stream>>>(p);
+        combine_sched_kernel<<<grid, kCombineWarps * 32, 0, stream>>>(p);
     } else {
         mma_path::verify_attn_mma_kernel<<<ctx->num_ctas, mma_path::kThreads, mma_path::kSmemBytes, stream>>>(p);
         ++ctx->launches;

@@ -67,6 +67,7 @@ struct Aux {
     long long scan_tiles[12];
     long long total_tiles;
     int scan_units[12];
+    int scan_tmin[12], scan_tmax[12];
     int sched_unit_begin;
     short parent[kMaxNodes];
     unsigned long long anc[kMaxNodes];
@@ -128,18 +129,21 @@ struct Walker {
     }
 };
 
-// Block-wide: totals of the flat tile range and the first sequence of this CTA's piece.
+// Block-wide: totals of the flat tile range, the choice of partition and the first sequence of this
+// CTA's piece.  CTA 0 also leaves the per-sequence prefix and the header for the combine kernel.
 __device__ __forceinline__ void build_walk(const AttnParams& p, Aux* aux, Walker& w) {
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int per = (p.batch + kThreads - 1) / kThreads;
     const int b_lo = tid * per, b_hi = min(p.batch, b_lo + per);
     long long my_tiles = 0;
-    int my_units = 0;
+    int my_units = 0, tmin = 0x7fffffff, tmax = 0;
     for (int b = b_lo; b < b_hi; ++b) {
         const int n = seq_nodes(p, b), L = p.ctx_lens[b];
         if (seq_shape_ok(p, b, n, L)) {
-            my_tiles += (long long)((L + n + kTileKeys - 1) / kTileKeys) * p.num_kv_heads;
+            const int tiles = (L + n + kTileKeys - 1) / kTileKeys;
+            my_tiles += (long long)tiles * p.num_kv_heads;
             my_units += p.num_kv_heads;
+            tmin = min(tmin, tiles); tmax = max(tmax, tiles);
         } else {
             report(p.status, seq_tree_shape_ok(p, b, n) ? kErrBadPage : kErrBadTree);
             p.seq_bad[b] = p.epoch;
@@ -153,22 +157,45 @@ __device__ __forceinline__ void build_walk(const AttnParams& p, Aux* aux, Walker
         const int vu = __shfl_up_sync(0xffffffffu, inc_u, o);
         if (lane >= o) { inc_t += vt; inc_u += vu; }
     }
-    if (lane == 31) { aux->scan_tiles[warp] = inc_t; aux->scan_units[warp] = inc_u; }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        tmin = min(tmin, __shfl_xor_sync(0xffffffffu, tmin, o));
+        tmax = max(tmax, __shfl_xor_sync(0xffffffffu, tmax, o));
+    }
+    if (lane == 31) { aux->scan_tiles[warp] = inc_t; aux->scan_units[warp] = inc_u; aux->scan_tmin[warp] = tmin; aux->scan_tmax[warp] = tmax; }
     __syncthreads();
-    long long off_t = 0;
-    int off_u = 0;
-    for (int w2 = 0; w2 < warp; ++w2) { off_t += aux->scan_tiles[w2]; off_u += aux->scan_units[w2]; }
+    long long off_t = 0, total = 0;
+    int off_u = 0, units = 0;
+#pragma unroll 1
+    for (int w2 = 0; w2 < kThreads / 32; ++w2) {
+        if (w2 < warp) { off_t += aux->scan_tiles[w2]; off_u += aux->scan_units[w2]; }
+        total += aux->scan_tiles[w2]; units += aux->scan_units[w2];
+        tmin = min(tmin, aux->scan_tmin[w2]); tmax = max(tmax, aux->scan_tmax[w2]);
+    }
+    const int uniform_tiles = (units > 0 && tmin == tmax) ? tmin : 0;
     const long long excl_t = off_t + inc_t - my_tiles;
     const int excl_u = off_u + inc_u - my_units;
-    if (tid == kThreads - 1) aux->total_tiles = off_t + inc_t;
-    __syncthreads();
     Partition part;
-    part.init(aux->total_tiles, gridDim.x);
+    part.init(total, gridDim.x, units, uniform_tiles);
     const long long t_begin = part.begin(blockIdx.x), t_end = part.begin(blockIdx.x + 1);
     if (t_begin < t_end && my_tiles > 0 && t_begin >= excl_t && t_begin < excl_t + my_tiles) {
         aux->sched_b0 = b_lo;                 // the walker skips ahead from the first sequence of this thread
         aux->sched_tile_begin = excl_t;
         aux->sched_unit_begin = excl_u;
+    }
+    if (blockIdx.x == 0) {
+        long long run = excl_t;
+        for (int b = b_lo; b < b_hi; ++b) {
+            p.sched_seq_begin[b] = run;
+            const int n = seq_nodes(p, b), L = p.ctx_lens[b];
+            if (seq_shape_ok(p, b, n, L)) run += (long long)((L + n + kTileKeys - 1) / kTileKeys) * p.num_kv_heads;
+        }
+        if (tid == 0) {
+            p.sched_seq_begin[p.batch] = total;
+            p.sched_header->total_tiles = total;
+            p.sched_header->uniform_tiles = uniform_tiles;
+            p.sched_header->units = units;
+        }
     }
     __syncthreads();
     w.t = t_begin;
@@ -176,6 +203,71 @@ __device__ __forceinline__ void build_walk(const AttnParams& p, Aux* aux, Walker
     w.b = aux->sched_b0;
     w.seq_begin = aux->sched_tile_begin;
     w.unit_begin = aux->sched_unit_begin;
+}
+
+// Batches of at most 32 sequences: every warp derives the same schedule on its own (lane b holds sequence
+// b, prefix sums by shuffle), with no shared memory and no CTA-wide barrier, so that each role can start
+// as soon as its own loads have returned.
+__device__ __forceinline__ void build_walk_small(const AttnParams& p, Walker& w) {
+    const int lane = threadIdx.x & 31;
+    int n = 0, L = 0, node_base = 0, tiles = 0;
+    bool ok = false;
+    if (lane < p.batch) {
+        n = seq_nodes(p, lane);
+        L = p.ctx_lens[lane];
+        node_base = seq_node_base(p, lane);
+        ok = seq_shape_ok(p, lane, n, L);
+        tiles = ok ? (L + n + kTileKeys - 1) / kTileKeys : 0;
+        if (!ok && threadIdx.x < 32) {
+            report(p.status, seq_tree_shape_ok(p, lane, n) ? kErrBadPage : kErrBadTree);
+            p.seq_bad[lane] = p.epoch;
+        }
+    }
+    const long long my_tiles = (long long)tiles * p.num_kv_heads;
+    const int my_units = ok ? p.num_kv_heads : 0;
+    long long inc_t = my_tiles;
+    int inc_u = my_units, tmin = ok ? tiles : 0x7fffffff, tmax = ok ? tiles : 0;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const long long vt = __shfl_up_sync(0xffffffffu, inc_t, o);
+        const int vu = __shfl_up_sync(0xffffffffu, inc_u, o);
+        if (lane >= o) { inc_t += vt; inc_u += vu; }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        tmin = min(tmin, __shfl_xor_sync(0xffffffffu, tmin, o));
+        tmax = max(tmax, __shfl_xor_sync(0xffffffffu, tmax, o));
+    }
+    const long long total = __shfl_sync(0xffffffffu, inc_t, 31);
+    const int units = __shfl_sync(0xffffffffu, inc_u, 31);
+    const int uniform_tiles = (units > 0 && tmin == tmax) ? tmin : 0;
+    const long long excl_t = inc_t - my_tiles;
+    const int excl_u = inc_u - my_units;
+    Partition part;
+    part.init(total, gridDim.x, units, uniform_tiles);
+    const long long t_begin = part.begin(blockIdx.x), t_end = part.begin(blockIdx.x + 1);
+    const unsigned owner = __ballot_sync(0xffffffffu, my_tiles > 0 && t_begin >= excl_t && t_begin < excl_t + my_tiles);
+    if (blockIdx.x == 0 && threadIdx.x < 32) {
+        if (lane < p.batch) p.sched_seq_begin[lane] = excl_t;
+        if (lane == 0) {
+            p.sched_seq_begin[p.batch] = total;
+            p.sched_header->total_tiles = total;
+            p.sched_header->uniform_tiles = uniform_tiles;
+            p.sched_header->units = units;
+        }
+    }
+    w.t = t_begin;
+    w.t_end = (t_begin < t_end && owner) ? t_end : t_begin;
+    const int b0 = owner ? __ffs(owner) - 1 : 0;
+    w.b = b0;
+    w.seq_begin = __shfl_sync(0xffffffffu, excl_t, b0);
+    w.unit_begin = __shfl_sync(0xffffffffu, excl_u, b0);
+    w.cur_b = b0;
+    w.cur_n = __shfl_sync(0xffffffffu, n, b0);
+    w.cur_L = __shfl_sync(0xffffffffu, L, b0);
+    w.cur_node_base = __shfl_sync(0xffffffffu, node_base, b0);
+    w.cur_tiles = __shfl_sync(0xffffffffu, tiles, b0);
+    w.cur_ok = true;
 }
 
 // ------------------------------------------------------------------------------------------ producer
@@ -609,13 +701,13 @@ verify_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap 
         tma_prefetch_desc(&vmap);
     }
     if (warp == 0) { tmem_alloc(smem_u32(&aux->tmem_base), kTmemCols); tmem_relinquish(); }
+    Walker w;
+    if (p.batch <= 32) build_walk_small(p, w);     // its global loads overlap the set-up above
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = aux->tmem_base;
-
-    Walker w;
-    build_walk(p, aux, w);
+    if (p.batch > 32) build_walk(p, aux, w);
 
     // registers move from the warpgroup of the producer / MMA warps to the two softmax warpgroups,
     // whose threads each hold a 128-column row of S: 128 x 56 + 256 x 224 = 384 x 168
