@@ -67,7 +67,7 @@ def ncu_traffic(workload_name):
 class ClockSampler(threading.Thread):
     """Polls SM clock and throttle reasons through NVML (read-only) while the timed region runs."""
 
-    def __init__(self, index: int, period: float = 0.02):
+    def __init__(self, index: int, period: float = 0.001):
         super().__init__(daemon=True)
         self.index, self.period = index, period
         self.samples, self.reasons = [], set()

@@ -167,9 +167,9 @@ int owl_verify_step_host(owl_ctx* ctx, const owl_dims* dims, const void* q_h, co
  * cudaMalloc - and the device-wide synchronisation it can imply - is forbidden.  Such callers
  * cannot use owl_create, which allocates a workspace.  This call takes no context and allocates
  * nothing, neither with cudaMalloc nor through any library: its scratch (one 64-bit arg-max key
- * per logits row and 8192-float vocabulary chunk, plus the status word) is a fixed array inside
+ * per logits row and 8192-float vocabulary chunk, a progress counter per sequence, the status word) is a fixed array inside
  * the library image.  The price: every GPU on which the library is loaded holds that array,
- * (OWL_STATIC_MAX_KEYS + 32) * 8 bytes = 128.25 KiB, until the process exits.
+ * (OWL_STATIC_MAX_KEYS + 32 + 1024) * 8 bytes = 136.25 KiB, until the process exits.
  *
  * Limit: total_nodes * ceil(vocab / 8192) <= OWL_STATIC_MAX_KEYS (e.g. 1024 nodes at a 128256-entry
  * vocabulary); anything larger returns OWL_ERR_TOO_LARGE and launches nothing.
@@ -209,7 +209,7 @@ const char* owl_last_error(const owl_ctx* ctx);
 int64_t owl_launch_count(const owl_ctx* ctx);
 
 /* Seconds of device time (CUDA events on `stream`) of the most recent call's kernels, by
- * kernel: t[0] verify-attention, t[1] combine, t[2] arg-max, t[3] acceptance walk.  Only
+ * kernel: t[0] verify-attention, t[1] combine, t[2] arg-max with the acceptance walk (one kernel), t[3] = 0.  Only
  * measured while profiling is on (owl_set_profiling(ctx, 1)); synchronises `stream`. */
 int owl_set_profiling(owl_ctx* ctx, int on);
 int owl_last_kernel_times(owl_ctx* ctx, void* stream, double t[4]);

@@ -7,9 +7,12 @@
 // give one key per (row, vocabulary chunk), stored to part_keys[row][chunk] (no atomics, nothing
 // to initialise).
 //
-// Kernel 2 (one CTA per sequence) reduces the chunk keys to arg-max tokens, evaluates for every node
-// whether all edges on its root path match (draft token == parent's arg-max), picks the deepest
-// matching node (lowest index among equals) and writes accept_len / accept_path / bonus_token.
+// The CTA that stores the last chunk key of a sequence (a per-sequence counter, bumped after a
+// __threadfence; nobody waits for anybody) then does that sequence's walk in the same launch: it reduces
+// the chunk keys to arg-max tokens, evaluates for every node whether all edges on its root path match
+// (draft token == parent's arg-max), picks the deepest matching node (lowest index among equals) and
+// writes accept_len / accept_path / bonus_token.  Calls alternate between two sets of counters and clear the
+// idle one, so no separate clearing pass is needed.
 #pragma once
 
 #include "owl_common.cuh"
@@ -17,6 +20,7 @@
 namespace owl {
 
 constexpr int kArgmaxThreads = 256;
+static_assert(kArgmaxThreads >= kMaxNodes, "the walk needs one thread per node");
 constexpr int kArgmaxChunk = 8192;  // floats per CTA: 8 x float4 per thread
 
 struct AcceptParams {
@@ -29,6 +33,9 @@ struct AcceptParams {
     int32_t* bonus_token;
     int32_t* node_argmax;
     unsigned long long* part_keys;   // [total_nodes, chunks]
+    unsigned int* seq_counter;       // [2, batch]: chunk keys of the sequence stored so far; set epoch & 1 is in use
+    uint32_t epoch;                  // call number: the other set is cleared for the next call
+    int32_t counter_stride;          // distance between the two sets
     int32_t* status;
     int32_t batch, total_nodes, nodes_uniform, max_nodes, vocab, path_stride, chunks;
 };
@@ -41,7 +48,58 @@ __device__ __forceinline__ unsigned long long argmax_key(float x, uint32_t idx) 
     return ((unsigned long long)u << 32) | (uint32_t)(~idx);
 }
 
+// Called by every thread of the CTA (threads >= kMaxNodes only keep the barriers company).
+__device__ __forceinline__ void accept_walk_seq(const AcceptParams& p, const int b) {
+    const int i = threadIdx.x;
+    const int base = p.node_offsets ? p.node_offsets[b] : b * p.nodes_uniform;
+    const int n = p.node_offsets ? p.node_offsets[b + 1] - base : p.nodes_uniform;
+    __shared__ int s_parent[kMaxNodes], s_am[kMaxNodes], s_tok[kMaxNodes];
+    __shared__ int s_bad, s_win;
+    if (i == 0) { s_bad = (n < 1 || n > p.max_nodes || n > p.path_stride || base < 0 || base + n > p.total_nodes) ? 1 : 0; s_win = 0; }
+    __syncthreads();
+    if (s_bad) { if (i == 0) report(p.status, kErrBadTree); return; }
+    if (i < n) {
+        const int pi = p.tree_parent[base + i];
+        s_parent[i] = pi;
+        s_tok[i] = p.draft_tokens[base + i];
+        unsigned long long k = 0;
+        const unsigned long long* pk = p.part_keys + (long long)(base + i) * p.chunks;
+        for (int c = 0; c < p.chunks; ++c) { const unsigned long long v = __ldcg(pk + c); k = v > k ? v : k; }
+        const int am = (int)(~(uint32_t)(k & 0xffffffffull));
+        s_am[i] = am;
+        if (p.node_argmax) p.node_argmax[base + i] = am;
+        if ((i == 0 && pi != -1) || (i > 0 && (pi < 0 || pi >= i))) atomicExch(&s_bad, 1);
+    }
+    __syncthreads();
+    if (s_bad) { if (i == 0) report(p.status, kErrBadTree); return; }
+
+    // ok(i): every edge on the root path of i matches; depth(i): number of edges
+    int key = 0;
+    if (i < n) {
+        bool ok = true;
+        int depth = 0;
+        for (int c = i; s_parent[c] >= 0 && depth < kMaxNodes; c = s_parent[c], ++depth)
+            ok = ok && s_tok[c] >= 0 && s_tok[c] == s_am[s_parent[c]];
+        if (ok) key = ((depth + 1) << 8) | (kMaxNodes - 1 - i);   // deeper first, then lower index
+    }
+    atomicMax(&s_win, key);
+    __syncthreads();
+    if (i == 0) {
+        const int win = kMaxNodes - 1 - (s_win & 0xff);
+        const int len = s_win >> 8;
+        p.accept_len[b] = len;
+        p.bonus_token[b] = s_am[win];
+        int32_t* path = p.accept_path + (long long)b * p.path_stride;
+        for (int k = len; k < p.path_stride; ++k) path[k] = -1;
+        int k = len - 1;
+        for (int c = win; c >= 0 && k >= 0; c = s_parent[c]) path[k--] = c;
+    }
+}
+
 __global__ void __launch_bounds__(kArgmaxThreads) argmax_partial_kernel(const AcceptParams p) {
+    // may be launched as a programmatic dependent of the kernel before it in the stream: nothing is read
+    // before that kernel has completed (a no-op in an ordinary launch)
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int row = blockIdx.y;
     const long long V = p.vocab;
     const long long c0 = (long long)blockIdx.x * kArgmaxChunk;
@@ -88,58 +146,34 @@ __global__ void __launch_bounds__(kArgmaxThreads) argmax_partial_kernel(const Ac
     __shared__ unsigned long long s_key[kArgmaxThreads / 32];
     if ((threadIdx.x & 31) == 0) s_key[threadIdx.x >> 5] = key;
     __syncthreads();
+    __shared__ int s_walk_b;
     if (threadIdx.x == 0) {
 #pragma unroll
         for (int w = 1; w < kArgmaxThreads / 32; ++w) key = s_key[w] > key ? s_key[w] : key;
         p.part_keys[(long long)row * p.chunks + blockIdx.x] = key;
-    }
-}
-
-__global__ void __launch_bounds__(kMaxNodes) accept_walk_kernel(const AcceptParams p) {
-    const int b = blockIdx.x, i = threadIdx.x;
-    const int base = p.node_offsets ? p.node_offsets[b] : b * p.nodes_uniform;
-    const int n = p.node_offsets ? p.node_offsets[b + 1] - base : p.nodes_uniform;
-    __shared__ int s_parent[kMaxNodes], s_am[kMaxNodes], s_tok[kMaxNodes];
-    __shared__ int s_bad, s_win;
-    if (i == 0) { s_bad = (n < 1 || n > p.max_nodes || n > p.path_stride || base < 0 || base + n > p.total_nodes) ? 1 : 0; s_win = 0; }
-    __syncthreads();
-    if (s_bad) { if (i == 0) report(p.status, kErrBadTree); return; }
-    if (i < n) {
-        const int pi = p.tree_parent[base + i];
-        s_parent[i] = pi;
-        s_tok[i] = p.draft_tokens[base + i];
-        unsigned long long k = 0;
-        const unsigned long long* pk = p.part_keys + (long long)(base + i) * p.chunks;
-        for (int c = 0; c < p.chunks; ++c) k = pk[c] > k ? pk[c] : k;
-        const int am = (int)(~(uint32_t)(k & 0xffffffffull));
-        s_am[i] = am;
-        if (p.node_argmax) p.node_argmax[base + i] = am;
-        if ((i == 0 && pi != -1) || (i > 0 && (pi < 0 || pi >= i))) atomicExch(&s_bad, 1);
+        // which sequence owns this row, and is this the last of its chunk keys?
+        int b, n_b;
+        if (p.node_offsets) {
+            int lo = 0, hi = p.batch;   // largest b with node_offsets[b] <= row
+            while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (p.node_offsets[mid] <= row) lo = mid; else hi = mid; }
+            b = lo;
+            n_b = p.node_offsets[b + 1] - p.node_offsets[b];
+        } else {
+            b = row / p.nodes_uniform;
+            n_b = p.nodes_uniform;
+        }
+        __threadfence();
+        // two sets of counters: this call counts in set (epoch & 1) and clears the other one for the next call,
+        // so a counter left dirty by malformed input never survives
+        unsigned int* ctr = p.seq_counter + (size_t)(p.epoch & 1u) * p.counter_stride + b;
+        p.seq_counter[(size_t)((p.epoch + 1u) & 1u) * p.counter_stride + b] = 0u;
+        const unsigned int want = atomicAdd(ctr, 1u) + 1u;
+        if ((long long)want == (long long)p.chunks * n_b) *ctr = 0u;   // a completed counter is left clean as well
+        s_walk_b = ((long long)want == (long long)p.chunks * n_b) ? b : -1;
+        __threadfence();
     }
     __syncthreads();
-    if (s_bad) { if (i == 0) report(p.status, kErrBadTree); return; }
-
-    // ok(i): every edge on the root path of i matches; depth(i): number of edges
-    int key = 0;
-    if (i < n) {
-        bool ok = true;
-        int depth = 0;
-        for (int c = i; s_parent[c] >= 0 && depth < kMaxNodes; c = s_parent[c], ++depth)
-            ok = ok && s_tok[c] >= 0 && s_tok[c] == s_am[s_parent[c]];
-        if (ok) key = ((depth + 1) << 8) | (kMaxNodes - 1 - i);   // deeper first, then lower index
-    }
-    atomicMax(&s_win, key);
-    __syncthreads();
-    if (i == 0) {
-        const int win = kMaxNodes - 1 - (s_win & 0xff);
-        const int len = s_win >> 8;
-        p.accept_len[b] = len;
-        p.bonus_token[b] = s_am[win];
-        int32_t* path = p.accept_path + (long long)b * p.path_stride;
-        for (int k = len; k < p.path_stride; ++k) path[k] = -1;
-        int k = len - 1;
-        for (int c = win; c >= 0 && k >= 0; c = s_parent[c]) path[k--] = c;
-    }
+    if (s_walk_b >= 0) accept_walk_seq(p, s_walk_b);
 }
 
 }  // namespace owl

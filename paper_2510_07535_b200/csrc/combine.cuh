@@ -78,6 +78,10 @@ __global__ void __launch_bounds__(kCombineWarps * 32) combine_kernel(const AttnP
 // output row finds the CTAs whose pieces cut the row's unit and merges their partials in CTA order.
 // A CTA stores at most two partials: slot 2c if its piece starts inside the unit, else 2c + 1.
 __global__ void __launch_bounds__(kCombineWarps * 32) combine_sched_kernel(const AttnParams p) {
+    // launched as a programmatic dependent of the split-KV pass: wait here until that grid has completed and
+    // its writes are visible (a no-op in an ordinary launch), then let the next kernel in the stream queue up
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const long long row_id = (long long)blockIdx.x * kCombineWarps + warp;
     if (row_id >= (long long)p.total_nodes * p.num_q_heads) return;
@@ -115,17 +119,27 @@ __global__ void __launch_bounds__(kCombineWarps * 32) combine_sched_kernel(const
     if (mx > -INFINITY) {
         for (int base = 0; base < count; base += 32) {
             const int mine = base + lane;
-            long long prow = 0;
+            long long prow = row_of(c0);          // any valid row: padding entries get weight 0
             float w = 0.f;
             if (mine < count) { prow = row_of(c0 + mine); w = __expf(p.part_lse[prow] - mx); }
             const int m = min(32, count - base);
-#pragma unroll 4
-            for (int j = 0; j < m; ++j) {
-                const float wj = __shfl_sync(0xffffffffu, w, j);
-                const long long pj = __shfl_sync(0xffffffffu, prow, j);
-                const float4 v = *reinterpret_cast<const float4*>(p.part_o + pj * kHeadDim + lane * 4);
-                acc.x += wj * v.x; acc.y += wj * v.y; acc.z += wj * v.z; acc.w += wj * v.w;
-                sum += wj;
+            // 16 partial rows in flight per lane, then their weighted sum, in CTA order
+            for (int j0 = 0; j0 < m; j0 += 16) {
+                float4 v[16];
+                float wj[16];
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    wj[j] = __shfl_sync(0xffffffffu, w, (j0 + j) & 31);
+                    const long long pj = __shfl_sync(0xffffffffu, prow, (j0 + j) & 31);
+                    v[j] = __ldcg(reinterpret_cast<const float4*>(p.part_o + pj * kHeadDim + lane * 4));
+                }
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    if (j0 + j < m) {
+                        acc.x += wj[j] * v[j].x; acc.y += wj[j] * v[j].y; acc.z += wj[j] * v[j].z; acc.w += wj[j] * v[j].w;
+                        sum += wj[j];
+                    }
+                }
             }
         }
     }

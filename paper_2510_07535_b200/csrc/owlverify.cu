@@ -6,6 +6,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <atomic>
 #include <mutex>
 #include <new>
 
@@ -31,6 +32,8 @@ struct owl_ctx {
     long long* sched_seq_begin = nullptr;
     SchedHeader* sched_header = nullptr;
     unsigned long long* part_keys = nullptr;
+    unsigned int* seq_counter = nullptr;
+    uint32_t accept_epoch = 0;
     long long part_keys_len = 0;
     // tcgen05 path: tensor maps over the caller's K and V caches, re-encoded when the cache changes
     bool use_umma = true;
@@ -63,6 +66,23 @@ struct DeviceGuard {
 int cuda_fail(owl_ctx* ctx, cudaError_t e, const char* what) {
     if (ctx) snprintf(ctx->err, sizeof ctx->err, "%s: %s", what, cudaGetErrorString(e));
     return OWL_ERR_CUDA;
+}
+
+// Launch `kernel(arg)` so that it may be scheduled while the kernel before it in the stream is still running
+// (programmatic dependent launch); the kernel itself waits (griddepcontrol.wait) before it reads anything.
+template <typename Arg>
+cudaError_t launch_dependent(void (*kernel)(Arg), dim3 grid, dim3 block, cudaStream_t stream, const Arg& arg) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, arg);
 }
 
 int log2_exact(int v) {
@@ -168,6 +188,8 @@ int owl_create(owl_ctx** out, int device, const owl_dims* max_dims) {
     if (acc) {
         ctx->part_keys_len = (long long)max_dims->total_nodes * ((max_dims->vocab + kArgmaxChunk - 1) / kArgmaxChunk);
         alloc((void**)&ctx->part_keys, (size_t)ctx->part_keys_len * sizeof(unsigned long long));
+        alloc((void**)&ctx->seq_counter, 2 * (size_t)max_dims->batch * sizeof(unsigned int));
+        if (ok) ok = cudaMemset(ctx->seq_counter, 0, 2 * (size_t)max_dims->batch * sizeof(unsigned int)) == cudaSuccess;
     }
     if (ok) {
         ok = cudaMemset(ctx->status, 0, sizeof(int32_t)) == cudaSuccess &&
@@ -199,6 +221,7 @@ int owl_destroy(owl_ctx* ctx) {
     cudaFree(ctx->sched_seq_begin);
     cudaFree(ctx->sched_header);
     cudaFree(ctx->part_keys);
+    cudaFree(ctx->seq_counter);
     for (auto& s : ctx->stg) cudaFree(s.p);
     for (auto& ev : ctx->ev)
         if (ev) cudaEventDestroy(ev);
@@ -277,7 +300,7 @@ int owl_verify_attn(owl_ctx* ctx, const owl_dims* d, const void* q, const void* 
             p, ctx->kmap, ctx->vmap);
         ++ctx->launches;
         if (ctx->profiling) cudaEventRecord(ctx->ev[1], stream);
-        combine_sched_kernel<<<grid, kCombineWarps * 32, 0, stream>>>(p);
+        launch_dependent(combine_sched_kernel, dim3(grid), dim3(kCombineWarps * 32), stream, p);
     } else {
         mma_path::verify_attn_mma_kernel<<<ctx->num_ctas, mma_path::kThreads, mma_path::kSmemBytes, stream>>>(p);
         ++ctx->launches;
@@ -325,14 +348,15 @@ int owl_tree_accept(owl_ctx* ctx, const owl_dims* d, const float* logits, const 
     p.vocab = d->vocab;
     p.path_stride = d->path_stride;
 
+    p.seq_counter = ctx->seq_counter;
+    p.counter_stride = ctx->max_dims.batch;
+    p.epoch = ++ctx->accept_epoch;
     if (ctx->profiling) cudaEventRecord(ctx->ev[3], stream);
     dim3 grid((unsigned)chunks, (unsigned)d->total_nodes);
-    argmax_partial_kernel<<<grid, kArgmaxThreads, 0, stream>>>(p);
+    launch_dependent(argmax_partial_kernel, grid, dim3(kArgmaxThreads), stream, p);   // the walk runs in the CTA that finishes a sequence
     ++ctx->launches;
     if (ctx->profiling) cudaEventRecord(ctx->ev[4], stream);
-    accept_walk_kernel<<<d->batch, kMaxNodes, 0, stream>>>(p);
-    ++ctx->launches;
-    if (ctx->profiling) { cudaEventRecord(ctx->ev[5], stream); ctx->ev_accept_valid = true; }
+    if (ctx->profiling) ctx->ev_accept_valid = true;
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(ctx, e, "owl_tree_accept launch");
     return OWL_OK;
@@ -420,7 +444,6 @@ int owl_last_kernel_times(owl_ctx* ctx, void* stream_, double t[4]) {
     }
     if (ctx->ev_accept_valid) {
         if (cudaEventElapsedTime(&ms, ctx->ev[3], ctx->ev[4]) == cudaSuccess) t[2] = ms * 1e-3;
-        if (cudaEventElapsedTime(&ms, ctx->ev[4], ctx->ev[5]) == cudaSuccess) t[3] = ms * 1e-3;
     }
     return OWL_OK;
 }
@@ -437,7 +460,7 @@ int owl_last_kernel_times(owl_ctx* ctx, void* stream_, double t[4]) {
 // those callers cannot own an owl_ctx.  For them the arg-max scratch (one 64-bit key per logits
 // row and 8192-float vocabulary chunk) and the device status word live in the fixed array below,
 // which is part of the loaded library image: every device that loads the library holds its
-// (OWL_STATIC_MAX_KEYS + 32) * 8 bytes until the process exits, whether or not this entry point is ever called.
+// (OWL_STATIC_MAX_KEYS + 32 + 1024) * 8 bytes until the process exits, whether or not this entry point is ever called.
 //
 // The array's name is only a host-side handle here; the device address handed to the kernels
 // comes from cudaGetSymbolAddress, looked up once per device with that device current.
@@ -446,9 +469,11 @@ namespace {
 
 constexpr int kStaticMaxKeys = OWL_STATIC_MAX_KEYS;            // (row, chunk) keys
 constexpr int kStaticStatusWords = 32;                         // one 256-byte line for the status word
+constexpr int kStaticCounterWords = kMaxBatch;                 // per-sequence progress counters of the scan
 constexpr int kStaticMaxDevices = 64;
 
-static __device__ __align__(256) unsigned long long g_accept_scratch[kStaticMaxKeys + kStaticStatusWords];
+static __device__ __align__(256) unsigned long long g_accept_scratch[kStaticMaxKeys + kStaticStatusWords + kStaticCounterWords];
+std::atomic<uint32_t> g_static_epoch{0};
 
 unsigned long long* g_static_addr[kStaticMaxDevices] = {nullptr};
 bool g_static_ready[kStaticMaxDevices] = {false};
@@ -509,9 +534,11 @@ extern "C" int owl_tree_accept_static(const owl_dims* d, const float* logits, co
     p.max_nodes = d->max_nodes;
     p.vocab = d->vocab;
     p.path_stride = d->path_stride;
+    p.seq_counter = reinterpret_cast<unsigned int*>(scratch + kStaticMaxKeys + kStaticStatusWords);   // 2 x kMaxBatch
+    p.counter_stride = kMaxBatch;
+    p.epoch = ++g_static_epoch;
     dim3 grid((unsigned)chunks, (unsigned)d->total_nodes);
     argmax_partial_kernel<<<grid, kArgmaxThreads, 0, stream>>>(p);
-    accept_walk_kernel<<<d->batch, kMaxNodes, 0, stream>>>(p);
     if (cudaGetLastError() != cudaSuccess) return OWL_ERR_CUDA;
     return OWL_OK;
 }

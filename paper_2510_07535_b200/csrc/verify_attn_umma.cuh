@@ -681,6 +681,8 @@ verify_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap 
     Aux* aux = reinterpret_cast<Aux*>(smem + kAuxOff);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t smem_base = smem_u32(smem);
+    // the combine kernel is launched as a programmatic dependent: let it queue up behind this grid's CTAs
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (smem_base & 1023u) {                       // operand tiles must sit on swizzle-atom boundaries
         if (tid == 0) report(p.status, kErrTimeout);
         return;
