@@ -51,12 +51,25 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     return ok != 0;
 }
 
-// Bounded wait.  Returns false at once if the CTA's abort flag is up.  Otherwise spins on try_wait;
+// Non-blocking test of a phase (try_wait may suspend the thread for a while before it answers).
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}\n"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+
+// Bounded wait.  A phase that has already completed returns true after one poll; otherwise the wait
+// returns false at once if the CTA's abort flag is up, and else spins on try_wait;
 // every 256 failed polls it looks at the abort flag and at the wall clock, and after `kWaitLimitNs`
 // it raises the abort flag itself and gives up.  A false return means: do not touch what the wait
 // guarded; carry on with the (finite) control flow so that every CTA-level barrier is still reached.
 constexpr uint64_t kWaitLimitNs = 2000000000ull;   // 2 s: three orders of magnitude above any real wait
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;      // the common case costs one poll
     if (*abort_flag) return false;
     uint64_t t0 = 0;
     for (uint32_t polls = 0;; ++polls) {

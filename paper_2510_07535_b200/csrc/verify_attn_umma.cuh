@@ -343,43 +343,60 @@ __device__ __forceinline__ void mma_loop(const AttnParams& p, Aux* aux, uint32_t
 #pragma unroll 1
             for (int s = 0; s < 2; ++s) {
                 const bool last_reader = !g.shared || s == 1;
-                if (i >= 0 && i < n_it[s]) {
+                const bool do_pv = i >= 0 && i < n_it[s], do_qk = i + 1 < n_it[s];
+                uint32_t v_slot = 0, k_slot = 0;
+                // the K / V tiles were requested long ago: make sure of them first, so that nothing stands between
+                // the arrival of P and the issue of both products
+                if (do_pv) {
                     const uint32_t item = item_base + 2u * (uint32_t)(g.tile(s, i) - g.tile0) + 1u;
-                    const uint32_t slot = item % kSlots, ph = (item / kSlots) & 1u;
+                    v_slot = item % kSlots;
+                    ok = mbar_wait(smem_u32(&aux->full[v_slot]), (item / kSlots) & 1u, abort_flag) && ok;
+                }
+                uint32_t k_phase = 0;
+                bool k_ready = false;
+                if (do_qk) {
+                    const uint32_t item = item_base + 2u * (uint32_t)(g.tile(s, i + 1) - g.tile0);
+                    k_slot = item % kSlots;
+                    k_phase = (item / kSlots) & 1u;
+                    k_ready = mbar_test_wait(smem_u32(&aux->full[k_slot]), k_phase);   // a look, no waiting yet
+                }
+                if (do_pv) {
                     ok = mbar_wait(smem_u32(&aux->p_full[s]), it[s] & 1u, abort_flag) && ok;
-                    ok = mbar_wait(smem_u32(&aux->full[slot]), ph, abort_flag) && ok;
-                    tc_fence_after();
-                    if (lane == 0 && ok) {
-                        const uint32_t va = ring + slot * kSlotBytes;
-#pragma unroll
-                        for (int ks = 0; ks < 8; ++ks)
-                            umma_ts(tmem + 256 + s * 128, tmem + s * 128 + ks * 8,
-                                    umma_smem_desc_sw128(va + ks * 4096, 1024, 2048), idesc_pv, (i | ks) ? 1u : 0u);
-                        umma_commit(smem_u32(&aux->o_done[s]));
-                        if (last_reader) umma_commit(smem_u32(&aux->empty[slot]));
-                    }
-                    __syncwarp();
                     ++it[s];
                 }
-                if (i + 1 < n_it[s]) {
-                    const uint32_t item = item_base + 2u * (uint32_t)(g.tile(s, i + 1) - g.tile0);
-                    const uint32_t slot = item % kSlots, ph = (item / kSlots) & 1u;
-                    ok = mbar_wait(smem_u32(&aux->full[slot]), ph, abort_flag) && ok;
+                tc_fence_after();
+                if (lane == 0 && ok) {
+                    if (do_pv) {
+                        // one descriptor per batch; the k-steps only move its start-address field (units of 16 bytes)
+                        const uint64_t vdesc = umma_smem_desc_sw128(ring + v_slot * kSlotBytes, 1024, 2048);
+                        const uint32_t tO = tmem + 256 + s * 128, tP = tmem + s * 128;
+#pragma unroll
+                        for (int ks = 0; ks < 8; ++ks)
+                            umma_ts(tO, tP + ks * 8, vdesc + (uint64_t)(ks * 4096 >> 4), idesc_pv, (i | ks) ? 1u : 0u);
+                        umma_commit(smem_u32(&aux->o_done[s]));
+                        if (last_reader) umma_commit(smem_u32(&aux->empty[v_slot]));
+                    }
+                }
+                if (do_qk && !k_ready) {     // the next K tile may still be on its way (its slot was freed late)
+                    ok = mbar_wait(smem_u32(&aux->full[k_slot]), k_phase, abort_flag) && ok;
                     tc_fence_after();
-                    if (lane == 0 && ok) {
-                        const uint32_t qa = smem_base + (g.shared ? s : 0) * kQBytes;
-                        const uint32_t ka = ring + slot * kSlotBytes;
+                }
+                if (lane == 0 && ok) {
+                    if (do_qk) {
+                        const uint64_t qdesc = umma_smem_desc_sw128(smem_base + (g.shared ? s : 0) * kQBytes, 16, 1024);
+                        const uint64_t kdesc = umma_smem_desc_sw128(ring + k_slot * kSlotBytes, 16, 2048);
+                        const uint32_t tS = tmem + s * 128;
 #pragma unroll
                         for (int hf = 0; hf < 2; ++hf)
 #pragma unroll
                             for (int ks = 0; ks < 4; ++ks)
-                                umma_ss(tmem + s * 128, umma_smem_desc_sw128(qa + hf * 16384 + ks * 32, 16, 1024),
-                                        umma_smem_desc_sw128(ka + hf * 1024 + ks * 32, 16, 2048), idesc_qk, (hf | ks) ? 1u : 0u);
+                                umma_ss(tS, qdesc + (uint64_t)((hf * 16384 + ks * 32) >> 4),
+                                        kdesc + (uint64_t)((hf * 1024 + ks * 32) >> 4), idesc_qk, (hf | ks) ? 1u : 0u);
                         umma_commit(smem_u32(&aux->s_full[s]));
-                        if (last_reader) umma_commit(smem_u32(&aux->empty[slot]));
+                        if (last_reader) umma_commit(smem_u32(&aux->empty[k_slot]));
                     }
-                    __syncwarp();
                 }
+                __syncwarp();
             }
         }
         item_base += 2u * (uint32_t)(g.tile1 - g.tile0);
