@@ -729,14 +729,14 @@ verify_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap 
     if (p.batch > 32) build_walk(p, aux, w);
 
     // registers move from the warpgroup of the producer / MMA warps to the two softmax warpgroups,
-    // whose threads each hold a 128-column row of S: 128 x 56 + 256 x 224 = 384 x 168
+    // whose threads each hold a 128-column row of S: 128 x 72 + 256 x 216 = 384 x 168, the registers the CTA was launched with
     uint32_t items = 0;
     if (warp < 4) {
-        asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
         if (warp == 0) producer_loop(p, &kmap, &vmap, aux, smem_base + kRingOff, w, items);
         else if (warp == 1) mma_loop(p, aux, smem_base, tmem, w);
     } else {
-        asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
         softmax_loop(p, aux, smem, tmem, w, warp >= 8 ? 1 : 0);
     }
 
