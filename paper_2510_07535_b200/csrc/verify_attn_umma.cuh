@@ -370,9 +370,10 @@ __device__ __forceinline__ void mma_loop(const AttnParams& p, Aux* aux, uint32_t
                         // one descriptor per batch; the k-steps only move its start-address field (units of 16 bytes)
                         const uint64_t vdesc = umma_smem_desc_sw128(ring + v_slot * kSlotBytes, 1024, 2048);
                         const uint32_t tO = tmem + 256 + s * 128, tP = tmem + s * 128;
+                        const uint32_t v_lo = (uint32_t)vdesc, v_hi = (uint32_t)(vdesc >> 32);
 #pragma unroll
                         for (int ks = 0; ks < 8; ++ks)
-                            umma_ts(tO, tP + ks * 8, vdesc + (uint64_t)(ks * 4096 >> 4), idesc_pv, (i | ks) ? 1u : 0u);
+                            umma_ts_lh(tO, tP + ks * 8, v_lo + (uint32_t)(ks * 4096 >> 4), v_hi, idesc_pv, (i | ks) ? 1u : 0u);
                         umma_commit(smem_u32(&aux->o_done[s]));
                         if (last_reader) umma_commit(smem_u32(&aux->empty[v_slot]));
                     }
@@ -386,12 +387,14 @@ __device__ __forceinline__ void mma_loop(const AttnParams& p, Aux* aux, uint32_t
                         const uint64_t qdesc = umma_smem_desc_sw128(smem_base + (g.shared ? s : 0) * kQBytes, 16, 1024);
                         const uint64_t kdesc = umma_smem_desc_sw128(ring + k_slot * kSlotBytes, 16, 2048);
                         const uint32_t tS = tmem + s * 128;
+                        const uint32_t q_lo = (uint32_t)qdesc, q_hi = (uint32_t)(qdesc >> 32);
+                        const uint32_t k_lo = (uint32_t)kdesc, k_hi = (uint32_t)(kdesc >> 32);
 #pragma unroll
                         for (int hf = 0; hf < 2; ++hf)
 #pragma unroll
                             for (int ks = 0; ks < 4; ++ks)
-                                umma_ss(tS, qdesc + (uint64_t)((hf * 16384 + ks * 32) >> 4),
-                                        kdesc + (uint64_t)((hf * 1024 + ks * 32) >> 4), idesc_qk, (hf | ks) ? 1u : 0u);
+                                umma_ss_lh(tS, q_lo + (uint32_t)((hf * 16384 + ks * 32) >> 4), q_hi,
+                                           k_lo + (uint32_t)((hf * 1024 + ks * 32) >> 4), k_hi, idesc_qk, (hf | ks) ? 1u : 0u);
                         umma_commit(smem_u32(&aux->s_full[s]));
                         if (last_reader) umma_commit(smem_u32(&aux->empty[k_slot]));
                     }
