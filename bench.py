@@ -317,12 +317,12 @@ def run_gpu(args, rank, world, local_rank):
                        "l2": f"rotating {copies} input copies ({copies * step_bytes / 1e6:.0f} MB > L2)"},
             "verify_step_us": step_s * 1e6,
             "frac_of_hbm_peak": step_bytes / step_s / 1e9 / peak,
-            "kernel_us": {"verify_attn": kt[0] * 1e6, "combine": kt[1] * 1e6, "argmax": kt[2] * 1e6, "accept_walk": kt[3] * 1e6},
+            "kernel_us": {"verify_attn": kt[0] * 1e6, "combine": kt[1] * 1e6, "argmax_accept": kt[2] * 1e6},
             "bytes_per_step": {"attention": attn_b, "logits": logit_b},
             "roofline": {"bound": "hbm", "kernel": "verify_attn", "achieved": achieved, "peak": peak, "unit": "GB/s",
                          "frac": achieved / peak if achieved else None, "peak_kind": f"of {peak_kind}",
                          "traffic": ncu_traffic(spec.name)},
-            "accept_gbs": logit_b / (kt[2] + kt[3]) / 1e9 if kt[2] > 0 else None,
+            "accept_gbs": logit_b / kt[2] / 1e9 if kt[2] > 0 else None,
             "e2e": {"value": world * step_bytes / e2e_s / 1e9, "unit": "GB/s", "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "us_per_step": e2e_s * 1e6, "steps": e2e_steps},
             "gpu_launches": launches,
