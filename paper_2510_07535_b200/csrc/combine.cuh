@@ -94,15 +94,18 @@ __global__ void __launch_bounds__(kCombineWarps * 32) combine_sched_kernel(const
     } else {
         b = n / p.nodes_uniform;
     }
-    if (p.seq_bad[b] == p.epoch) return;
-    const long long seq_begin = p.sched_seq_begin[b];
-    const int tiles = (int)((p.sched_seq_begin[b + 1] - seq_begin) / p.num_kv_heads);
-    if (tiles == 0) return;
+    // independent loads first, tests afterwards: one round trip instead of four
+    const int bad_epoch = p.seq_bad[b];
+    const long long seq_begin = p.sched_seq_begin[b], seq_end = p.sched_seq_begin[b + 1];
     const SchedHeader hdr = *p.sched_header;
+    const int node_base = seq_node_base(p, b);
+    if (bad_epoch == p.epoch) return;
+    const int tiles = (int)((seq_end - seq_begin) / p.num_kv_heads);
+    if (tiles == 0) return;
     Partition part;
     part.init(hdr.total_tiles, p.num_ctas, hdr.units, hdr.uniform_tiles);
     const int G = p.group;
-    const int lrow = (n - seq_node_base(p, b)) * G + hq % G;
+    const int lrow = (n - node_base) * G + hq % G;
     const long long t0 = seq_begin + (long long)(hq / G) * tiles;
     const int c0 = part.owner(t0), c1 = part.owner(t0 + tiles - 1);
     if (c0 == c1) return;  // a single CTA saw every key of this unit and wrote the result itself
