@@ -64,7 +64,14 @@ __device__ __forceinline__ void accept_walk_seq(const AcceptParams& p, const int
         s_tok[i] = p.draft_tokens[base + i];
         unsigned long long k = 0;
         const unsigned long long* pk = p.part_keys + (long long)(base + i) * p.chunks;
-        for (int c = 0; c < p.chunks; ++c) { const unsigned long long v = __ldcg(pk + c); k = v > k ? v : k; }
+        // independent loads, eight in flight (a dependent one-by-one walk would cost a memory round trip per chunk)
+        for (int c0 = 0; c0 < p.chunks; c0 += 8) {
+            unsigned long long v[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) v[j] = c0 + j < p.chunks ? __ldcg(pk + c0 + j) : 0ull;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) k = v[j] > k ? v[j] : k;
+        }
         const int am = (int)(~(uint32_t)(k & 0xffffffffull));
         s_am[i] = am;
         if (p.node_argmax) p.node_argmax[base + i] = am;
@@ -100,6 +107,7 @@ __global__ void __launch_bounds__(kArgmaxThreads) argmax_partial_kernel(const Ac
     // may be launched as a programmatic dependent of the kernel before it in the stream: nothing is read
     // before that kernel has completed (a no-op in an ordinary launch)
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next kernel may queue up; it waits likewise
     const int row = blockIdx.y;
     const long long V = p.vocab;
     const long long c0 = (long long)blockIdx.x * kArgmaxChunk;

@@ -296,8 +296,19 @@ int owl_verify_attn(owl_ctx* ctx, const owl_dims* d, const void* q, const void* 
     const long long rows = (long long)d->total_nodes * d->num_q_heads;
     const unsigned grid = (unsigned)((rows + kCombineWarps - 1) / kCombineWarps);
     if (ctx->use_umma) {
-        umma_path::verify_attn_umma_kernel<<<ctx->num_ctas, umma_path::kThreads, umma_path::kSmemBytes, stream>>>(
-            p, ctx->kmap, ctx->vmap);
+        {
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3(ctx->num_ctas);
+            cfg.blockDim = dim3(umma_path::kThreads);
+            cfg.dynamicSmemBytes = umma_path::kSmemBytes;
+            cfg.stream = stream;
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+            attr[0].val.programmaticStreamSerializationAllowed = 1;
+            cfg.attrs = attr;
+            cfg.numAttrs = 1;
+            cudaLaunchKernelEx(&cfg, umma_path::verify_attn_umma_kernel, p, ctx->kmap, ctx->vmap);
+        }
         ++ctx->launches;
         if (ctx->profiling) cudaEventRecord(ctx->ev[1], stream);
         launch_dependent(combine_sched_kernel, dim3(grid), dim3(kCombineWarps * 32), stream, p);

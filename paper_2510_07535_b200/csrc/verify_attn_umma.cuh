@@ -723,6 +723,9 @@ verify_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap 
         tma_prefetch_desc(&vmap);
     }
     if (warp == 0) { tmem_alloc(smem_u32(&aux->tmem_base), kTmemCols); tmem_relinquish(); }
+    // launched as a programmatic dependent itself: everything above touched no input; from here on the kernel
+    // before this one in the stream has completed (a no-op in an ordinary launch)
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     Walker w;
     if (p.batch <= 32) build_walk_small(p, w);     // its global loads overlap the set-up above
     tc_fence_before();
