@@ -347,10 +347,12 @@ __device__ __forceinline__ void mma_loop(const AttnParams& p, Aux* aux, uint32_t
                 uint32_t v_slot = 0, k_slot = 0;
                 // the K / V tiles were requested long ago: make sure of them first, so that nothing stands between
                 // the arrival of P and the issue of both products
+                // (when both streams read every tile, stream 1 finds what stream 0 has just made sure of)
+                const bool seen = g.shared && s == 1;
                 if (do_pv) {
                     const uint32_t item = item_base + 2u * (uint32_t)(g.tile(s, i) - g.tile0) + 1u;
                     v_slot = item % kSlots;
-                    ok = mbar_wait(smem_u32(&aux->full[v_slot]), (item / kSlots) & 1u, abort_flag) && ok;
+                    if (!seen) ok = mbar_wait(smem_u32(&aux->full[v_slot]), (item / kSlots) & 1u, abort_flag) && ok;
                 }
                 uint32_t k_phase = 0;
                 bool k_ready = false;
@@ -358,7 +360,7 @@ __device__ __forceinline__ void mma_loop(const AttnParams& p, Aux* aux, uint32_t
                     const uint32_t item = item_base + 2u * (uint32_t)(g.tile(s, i + 1) - g.tile0);
                     k_slot = item % kSlots;
                     k_phase = (item / kSlots) & 1u;
-                    k_ready = mbar_test_wait(smem_u32(&aux->full[k_slot]), k_phase);   // a look, no waiting yet
+                    k_ready = seen || mbar_test_wait(smem_u32(&aux->full[k_slot]), k_phase);   // a look, no waiting yet
                 }
                 if (do_pv) {
                     ok = mbar_wait(smem_u32(&aux->p_full[s]), it[s] & 1u, abort_flag) && ok;
