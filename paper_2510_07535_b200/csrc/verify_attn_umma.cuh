@@ -363,7 +363,9 @@ __device__ __forceinline__ void mma_loop(const AttnParams& p, Aux* aux, uint32_t
                     k_ready = seen || mbar_test_wait(smem_u32(&aux->full[k_slot]), k_phase);   // a look, no waiting yet
                 }
                 if (do_pv) {
-                    ok = mbar_wait(smem_u32(&aux->p_full[s]), it[s] & 1u, abort_flag) && ok;
+                    // P of this stream: hardware barrier 4 + s, the warpgroup's 128 threads arrive, this warp waits
+                    // (every arrival is executed whatever happens, so the wait always ends)
+                    asm volatile("bar.sync %0, 160;" ::"r"(4 + s) : "memory");
                     ++it[s];
                 }
                 tc_fence_after();
@@ -625,7 +627,7 @@ __device__ __forceinline__ void softmax_loop(const AttnParams& p, Aux* aux, unsi
             }
             tmem_wait_st();
             tc_fence_before();
-            mbar_arrive(smem_u32(&aux->p_full[s]));
+            asm volatile("bar.arrive %0, 160;" ::"r"(4 + s) : "memory");
             ++it;
         }
 
