@@ -378,7 +378,7 @@ __device__ __forceinline__ void mma_loop(const AttnParams& p, Aux* aux, uint32_t
 #pragma unroll
                         for (int ks = 0; ks < 8; ++ks)
                             umma_ts_lh(tO, tP + ks * 8, v_lo + (uint32_t)(ks * 4096 >> 4), v_hi, idesc_pv, (i | ks) ? 1u : 0u);
-                        umma_commit(smem_u32(&aux->o_done[s]));
+                        if (i == n_it[s] - 1) umma_commit(smem_u32(&aux->o_done[s]));   // only the segment end waits for it
                         if (last_reader) umma_commit(smem_u32(&aux->empty[v_slot]));
                     }
                 }
@@ -469,7 +469,7 @@ __device__ __forceinline__ void softmax_loop(const AttnParams& p, Aux* aux, unsi
     const uint32_t tS = tmem + lane_sel + s * 128;
     const float scale2 = p.sm_scale * 1.4426950408889634f;   // > 0 (checked on the host)
     const int G = p.group;
-    uint32_t it = 0, seg_no = 0;
+    uint32_t it = 0, seg_no = 0, od_phase = 0;   // od_phase: segments of this stream that issued a product
     Segment g;
 
     while (w.next(p, g)) {
@@ -576,7 +576,8 @@ __device__ __forceinline__ void softmax_loop(const AttnParams& p, Aux* aux, unsi
             if (__any_sync(0xffffffffu, need)) {
                 const float alpha = (m_new == -INFINITY) ? 1.f : fast_exp2(m - m_new);
                 if (i > 0) {
-                    mbar_wait(smem_u32(&aux->o_done[s]), (it - 1u) & 1u, abort_flag);
+                    // S of this tile is here, and its product was issued after O += P V of the tile before: the
+                    // commit that announced S covers that product too, so O may be touched now
                     tc_fence_after();
                     const uint32_t tO = tmem + lane_sel + 256 + s * 128;
 #pragma unroll 1
@@ -632,7 +633,7 @@ __device__ __forceinline__ void softmax_loop(const AttnParams& p, Aux* aux, unsi
         }
 
         // ---- segment end: every product of this stream has completed
-        if (n_it > 0) mbar_wait(smem_u32(&aux->o_done[s]), (it - 1u) & 1u, abort_flag);
+        if (n_it > 0) { mbar_wait(smem_u32(&aux->o_done[s]), od_phase & 1u, abort_flag); ++od_phase; }
         tc_fence_after();
         // split mode: the streams exchange (m, l, lx) through the second Q block, which only the shared mode uses
         float (*ml)[128][3] = reinterpret_cast<float (*)[128][3]>(smem + kQBytes);
