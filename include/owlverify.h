@@ -141,6 +141,21 @@ int owl_tree_accept(owl_ctx* ctx, const owl_dims* dims, const float* logits,
                     int32_t* bonus_token, int32_t* node_argmax, void* stream);
 
 /*
+ * One whole verify step on device buffers: owl_verify_attn and owl_tree_accept of the same batch
+ * (Section 3.2.2 "Decode Stage" followed by the acceptance of the Introduction), arguments as in those
+ * two calls.  The two halves do not depend on each other (the logits are an input), so a small acceptance
+ * scan (about one wave of CTAs or less) is queued on a stream of the context's own and runs beside the
+ * tail of the attention pass; the call forks from `stream` and joins it again, i.e. for the caller
+ * everything happens in stream order.  Larger scans follow the attention pass on `stream`.
+ * Asynchronous; errors as in the two calls.
+ */
+int owl_verify_step(owl_ctx* ctx, const owl_dims* dims, const void* q, const void* k_cache, const void* v_cache,
+                    const int32_t* block_table, const int32_t* ctx_lens, const int32_t* node_offsets,
+                    const int32_t* tree_parent, void* out, float* lse, const float* logits,
+                    const int32_t* draft_tokens, int32_t* accept_len, int32_t* accept_path,
+                    int32_t* bonus_token, int32_t* node_argmax, void* stream);
+
+/*
  * One whole verify step from HOST memory: copies every input to device staging buffers owned by
  * the context (grown on demand, so the first call at a given size allocates), runs
  * owl_verify_attn and owl_tree_accept, copies the results back and synchronises `stream`.

@@ -52,6 +52,8 @@ def load_library() -> ctypes.CDLL:
     lib.owl_tree_accept.argtypes = [vp, dp] + [vp] * 9
     lib.owl_tree_accept_static.restype = i32
     lib.owl_tree_accept_static.argtypes = [dp] + [vp] * 10
+    lib.owl_verify_step.restype = i32
+    lib.owl_verify_step.argtypes = [vp, dp] + [vp] * 16
     lib.owl_verify_step_host.restype = i32
     lib.owl_verify_step_host.argtypes = [vp, dp] + [vp] * 15
     lib.owl_get_status.restype = i32
@@ -138,6 +140,21 @@ class OwlContext:
             _ptr(node_argmax, torch.int32, dev, "node_argmax"), _stream(dev))
         if check and rc != OWL_OK:
             raise OwlError(rc, "owl_tree_accept", self.last_error())
+        return rc
+
+    def owl_verify_step(self, dims: OwlDims, q, k_cache, v_cache, block_table, ctx_lens, node_offsets, tree_parent, out, lse,
+                        logits, draft_tokens, accept_len, accept_path, bonus_token, node_argmax=None, check: bool = True) -> int:
+        dev = self.device
+        i32, bf, f32 = torch.int32, torch.bfloat16, torch.float32
+        rc = self.lib.owl_verify_step(
+            self._h, ctypes.byref(dims), _ptr(q, bf, dev, "q"), _ptr(k_cache, bf, dev, "k_cache"), _ptr(v_cache, bf, dev, "v_cache"),
+            _ptr(block_table, i32, dev, "block_table"), _ptr(ctx_lens, i32, dev, "ctx_lens"),
+            _ptr(node_offsets, i32, dev, "node_offsets"), _ptr(tree_parent, i32, dev, "tree_parent"), _ptr(out, bf, dev, "out"),
+            _ptr(lse, f32, dev, "lse"), _ptr(logits, f32, dev, "logits"), _ptr(draft_tokens, i32, dev, "draft_tokens"),
+            _ptr(accept_len, i32, dev, "accept_len"), _ptr(accept_path, i32, dev, "accept_path"),
+            _ptr(bonus_token, i32, dev, "bonus_token"), _ptr(node_argmax, i32, dev, "node_argmax"), _stream(dev))
+        if check and rc != OWL_OK:
+            raise OwlError(rc, "owl_verify_step", self.last_error())
         return rc
 
     def owl_verify_step_host(self, dims: OwlDims, q, k_cache, v_cache, block_table, ctx_lens, node_offsets,

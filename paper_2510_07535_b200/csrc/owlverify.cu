@@ -46,6 +46,9 @@ struct owl_ctx {
     int64_t launches = 0;
     bool profiling = false;
     cudaEvent_t ev[6] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
+    // owl_verify_step: acceptance runs on a stream of its own beside the attention's tail and the combine
+    cudaStream_t side = nullptr;
+    cudaEvent_t fork = nullptr, join = nullptr;
     bool ev_attn_valid = false, ev_accept_valid = false;
     char err[256] = {0};
     // device staging of owl_verify_step_host (grown on demand)
@@ -196,6 +199,9 @@ int owl_create(owl_ctx** out, int device, const owl_dims* max_dims) {
              cudaMemset(ctx->seq_bad, 0, (size_t)max_dims->batch * sizeof(int32_t)) == cudaSuccess;
     }
     for (int i = 0; ok && i < 6; ++i) ok = cudaEventCreate(&ctx->ev[i]) == cudaSuccess;
+    if (ok) ok = cudaStreamCreateWithFlags(&ctx->side, cudaStreamNonBlocking) == cudaSuccess &&
+                 cudaEventCreateWithFlags(&ctx->fork, cudaEventDisableTiming) == cudaSuccess &&
+                 cudaEventCreateWithFlags(&ctx->join, cudaEventDisableTiming) == cudaSuccess;
     if (ok && attn) {
         ok = cudaFuncSetAttribute(mma_path::verify_attn_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                   mma_path::kSmemBytes) == cudaSuccess &&
@@ -225,6 +231,9 @@ int owl_destroy(owl_ctx* ctx) {
     for (auto& s : ctx->stg) cudaFree(s.p);
     for (auto& ev : ctx->ev)
         if (ev) cudaEventDestroy(ev);
+    if (ctx->fork) cudaEventDestroy(ctx->fork);
+    if (ctx->join) cudaEventDestroy(ctx->join);
+    if (ctx->side) cudaStreamDestroy(ctx->side);
     delete ctx;
     return OWL_OK;
 }
@@ -370,6 +379,42 @@ int owl_tree_accept(owl_ctx* ctx, const owl_dims* d, const float* logits, const 
     if (ctx->profiling) ctx->ev_accept_valid = true;
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(ctx, e, "owl_tree_accept launch");
+    return OWL_OK;
+}
+
+int owl_verify_step(owl_ctx* ctx, const owl_dims* d, const void* q, const void* k_cache, const void* v_cache,
+                    const int32_t* block_table, const int32_t* ctx_lens, const int32_t* node_offsets,
+                    const int32_t* tree_parent, void* out, float* lse, const float* logits, const int32_t* draft_tokens,
+                    int32_t* accept_len, int32_t* accept_path, int32_t* bonus_token, int32_t* node_argmax, void* stream_) {
+    if (!ctx) return OWL_ERR_INVALID_ARG;
+    int rc = check_dims(d, true, true);
+    if (rc != OWL_OK) return rc;
+    DeviceGuard guard(ctx->device);
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    // A scan of at most about one wave of CTAs hides in the tail of the attention pass; a larger one would
+    // take SMs from the persistent attention CTAs at their start, so it simply follows in stream order.
+    const long long scan_ctas = (long long)d->total_nodes * ((d->vocab + kArgmaxChunk - 1) / kArgmaxChunk);
+    if (scan_ctas > 1024) {
+        rc = owl_verify_attn(ctx, d, q, k_cache, v_cache, block_table, ctx_lens, node_offsets, tree_parent, out, lse, stream_);
+        if (rc != OWL_OK) return rc;
+        return owl_tree_accept(ctx, d, logits, draft_tokens, node_offsets, tree_parent, accept_len, accept_path, bonus_token,
+                               node_argmax, stream_);
+    }
+    // fork: what the caller queued before this call is complete before either half starts
+    cudaError_t e = cudaEventRecord(ctx->fork, stream);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->side, ctx->fork, 0);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "owl_verify_step fork");
+    rc = owl_verify_attn(ctx, d, q, k_cache, v_cache, block_table, ctx_lens, node_offsets, tree_parent, out, lse, stream_);
+    int rc2 = OWL_OK;
+    if (rc == OWL_OK)
+        rc2 = owl_tree_accept(ctx, d, logits, draft_tokens, node_offsets, tree_parent, accept_len, accept_path, bonus_token,
+                              node_argmax, ctx->side);
+    // join (always, so that the side stream never runs ahead of the caller's)
+    e = cudaEventRecord(ctx->join, ctx->side);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(stream, ctx->join, 0);
+    if (rc != OWL_OK) return rc;
+    if (rc2 != OWL_OK) return rc2;
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "owl_verify_step join");
     return OWL_OK;
 }
 

@@ -73,9 +73,12 @@ class DeviceWorkload:
 
     def step(self, ctx: OwlContext) -> None:
         """One verify step: attention of the drafted nodes, then acceptance from the logits."""
-        self.attn(ctx)
-        if self.logits is not None:
-            self.accept(ctx)
+        if self.logits is None:
+            self.attn(ctx)
+        else:
+            ctx.owl_verify_step(self.dims, self.q, self.k_cache, self.v_cache, self.block_table, self.ctx_lens,
+                                self.node_offsets, self.tree_parent, self.out, self.lse, self.logits, self.draft_tokens,
+                                self.accept_len, self.accept_path, self.bonus_token, self.node_argmax)
 
     def out_f32(self) -> np.ndarray:
         return self.out.float().cpu().numpy()
