@@ -112,38 +112,38 @@ __global__ void __launch_bounds__(kCombineWarps * 32) combine_sched_kernel(const
     const int count = c1 - c0 + 1;
 
     auto row_of = [&](int c) -> long long { return (2ll * c + (part.begin(c) < t0 ? 1 : 0)) * p.rows_per_slot + lrow; };
-    float mx = -INFINITY;
-    for (int i = lane; i < count; i += 32) mx = fmaxf(mx, p.part_lse[row_of(c0 + i)]);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-
+    // Partials are taken 16 at a time: lane j (< 16) of a group owns partial base + j.  The row loads do not
+    // depend on the LSE values, so both go out together: one memory round trip per group, and units cut into
+    // at most 16 pieces - the usual case - need a single group.  Groups are folded online (running maximum).
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    float sum = 0.f;
-    if (mx > -INFINITY) {
-        for (int base = 0; base < count; base += 32) {
-            const int mine = base + lane;
-            long long prow = row_of(c0);          // any valid row: padding entries get weight 0
-            float w = 0.f;
-            if (mine < count) { prow = row_of(c0 + mine); w = __expf(p.part_lse[prow] - mx); }
-            const int m = min(32, count - base);
-            // 16 partial rows in flight per lane, then their weighted sum, in CTA order
-            for (int j0 = 0; j0 < m; j0 += 16) {
-                float4 v[16];
-                float wj[16];
+    float sum = 0.f, mx = -INFINITY;
+    for (int base = 0; base < count; base += 16) {
+        const int mine = base + (lane & 15);
+        const bool have = mine < count;
+        const long long prow = row_of(c0 + (have ? mine : 0));
+        const float my_lse = have ? __ldcg(p.part_lse + prow) : -INFINITY;
+        float4 v[16];
 #pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    wj[j] = __shfl_sync(0xffffffffu, w, (j0 + j) & 31);
-                    const long long pj = __shfl_sync(0xffffffffu, prow, (j0 + j) & 31);
-                    v[j] = __ldcg(reinterpret_cast<const float4*>(p.part_o + pj * kHeadDim + lane * 4));
-                }
+        for (int j = 0; j < 16; ++j) {
+            const long long pj = __shfl_sync(0xffffffffu, prow, j);
+            v[j] = __ldcg(reinterpret_cast<const float4*>(p.part_o + pj * kHeadDim + lane * 4));
+        }
+        float gmx = my_lse;
 #pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    if (j0 + j < m) {
-                        acc.x += wj[j] * v[j].x; acc.y += wj[j] * v[j].y; acc.z += wj[j] * v[j].z; acc.w += wj[j] * v[j].w;
-                        sum += wj[j];
-                    }
-                }
+        for (int o = 8; o > 0; o >>= 1) gmx = fmaxf(gmx, __shfl_xor_sync(0xffffffffu, gmx, o));
+        const float mx_new = fmaxf(mx, gmx);
+        if (mx_new > -INFINITY) {
+            const float rescale = mx > -INFINITY ? __expf(mx - mx_new) : 0.f;
+            acc.x *= rescale; acc.y *= rescale; acc.z *= rescale; acc.w *= rescale;
+            sum *= rescale;
+            const float w = have ? __expf(my_lse - mx_new) : 0.f;     // -inf partial: weight 0
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+                const float wj = __shfl_sync(0xffffffffu, w, j);
+                acc.x += wj * v[j].x; acc.y += wj * v[j].y; acc.z += wj * v[j].z; acc.w += wj * v[j].w;
+                sum += wj;
             }
+            mx = mx_new;
         }
     }
     const float inv = sum > 0.f ? 1.f / sum : 0.f;

@@ -109,9 +109,14 @@ struct Partition {
     __device__ __host__ int owner(long long t) const {
         if (unit_tiles == 0) {
             long long big = (long long)rem * (q + 1);
+            if (total <= 0x7fffffffll) {      // the usual case: 32-bit divisions
+                const unsigned tt = (unsigned)t, qq = (unsigned)q, bb = (unsigned)big;
+                return tt < bb ? (int)(tt / (qq + 1u)) : rem + (int)((tt - bb) / qq);
+            }
             return t < big ? (int)(t / (q + 1)) : rem + (int)((t - big) / q);
         }
-        const int u = (int)(t / unit_tiles), local = (int)(t - (long long)u * unit_tiles);
+        const int u = total <= 0x7fffffffll ? (int)((unsigned)t / (unsigned)unit_tiles) : (int)(t / unit_tiles);
+        const int local = (int)(t - (long long)u * unit_tiles);
         const int cu = base + (u < urem ? 1 : 0), c0 = u * base + (u < urem ? u : urem);
         const int qq = unit_tiles / cu, rr = unit_tiles % cu, bigl = rr * (qq + 1);
         return c0 + (local < bigl ? local / (qq + 1) : rr + (local - bigl) / qq);
