@@ -46,6 +46,7 @@ constexpr int kRows = 256;                 // packed rows per unit (two streams 
 constexpr int kThreads = 384;
 constexpr int kSlots = 5;                  // ring of K / V tiles
 constexpr int kSlotBytes = kTileKeys * kHeadDim * 2;     // 32 KB
+constexpr int kTilesInFlight = 3;          // five slots never hold parts of more than three tiles
 constexpr int kQBytes = 128 * kHeadDim * 2;              // 32 KB per 128-row block
 constexpr int kRingOff = 2 * kQBytes;
 constexpr int kAuxOff = kRingOff + kSlots * kSlotBytes;  // 224 KB
@@ -55,7 +56,7 @@ constexpr uint32_t kTmemCols = 512;
 constexpr float kLazyRescale = 8.0f;       // log2 units
 
 struct Aux {
-    uint64_t full[kSlots];
+    uint64_t full[kTilesInFlight];   // one per tile: its K and its V slot complete the same barrier
     uint64_t empty[kSlots];
     uint64_t s_full[2], p_full[2], o_done[2];
     uint64_t q_full;
@@ -303,10 +304,11 @@ __device__ __forceinline__ void producer_loop(const AttnParams& p, const CUtenso
 #pragma unroll
             for (int kv = 0; kv < 2; ++kv) {
                 const uint32_t slot = item % kSlots, ph = (item / kSlots) & 1u;
-                const uint32_t full = smem_u32(&aux->full[slot]);
+                const uint32_t full = smem_u32(&aux->full[(item >> 1) % kTilesInFlight]);
                 const bool ok = mbar_wait(smem_u32(&aux->empty[slot]), ph ^ 1u, abort_flag);
                 if (ok) {
-                    if (lane == 0) mbar_arrive_expect_tx(full, (uint32_t)kSlotBytes);
+                    // the tile's barrier expects K and V together (announced with K; V follows as its slot frees up)
+                    if (lane == 0 && kv == 0) mbar_arrive_expect_tx(full, 2u * (uint32_t)kSlotBytes);
                     __syncwarp();
                     if (lane < ppt)
                         tma_load_5d_hint(ring + slot * kSlotBytes + lane * box_bytes, kv ? vmap : kmap, full, 0, 0, 0, 0, c_cur,
@@ -350,17 +352,19 @@ __device__ __forceinline__ void mma_loop(const AttnParams& p, Aux* aux, uint32_t
                 // (when both streams read every tile, stream 1 finds what stream 0 has just made sure of)
                 const bool seen = g.shared && s == 1;
                 if (do_pv) {
+                    // no check: V of this tile completed the same barrier as its K, seen before S = Q K^T was issued
                     const uint32_t item = item_base + 2u * (uint32_t)(g.tile(s, i) - g.tile0) + 1u;
                     v_slot = item % kSlots;
-                    if (!seen) ok = mbar_wait(smem_u32(&aux->full[v_slot]), (item / kSlots) & 1u, abort_flag) && ok;
                 }
-                uint32_t k_phase = 0;
+                uint32_t k_phase = 0, k_bar = 0;
                 bool k_ready = false;
                 if (do_qk) {
                     const uint32_t item = item_base + 2u * (uint32_t)(g.tile(s, i + 1) - g.tile0);
                     k_slot = item % kSlots;
-                    k_phase = (item / kSlots) & 1u;
-                    k_ready = seen || mbar_test_wait(smem_u32(&aux->full[k_slot]), k_phase);   // a look, no waiting yet
+                    const uint32_t tl = item >> 1;
+                    k_bar = smem_u32(&aux->full[tl % kTilesInFlight]);
+                    k_phase = (tl / kTilesInFlight) & 1u;
+                    k_ready = seen || mbar_test_wait(k_bar, k_phase);   // a look, no waiting yet
                 }
                 if (do_pv) {
                     // P of this stream: hardware barrier 4 + s, the warpgroup's 128 threads arrive, this warp waits
@@ -383,7 +387,7 @@ __device__ __forceinline__ void mma_loop(const AttnParams& p, Aux* aux, uint32_t
                     }
                 }
                 if (do_qk && !k_ready) {     // the next K tile may still be on its way (its slot was freed late)
-                    ok = mbar_wait(smem_u32(&aux->full[k_slot]), k_phase, abort_flag) && ok;
+                    ok = mbar_wait(k_bar, k_phase, abort_flag) && ok;
                     tc_fence_after();
                 }
                 if (lane == 0 && ok) {
@@ -713,7 +717,8 @@ verify_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap 
         return;
     }
     if (tid == 0) {
-        for (int i = 0; i < kSlots; ++i) { mbar_init(smem_u32(&aux->full[i]), 1); mbar_init(smem_u32(&aux->empty[i]), 1); }
+        for (int i = 0; i < kSlots; ++i) mbar_init(smem_u32(&aux->empty[i]), 1);
+        for (int i = 0; i < kTilesInFlight; ++i) mbar_init(smem_u32(&aux->full[i]), 1);
         for (int s = 0; s < 2; ++s) {
             mbar_init(smem_u32(&aux->s_full[s]), 1);
             mbar_init(smem_u32(&aux->p_full[s]), 128);
@@ -756,9 +761,10 @@ verify_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap 
     if (warp == 0) {
         if (aux->abort_flag) {
             // give the copies still in flight a bounded time to land before the CTA's shared memory is released
-            const uint32_t first = items > (uint32_t)kSlots ? items - kSlots : 0u;
-            for (uint32_t it = first; it < items; ++it) {
-                const uint32_t bar = smem_u32(&aux->full[it % kSlots]), ph = (it / kSlots) & 1u;
+            const uint32_t tiles_issued = (items + 1u) >> 1;
+            const uint32_t first = tiles_issued > (uint32_t)kTilesInFlight ? tiles_issued - kTilesInFlight : 0u;
+            for (uint32_t it = first; it < tiles_issued; ++it) {
+                const uint32_t bar = smem_u32(&aux->full[it % kTilesInFlight]), ph = (it / kTilesInFlight) & 1u;
                 for (int polls = 0; polls < (1 << 20) && !mbar_try_wait(bar, ph); ++polls) {}
             }
             if (lane == 0) report(p.status, kErrTimeout);
