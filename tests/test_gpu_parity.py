@@ -199,3 +199,32 @@ def test_unaligned_logits_rows():
     assert st == 0
     np.testing.assert_array_equal(am, r[3]); np.testing.assert_array_equal(alen, r[0])
     np.testing.assert_array_equal(path, r[1]); np.testing.assert_array_equal(bonus, r[2])
+
+
+# ----------------------------------------------------------------------------- other page sizes, fused step
+
+@pytest.mark.parametrize("page", [32, 64, 128])
+def test_other_page_sizes(page):
+    """One TMA box per (page, head): 8, 16 and 32 KB boxes instead of 4 KB; tails inside a page and a tile."""
+    wl = W.generate(W.Spec(f"page{page}", 16, 4, [777, 130, 1], [("tree", 33, 6), ("chain", 8), ("tree", 64, 8)],
+                           shuffle_pages=True, page_size=page, seed=300 + page, with_logits=False))
+    check_attention(wl)
+
+
+def test_verify_step_equals_the_two_calls():
+    """owl_verify_step (acceptance beside the attention pass) gives bit for bit what the two calls give."""
+    wl = W.generate(W.Spec("step", 32, 8, [1500, 40], [("tree", 32, 6), ("chain", 8)], shuffle_pages=True, seed=411, vocab=20000))
+    dw = DeviceWorkload.upload(wl)
+    ctx = OwlContext(dims_of(wl))
+    dw.attn(ctx)
+    dw.accept(ctx)
+    assert ctx.owl_get_status() == 0
+    want = [t.clone() for t in (dw.out, dw.lse, dw.accept_len, dw.accept_path, dw.bonus_token, dw.node_argmax)]
+    for _ in range(3):
+        for t in (dw.out, dw.lse, dw.accept_len, dw.accept_path, dw.bonus_token, dw.node_argmax):
+            t.zero_()
+        dw.step(ctx)
+        assert ctx.owl_get_status() == 0
+        for got, ref in zip((dw.out, dw.lse, dw.accept_len, dw.accept_path, dw.bonus_token, dw.node_argmax), want):
+            assert torch.equal(got, ref)
+    ctx.close()
