@@ -329,7 +329,6 @@ __device__ __forceinline__ void mma_loop(const AttnParams& p, Aux* aux, uint32_t
     constexpr uint32_t idesc_qk = umma_idesc_bf16(128, kTileKeys, 0, 0);
     constexpr uint32_t idesc_pv = umma_idesc_bf16(128, kHeadDim, 0, 1);
     const uint32_t ring = smem_base + kRingOff;
-    uint32_t it[2] = {0, 0};
     uint32_t seg_no = 0, item_base = 0;
     Segment g;
 
@@ -338,74 +337,73 @@ __device__ __forceinline__ void mma_loop(const AttnParams& p, Aux* aux, uint32_t
         tc_fence_after();
         const int n_it[2] = {g.iters(0), g.iters(1)};
 
+        // Ring slot and arrival barrier of the tile each stream needs next, kept as running counters (the issue
+        // loop is a chain of dependent scalar instructions: no divisions or remainders in it).
+        const uint32_t step_items = g.shared ? 2u : 4u, step_tiles = g.shared ? 1u : 2u;
+        uint32_t k_slot[2], v_slot[2], tb_idx[2], tb_ph[2];
+#pragma unroll
+        for (int s = 0; s < 2; ++s) {
+            const uint32_t first = item_base + (g.shared ? 0u : 2u * (uint32_t)s);
+            k_slot[s] = first % kSlots;
+            v_slot[s] = (first + 1u) % kSlots;
+            tb_idx[s] = (first >> 1) % kTilesInFlight;
+            tb_ph[s] = ((first >> 1) / kTilesInFlight) & 1u;
+        }
         // i = -1 issues the first S = Q K^T of both streams; afterwards, per stream: O += P V of tile i, then
         // S = Q K^T of tile i + 1 (which overwrites the P just consumed; the tensor pipe runs them in order)
 #pragma unroll 1
         for (int i = -1; i < n_it[0]; ++i) {
-#pragma unroll 1
+#pragma unroll
             for (int s = 0; s < 2; ++s) {
                 const bool last_reader = !g.shared || s == 1;
                 const bool do_pv = i >= 0 && i < n_it[s], do_qk = i + 1 < n_it[s];
-                uint32_t v_slot = 0, k_slot = 0;
-                // the K / V tiles were requested long ago: make sure of them first, so that nothing stands between
-                // the arrival of P and the issue of both products
                 // (when both streams read every tile, stream 1 finds what stream 0 has just made sure of)
                 const bool seen = g.shared && s == 1;
-                if (do_pv) {
-                    // no check: V of this tile completed the same barrier as its K, seen before S = Q K^T was issued
-                    const uint32_t item = item_base + 2u * (uint32_t)(g.tile(s, i) - g.tile0) + 1u;
-                    v_slot = item % kSlots;
-                }
-                uint32_t k_phase = 0, k_bar = 0;
+                const uint32_t k_bar = smem_u32(&aux->full[tb_idx[s]]);
                 bool k_ready = false;
-                if (do_qk) {
-                    const uint32_t item = item_base + 2u * (uint32_t)(g.tile(s, i + 1) - g.tile0);
-                    k_slot = item % kSlots;
-                    const uint32_t tl = item >> 1;
-                    k_bar = smem_u32(&aux->full[tl % kTilesInFlight]);
-                    k_phase = (tl / kTilesInFlight) & 1u;
-                    k_ready = seen || mbar_test_wait(k_bar, k_phase);   // a look, no waiting yet
-                }
+                if (do_qk) k_ready = seen || mbar_test_wait(k_bar, tb_ph[s]);   // a look, no waiting yet
                 if (do_pv) {
                     // P of this stream: hardware barrier 4 + s, the warpgroup's 128 threads arrive, this warp waits
                     // (every arrival is executed whatever happens, so the wait always ends)
                     asm volatile("bar.sync %0, 160;" ::"r"(4 + s) : "memory");
-                    ++it[s];
                 }
                 tc_fence_after();
-                if (lane == 0 && ok) {
-                    if (do_pv) {
-                        // one descriptor per batch; the k-steps only move its start-address field (units of 16 bytes)
-                        const uint64_t vdesc = umma_smem_desc_sw128(ring + v_slot * kSlotBytes, 1024, 2048);
-                        const uint32_t tO = tmem + 256 + s * 128, tP = tmem + s * 128;
-                        const uint32_t v_lo = (uint32_t)vdesc, v_hi = (uint32_t)(vdesc >> 32);
+                if (lane == 0 && ok && do_pv) {
+                    // V needs no check: it completed the same barrier as the tile's K, seen before S = Q K^T was issued.
+                    // One descriptor per batch; the k-steps only move its start-address word (units of 16 bytes).
+                    const uint64_t vdesc = umma_smem_desc_sw128(ring + v_slot[s] * kSlotBytes, 1024, 2048);
+                    const uint32_t tO = tmem + 256 + s * 128, tP = tmem + s * 128;
+                    const uint32_t v_lo = (uint32_t)vdesc, v_hi = (uint32_t)(vdesc >> 32);
 #pragma unroll
-                        for (int ks = 0; ks < 8; ++ks)
-                            umma_ts_lh(tO, tP + ks * 8, v_lo + (uint32_t)(ks * 4096 >> 4), v_hi, idesc_pv, (i | ks) ? 1u : 0u);
-                        if (i == n_it[s] - 1) umma_commit(smem_u32(&aux->o_done[s]));   // only the segment end waits for it
-                        if (last_reader) umma_commit(smem_u32(&aux->empty[v_slot]));
-                    }
+                    for (int ks = 0; ks < 8; ++ks)
+                        umma_ts_lh(tO, tP + ks * 8, v_lo + (uint32_t)(ks * 4096 >> 4), v_hi, idesc_pv, (i | ks) ? 1u : 0u);
+                    if (i == n_it[s] - 1) umma_commit(smem_u32(&aux->o_done[s]));   // only the segment end waits for it
+                    if (last_reader) umma_commit(smem_u32(&aux->empty[v_slot[s]]));
                 }
+                if (do_pv) { v_slot[s] += step_items; if (v_slot[s] >= (uint32_t)kSlots) v_slot[s] -= kSlots; }
                 if (do_qk && !k_ready) {     // the next K tile may still be on its way (its slot was freed late)
-                    ok = mbar_wait(k_bar, k_phase, abort_flag) && ok;
+                    ok = mbar_wait(k_bar, tb_ph[s], abort_flag) && ok;
                     tc_fence_after();
                 }
-                if (lane == 0 && ok) {
-                    if (do_qk) {
-                        const uint64_t qdesc = umma_smem_desc_sw128(smem_base + (g.shared ? s : 0) * kQBytes, 16, 1024);
-                        const uint64_t kdesc = umma_smem_desc_sw128(ring + k_slot * kSlotBytes, 16, 2048);
-                        const uint32_t tS = tmem + s * 128;
-                        const uint32_t q_lo = (uint32_t)qdesc, q_hi = (uint32_t)(qdesc >> 32);
-                        const uint32_t k_lo = (uint32_t)kdesc, k_hi = (uint32_t)(kdesc >> 32);
+                if (lane == 0 && ok && do_qk) {
+                    const uint64_t qdesc = umma_smem_desc_sw128(smem_base + (g.shared ? s : 0) * kQBytes, 16, 1024);
+                    const uint64_t kdesc = umma_smem_desc_sw128(ring + k_slot[s] * kSlotBytes, 16, 2048);
+                    const uint32_t tS = tmem + s * 128;
+                    const uint32_t q_lo = (uint32_t)qdesc, q_hi = (uint32_t)(qdesc >> 32);
+                    const uint32_t k_lo = (uint32_t)kdesc, k_hi = (uint32_t)(kdesc >> 32);
 #pragma unroll
-                        for (int hf = 0; hf < 2; ++hf)
+                    for (int hf = 0; hf < 2; ++hf)
 #pragma unroll
-                            for (int ks = 0; ks < 4; ++ks)
-                                umma_ss_lh(tS, q_lo + (uint32_t)((hf * 16384 + ks * 32) >> 4), q_hi,
-                                           k_lo + (uint32_t)((hf * 1024 + ks * 32) >> 4), k_hi, idesc_qk, (hf | ks) ? 1u : 0u);
-                        umma_commit(smem_u32(&aux->s_full[s]));
-                        if (last_reader) umma_commit(smem_u32(&aux->empty[k_slot]));
-                    }
+                        for (int ks = 0; ks < 4; ++ks)
+                            umma_ss_lh(tS, q_lo + (uint32_t)((hf * 16384 + ks * 32) >> 4), q_hi,
+                                       k_lo + (uint32_t)((hf * 1024 + ks * 32) >> 4), k_hi, idesc_qk, (hf | ks) ? 1u : 0u);
+                    umma_commit(smem_u32(&aux->s_full[s]));
+                    if (last_reader) umma_commit(smem_u32(&aux->empty[k_slot[s]]));
+                }
+                if (do_qk) {
+                    k_slot[s] += step_items; if (k_slot[s] >= (uint32_t)kSlots) k_slot[s] -= kSlots;
+                    tb_idx[s] += step_tiles;
+                    if (tb_idx[s] >= (uint32_t)kTilesInFlight) { tb_idx[s] -= kTilesInFlight; tb_ph[s] ^= 1u; }
                 }
                 __syncwarp();
             }
