@@ -123,3 +123,17 @@ def test_bad_page_is_reported_and_isolated():
     out = dw.out_f32()
     assert np.all(out[:8] == 7.0) and np.abs(out[8:] - ref_out[8:]).max() <= 1e-2
     ctx.close()
+
+
+def test_scale_and_head_limits():
+    wl = _wl()
+    dw = DeviceWorkload.upload(wl)
+    ctx = OwlContext(dims_of(wl))
+    n0 = ctx.launch_count()
+    for bad_scale in (0.0, -0.5, float("nan"), float("inf")):
+        bad = dims_of(wl); bad.sm_scale = bad_scale
+        assert DeviceWorkload.attn(dataclass_replace(dw, dims=bad), ctx, check=False) == -1
+    bad = dims_of(wl); bad.num_q_heads = 512; bad.num_kv_heads = 256
+    assert DeviceWorkload.attn(dataclass_replace(dw, dims=bad), ctx, check=False) == -2
+    assert ctx.launch_count() == n0
+    ctx.close()

@@ -228,3 +228,27 @@ def test_verify_step_equals_the_two_calls():
         for got, ref in zip((dw.out, dw.lse, dw.accept_len, dw.accept_path, dw.bonus_token, dw.node_argmax), want):
             assert torch.equal(got, ref)
     ctx.close()
+
+
+# ----------------------------------------------------------------------------- partition and schedule corners
+
+@pytest.mark.parametrize("ctx_len,trees", [
+    (3000, [("tree", 32, 6)] * 4),     # uniform batch, 8 units over 148 CTAs: unit-aligned cut, pieces of 1-2 tiles
+    (300, [("tree", 32, 6)] * 4),      # fewer tiles per unit than CTAs per unit: most CTAs get nothing
+    (5000, [("tree", 64, 8)] * 2),     # uniform, M = 256 (both streams read every tile), aligned cut
+    (129, [("chain", 2)] * 3),         # two tiles per unit, second one holds a single key
+])
+def test_uniform_batches_take_the_aligned_cut(ctx_len, trees):
+    wl = W.generate(W.Spec("aligned", 8, 2, [ctx_len] * len(trees), trees, shuffle_pages=True, seed=500 + ctx_len,
+                           with_logits=False))
+    check_attention(wl)
+
+
+def test_large_batch_mixed_row_counts():
+    """More than 32 sequences (block-wide schedule) with M = 256, M = 128 and tiny units next to one another."""
+    rng = np.random.default_rng(6)
+    kinds = [("tree", 64, 8), ("tree", 32, 6), ("chain", 3), ("tree", 17, 4)]
+    trees = [kinds[int(rng.integers(0, 4))] for _ in range(40)]
+    ctx = [int(x) for x in rng.integers(0, 700, size=40)]
+    wl = W.generate(W.Spec("mixed40", 16, 4, ctx, trees, shuffle_pages=True, seed=601, with_logits=False))
+    check_attention(wl)
