@@ -323,92 +323,123 @@ __device__ __forceinline__ void producer_loop(const AttnParams& p, const CUtenso
 }
 
 // ------------------------------------------------------------------------------------------ MMA issuer
+// One thread's time is what bounds a 256-row unit: each tcgen05.mma costs the issuing thread about 60 clocks, and
+// whatever it executes between two batches (waits, slot arithmetic, commits) is added to that, not hidden behind it.
+// So the loop is kept lean:
+//  * the warp stays converged from top to bottom; all 32 lanes run the loop and the tensor-core instructions carry
+//    the guard (`elected` lane, waits succeeded, work to do) themselves.  What steers the loop (the segment's tile
+//    range and mode, the verdicts of the waits) goes through a warp reduction or a vote first, so that trip counts,
+//    ring slots and descriptors are uniform by construction;
+//  * per stream and tile it waits on two hardware barriers (about 25 clocks each when the arrival is already in; a
+//    look at an mbarrier costs 70 to 130): on one the softmax warpgroup announces P, on the other that it has seen
+//    the stream's next key tile arrive;
+//  * the iterations in which both streams have both products to issue run in a loop of their own without
+//    per-product conditions; the first and the last ones of a segment take the general form.
 __device__ __forceinline__ void mma_loop(const AttnParams& p, Aux* aux, uint32_t smem_base, uint32_t tmem, Walker w) {
-    const int lane = threadIdx.x & 31;
+    constexpr unsigned kAll = 0xffffffffu;
     volatile int* abort_flag = &aux->abort_flag;
     constexpr uint32_t idesc_qk = umma_idesc_bf16(128, kTileKeys, 0, 0);
     constexpr uint32_t idesc_pv = umma_idesc_bf16(128, kHeadDim, 0, 1);
     const uint32_t ring = smem_base + kRingOff;
+    const uint32_t elected = elect_one() ? 1u : 0u;
+    // descriptors of Q block 0 and of ring slot 0; those of the other blocks and slots differ in the start-address
+    // field only (units of 16 bytes; shared memory ends below 2^18, so the field never carries)
+    const uint64_t q_desc0 = umma_smem_desc_sw128(smem_base, 16, 1024);
+    const uint64_t k_desc0 = umma_smem_desc_sw128(ring, 16, 2048), v_desc0 = umma_smem_desc_sw128(ring, 1024, 2048);
     uint32_t seg_no = 0, item_base = 0;
     Segment g;
 
-    while (w.next(p, g)) {
-        bool ok = mbar_wait(smem_u32(&aux->q_full), seg_no & 1u, abort_flag);
-        tc_fence_after();
-        const int n_it[2] = {g.iters(0), g.iters(1)};
+    for (;;) {
+        const bool more = w.next(p, g);
+        if (!__any_sync(kAll, more)) break;
+        const int tile0 = __reduce_max_sync(kAll, g.tile0), tile1 = __reduce_max_sync(kAll, g.tile1);
+        const bool shared = __reduce_max_sync(kAll, g.shared ? 1 : 0) != 0;
+        bool ok = __all_sync(kAll, mbar_wait(smem_u32(&aux->q_full), seg_no & 1u, abort_flag));
+        const int T = tile1 - tile0;
+        const int n_it[2] = {shared ? T : (T + 1) >> 1, shared ? T : T >> 1};
 
-        // Ring slot and arrival barrier of the tile each stream needs next, kept as running counters (the issue
-        // loop is a chain of dependent scalar instructions: no divisions or remainders in it).
-        const uint32_t step_items = g.shared ? 2u : 4u, step_tiles = g.shared ? 1u : 2u;
-        uint32_t k_slot[2], v_slot[2], tb_idx[2], tb_ph[2];
+        // ring slots of the K tile and of the V tile each stream needs next, as running counters
+        const uint32_t step_items = shared ? 2u : 4u;
+        uint32_t k_slot[2], v_slot[2];
 #pragma unroll
         for (int s = 0; s < 2; ++s) {
-            const uint32_t first = item_base + (g.shared ? 0u : 2u * (uint32_t)s);
+            const uint32_t first = item_base + (shared ? 0u : 2u * (uint32_t)s);
             k_slot[s] = first % kSlots;
             v_slot[s] = (first + 1u) % kSlots;
-            tb_idx[s] = (first >> 1) % kTilesInFlight;
-            tb_ph[s] = ((first >> 1) / kTilesInFlight) & 1u;
         }
-        // i = -1 issues the first S = Q K^T of both streams; afterwards, per stream: O += P V of tile i, then
-        // S = Q K^T of tile i + 1 (which overwrites the P just consumed; the tensor pipe runs them in order)
-#pragma unroll 1
-        for (int i = -1; i < n_it[0]; ++i) {
+        auto advance = [&](uint32_t& slot) { slot += step_items; if (slot >= (uint32_t)kSlots) slot -= kSlots; };
+        // O_s (+)= P_s V: A from tensor memory, B = the V tile as it lies in the ring (MN-major)
+        auto issue_pv = [&](int s, uint32_t issue, uint32_t acc0) {
+            const uint64_t vdesc = v_desc0 + (uint64_t)(v_slot[s] * (uint32_t)(kSlotBytes >> 4));
+            const uint32_t tO = tmem + 256 + s * 128, tP = tmem + s * 128;
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks)
+                umma_ts_if(issue, tO, tP + ks * 8, vdesc + (uint64_t)(ks * 4096 >> 4), idesc_pv, ks ? 1u : acc0);
+        };
+        // S_s = Q K^T: both operands K-major in shared memory
+        auto issue_qk = [&](int s, uint32_t issue) {
+            const uint64_t qdesc = q_desc0 + (uint64_t)((shared && s) ? (kQBytes >> 4) : 0);
+            const uint64_t kdesc = k_desc0 + (uint64_t)(k_slot[s] * (uint32_t)(kSlotBytes >> 4));
+#pragma unroll
+            for (int hf = 0; hf < 2; ++hf)
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks)
+                    umma_ss_if(issue, tmem + s * 128, qdesc + (uint64_t)((hf * 16384 + ks * 32) >> 4),
+                               kdesc + (uint64_t)((hf * 1024 + ks * 32) >> 4), idesc_qk, (hf | ks) ? 1u : 0u);
+        };
+        // General form of one iteration: O += P V of tile i, then S = Q K^T of tile i + 1 (which overwrites the P just
+        // consumed; the tensor pipe runs them in order), each where the stream has such a tile.  i = -1 issues the
+        // first S of both streams, after this warp's own look at the arrival barrier of their first tiles.
+        auto general = [&](int i) {
 #pragma unroll
             for (int s = 0; s < 2; ++s) {
-                const bool last_reader = !g.shared || s == 1;
+                const bool last_reader = !shared || s == 1;
                 const bool do_pv = i >= 0 && i < n_it[s], do_qk = i + 1 < n_it[s];
-                // (when both streams read every tile, stream 1 finds what stream 0 has just made sure of)
-                const bool seen = g.shared && s == 1;
-                const uint32_t k_bar = smem_u32(&aux->full[tb_idx[s]]);
-                bool k_ready = false;
-                if (do_qk) k_ready = seen || mbar_test_wait(k_bar, tb_ph[s]);   // a look, no waiting yet
-                if (do_pv) {
-                    // P of this stream: hardware barrier 4 + s, the warpgroup's 128 threads arrive, this warp waits
-                    // (every arrival is executed whatever happens, so the wait always ends)
-                    asm volatile("bar.sync %0, 160;" ::"r"(4 + s) : "memory");
+                if (do_pv) asm volatile("bar.sync %0, 160;" ::"r"(4 + s) : "memory");
+                if (i < 0 && do_qk && !(shared && s == 1)) {
+                    const uint32_t seq = (item_base >> 1) + (uint32_t)s;
+                    ok = __all_sync(kAll, mbar_wait(smem_u32(&aux->full[seq % kTilesInFlight]),
+                                                    (seq / kTilesInFlight) & 1u, abort_flag)) && ok;
                 }
                 tc_fence_after();
-                if (lane == 0 && ok && do_pv) {
-                    // V needs no check: it completed the same barrier as the tile's K, seen before S = Q K^T was issued.
-                    // One descriptor per batch; the k-steps only move its start-address word (units of 16 bytes).
-                    const uint64_t vdesc = umma_smem_desc_sw128(ring + v_slot[s] * kSlotBytes, 1024, 2048);
-                    const uint32_t tO = tmem + 256 + s * 128, tP = tmem + s * 128;
-                    const uint32_t v_lo = (uint32_t)vdesc, v_hi = (uint32_t)(vdesc >> 32);
+                uint32_t issue = (ok && do_pv) ? elected : 0u;
+                issue_pv(s, issue, i > 0 ? 1u : 0u);
+                umma_commit_if(i == n_it[s] - 1 ? issue : 0u, smem_u32(&aux->o_done[s]));   // only the segment end waits for it
+                umma_commit_if(last_reader ? issue : 0u, smem_u32(&aux->empty[v_slot[s]]));
+                if (do_pv) advance(v_slot[s]);
+                if (i >= 0 && do_qk) { asm volatile("bar.sync %0, 64;" ::"r"(6 + s) : "memory"); tc_fence_after(); }
+                issue = (ok && do_qk) ? elected : 0u;
+                issue_qk(s, issue);
+                umma_commit_if(issue, smem_u32(&aux->s_full[s]));
+                umma_commit_if(last_reader ? issue : 0u, smem_u32(&aux->empty[k_slot[s]]));
+                if (do_qk) advance(k_slot[s]);
+            }
+        };
+        general(-1);
+        int i = 0;
+        {
+            const uint32_t issue = ok ? elected : 0u;
+#pragma unroll 1
+            for (; i < n_it[1] - 1; ++i) {
 #pragma unroll
-                    for (int ks = 0; ks < 8; ++ks)
-                        umma_ts_lh(tO, tP + ks * 8, v_lo + (uint32_t)(ks * 4096 >> 4), v_hi, idesc_pv, (i | ks) ? 1u : 0u);
-                    if (i == n_it[s] - 1) umma_commit(smem_u32(&aux->o_done[s]));   // only the segment end waits for it
-                    if (last_reader) umma_commit(smem_u32(&aux->empty[v_slot[s]]));
-                }
-                if (do_pv) { v_slot[s] += step_items; if (v_slot[s] >= (uint32_t)kSlots) v_slot[s] -= kSlots; }
-                if (do_qk && !k_ready) {     // the next K tile may still be on its way (its slot was freed late)
-                    ok = mbar_wait(k_bar, tb_ph[s], abort_flag) && ok;
+                for (int s = 0; s < 2; ++s) {
+                    const uint32_t issue_last = (shared && s == 0) ? 0u : issue;
+                    asm volatile("bar.sync %0, 160;" ::"r"(4 + s) : "memory");
                     tc_fence_after();
+                    issue_pv(s, issue, i > 0 ? 1u : 0u);
+                    umma_commit_if(issue_last, smem_u32(&aux->empty[v_slot[s]]));
+                    advance(v_slot[s]);
+                    asm volatile("bar.sync %0, 64;" ::"r"(6 + s) : "memory");   // the next K tile has landed
+                    issue_qk(s, issue);
+                    umma_commit_if(issue, smem_u32(&aux->s_full[s]));
+                    umma_commit_if(issue_last, smem_u32(&aux->empty[k_slot[s]]));
+                    advance(k_slot[s]);
                 }
-                if (lane == 0 && ok && do_qk) {
-                    const uint64_t qdesc = umma_smem_desc_sw128(smem_base + (g.shared ? s : 0) * kQBytes, 16, 1024);
-                    const uint64_t kdesc = umma_smem_desc_sw128(ring + k_slot[s] * kSlotBytes, 16, 2048);
-                    const uint32_t tS = tmem + s * 128;
-                    const uint32_t q_lo = (uint32_t)qdesc, q_hi = (uint32_t)(qdesc >> 32);
-                    const uint32_t k_lo = (uint32_t)kdesc, k_hi = (uint32_t)(kdesc >> 32);
-#pragma unroll
-                    for (int hf = 0; hf < 2; ++hf)
-#pragma unroll
-                        for (int ks = 0; ks < 4; ++ks)
-                            umma_ss_lh(tS, q_lo + (uint32_t)((hf * 16384 + ks * 32) >> 4), q_hi,
-                                       k_lo + (uint32_t)((hf * 1024 + ks * 32) >> 4), k_hi, idesc_qk, (hf | ks) ? 1u : 0u);
-                    umma_commit(smem_u32(&aux->s_full[s]));
-                    if (last_reader) umma_commit(smem_u32(&aux->empty[k_slot[s]]));
-                }
-                if (do_qk) {
-                    k_slot[s] += step_items; if (k_slot[s] >= (uint32_t)kSlots) k_slot[s] -= kSlots;
-                    tb_idx[s] += step_tiles;
-                    if (tb_idx[s] >= (uint32_t)kTilesInFlight) { tb_idx[s] -= kTilesInFlight; tb_ph[s] ^= 1u; }
-                }
-                __syncwarp();
             }
         }
-        item_base += 2u * (uint32_t)(g.tile1 - g.tile0);
+#pragma unroll 1
+        for (; i < n_it[0]; ++i) general(i);
+        item_base += 2u * (uint32_t)T;
         ++seg_no;
     }
 }
@@ -419,6 +450,36 @@ __device__ __forceinline__ void named_barrier(int id, int count) {
 }
 
 __device__ __forceinline__ float max3(float a, float b, float c) { return fmaxf(fmaxf(a, b), c); }
+
+// 2^x for a pair of arguments on the FMA pipe instead of the special-function unit, whose 16 results per clock
+// per SM bound the softmax of a 256-row unit (256 x 128 exponentials per key tile take as long as its MMAs).
+// Range reduction by the rounding of a large constant: t = x + 1.5 * 2^23 holds n = round(x) in its low mantissa
+// bits, f = x - n lies in [-1/2, 1/2], 2^f is a cubic fitted to a relative error of 7.5e-5 (the weights are
+// rounded to bf16, 2e-3, afterwards), and n goes into the exponent field by an integer add.  Arguments below
+// -125 are clamped: the result is then about 2^-125, zero for every purpose here.
+#ifndef OWL_POLY_PERIOD
+#define OWL_POLY_PERIOD 0
+#endif
+constexpr int kPolyPeriod = OWL_POLY_PERIOD;   // every kPolyPeriod-th pair of a row takes this path; 0: none
+__device__ __forceinline__ void exp2_poly_x2(uint64_t xx, float& p0, float& p1) {
+    float x0, x1;
+    unpack_f32x2(xx, x0, x1);
+    x0 = fmaxf(x0, -125.f);
+    x1 = fmaxf(x1, -125.f);
+    const uint64_t x = pack_f32x2(x0, x1);
+    const uint64_t magic = pack_f32x2(12582912.f, 12582912.f), neg_magic = pack_f32x2(-12582912.f, -12582912.f);
+    const uint64_t t = add_f32x2(x, magic);
+    const uint64_t n = add_f32x2(t, neg_magic);
+    const uint64_t f = fma_f32x2(n, pack_f32x2(-1.f, -1.f), x);
+    uint64_t r = fma_f32x2(f, pack_f32x2(0.0551716685f, 0.0551716685f), pack_f32x2(0.242611125f, 0.242611125f));
+    r = fma_f32x2(r, f, pack_f32x2(0.693260968f, 0.693260968f));
+    r = fma_f32x2(r, f, pack_f32x2(0.999928057f, 0.999928057f));
+    float t0, t1, r0, r1;
+    unpack_f32x2(t, t0, t1);
+    unpack_f32x2(r, r0, r1);
+    p0 = __uint_as_float(__float_as_uint(r0) + (__float_as_uint(t0) << 23));
+    p1 = __uint_as_float(__float_as_uint(r1) + (__float_as_uint(t1) << 23));
+}
 
 // Writes a warp's 32 rows x 32 columns (lane = row, v = its 32 fp32 values) to global memory through a
 // per-warp staging area in shared memory, so that every store instruction covers whole 64- or 128-byte
@@ -472,6 +533,7 @@ __device__ __forceinline__ void softmax_loop(const AttnParams& p, Aux* aux, unsi
     const float scale2 = p.sm_scale * 1.4426950408889634f;   // > 0 (checked on the host)
     const int G = p.group;
     uint32_t it = 0, seg_no = 0, od_phase = 0;   // od_phase: segments of this stream that issued a product
+    uint32_t tile_base = 0;                      // key tiles of the CTA's earlier segments (the ring counts them through)
     Segment g;
 
     while (w.next(p, g)) {
@@ -569,10 +631,15 @@ __device__ __forceinline__ void softmax_loop(const AttnParams& p, Aux* aux, unsi
                 tmem_ld64(tS + 64, reinterpret_cast<uint32_t(&)[64]>(raw[64]));
                 tmem_wait_ld();
             }
-            float mx = max3(sv[0], sv[1], sv[2]);
+            // four independent chains: a single one would be 64 dependent instructions long
+            float mx4[4];
 #pragma unroll
-            for (int c = 3; c + 1 < 128; c += 2) mx = max3(mx, sv[c], sv[c + 1]);
-            mx = fmaxf(mx, sv[127]);
+            for (int q = 0; q < 4; ++q) mx4[q] = max3(sv[32 * q], sv[32 * q + 1], sv[32 * q + 2]);
+#pragma unroll
+            for (int c = 3; c + 1 < 32; c += 2)
+#pragma unroll
+                for (int q = 0; q < 4; ++q) mx4[q] = max3(mx4[q], sv[32 * q + c], sv[32 * q + c + 1]);
+            const float mx = fmaxf(fmaxf(max3(mx4[0], sv[31], sv[63]), max3(mx4[1], sv[95], sv[127])), fmaxf(mx4[2], mx4[3]));
             const float m_new = fmaxf(m, mx * scale2);
             const bool need = (m_new - m) > kLazyRescale;      // false when both are -inf (NaN compares false)
             if (__any_sync(0xffffffffu, need)) {
@@ -609,8 +676,10 @@ __device__ __forceinline__ void softmax_loop(const AttnParams& p, Aux* aux, unsi
 #pragma unroll
                 for (int j = 0; j < 32; ++j) {
                     float x0, x1;
-                    unpack_f32x2(fma_f32x2(pack_f32x2(sv[hf * 64 + 2 * j], sv[hf * 64 + 2 * j + 1]), scale2_x2, neg_m_x2), x0, x1);
-                    const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
+                    const uint64_t xx = fma_f32x2(pack_f32x2(sv[hf * 64 + 2 * j], sv[hf * 64 + 2 * j + 1]), scale2_x2, neg_m_x2);
+                    float p0, p1;
+                    if (kPolyPeriod > 0 && j % (kPolyPeriod > 0 ? kPolyPeriod : 1) == 0) exp2_poly_x2(xx, p0, p1);
+                    else { unpack_f32x2(xx, x0, x1); p0 = fast_exp2(x0); p1 = fast_exp2(x1); }
                     __nv_bfloat162 b2 = __floats2bfloat162_rn(p0, p1);
                     const uint32_t u = *reinterpret_cast<uint32_t*>(&b2);
                     pk[j] = u;
@@ -631,6 +700,15 @@ __device__ __forceinline__ void softmax_loop(const AttnParams& p, Aux* aux, unsi
             tmem_wait_st();
             tc_fence_before();
             asm volatile("bar.arrive %0, 160;" ::"r"(4 + s) : "memory");
+            // The MMA warp polls no mbarrier between O += P V of this tile and S = Q K^T of the stream's next one: the
+            // first warp of the warpgroup looks at that tile's arrival barrier for it (after P is announced, so that
+            // nothing this tile holds is released any later) and passes the news on through hardware barrier 6 + s.
+            // A wait that gives up raises the abort flag; the arrival happens all the same.
+            if (wtid < 32 && i + 1 < n_it) {
+                const uint32_t seq = tile_base + (uint32_t)(g.shared ? i + 1 : 2 * (i + 1) + s);
+                mbar_wait(smem_u32(&aux->full[seq % kTilesInFlight]), (seq / kTilesInFlight) & 1u, abort_flag);
+                asm volatile("bar.arrive %0, 64;" ::"r"(6 + s) : "memory");
+            }
             ++it;
         }
 
@@ -697,6 +775,7 @@ __device__ __forceinline__ void softmax_loop(const AttnParams& p, Aux* aux, unsi
             else p.part_lse[part_row] = lse;
         }
         tc_fence_before();
+        tile_base += (uint32_t)(g.tile1 - g.tile0);
         ++seg_no;
     }
 }
