@@ -415,30 +415,25 @@ __device__ __forceinline__ void mma_loop(const AttnParams& p, Aux* aux, uint32_t
                 if (do_qk) advance(k_slot[s]);
             }
         };
-        general(-1);
-        int i = 0;
-        {
-            const uint32_t issue = ok ? elected : 0u;
 #pragma unroll 1
-            for (; i < n_it[1] - 1; ++i) {
+        for (int i = -1; i < n_it[0]; ++i) {
+            if (i < 0 || i >= n_it[1] - 1) { general(i); continue; }
+            const uint32_t issue = ok ? elected : 0u;
 #pragma unroll
-                for (int s = 0; s < 2; ++s) {
-                    const uint32_t issue_last = (shared && s == 0) ? 0u : issue;
-                    asm volatile("bar.sync %0, 160;" ::"r"(4 + s) : "memory");
-                    tc_fence_after();
-                    issue_pv(s, issue, i > 0 ? 1u : 0u);
-                    umma_commit_if(issue_last, smem_u32(&aux->empty[v_slot[s]]));
-                    advance(v_slot[s]);
-                    asm volatile("bar.sync %0, 64;" ::"r"(6 + s) : "memory");   // the next K tile has landed
-                    issue_qk(s, issue);
-                    umma_commit_if(issue, smem_u32(&aux->s_full[s]));
-                    umma_commit_if(issue_last, smem_u32(&aux->empty[k_slot[s]]));
-                    advance(k_slot[s]);
-                }
+            for (int s = 0; s < 2; ++s) {
+                const uint32_t issue_last = (shared && s == 0) ? 0u : issue;
+                asm volatile("bar.sync %0, 160;" ::"r"(4 + s) : "memory");
+                tc_fence_after();
+                issue_pv(s, issue, i > 0 ? 1u : 0u);
+                umma_commit_if(issue_last, smem_u32(&aux->empty[v_slot[s]]));
+                advance(v_slot[s]);
+                asm volatile("bar.sync %0, 64;" ::"r"(6 + s) : "memory");   // the next K tile has landed
+                issue_qk(s, issue);
+                umma_commit_if(issue, smem_u32(&aux->s_full[s]));
+                umma_commit_if(issue_last, smem_u32(&aux->empty[k_slot[s]]));
+                advance(k_slot[s]);
             }
         }
-#pragma unroll 1
-        for (; i < n_it[0]; ++i) general(i);
         item_base += 2u * (uint32_t)T;
         ++seg_no;
     }
@@ -450,36 +445,6 @@ __device__ __forceinline__ void named_barrier(int id, int count) {
 }
 
 __device__ __forceinline__ float max3(float a, float b, float c) { return fmaxf(fmaxf(a, b), c); }
-
-// 2^x for a pair of arguments on the FMA pipe instead of the special-function unit, whose 16 results per clock
-// per SM bound the softmax of a 256-row unit (256 x 128 exponentials per key tile take as long as its MMAs).
-// Range reduction by the rounding of a large constant: t = x + 1.5 * 2^23 holds n = round(x) in its low mantissa
-// bits, f = x - n lies in [-1/2, 1/2], 2^f is a cubic fitted to a relative error of 7.5e-5 (the weights are
-// rounded to bf16, 2e-3, afterwards), and n goes into the exponent field by an integer add.  Arguments below
-// -125 are clamped: the result is then about 2^-125, zero for every purpose here.
-#ifndef OWL_POLY_PERIOD
-#define OWL_POLY_PERIOD 0
-#endif
-constexpr int kPolyPeriod = OWL_POLY_PERIOD;   // every kPolyPeriod-th pair of a row takes this path; 0: none
-__device__ __forceinline__ void exp2_poly_x2(uint64_t xx, float& p0, float& p1) {
-    float x0, x1;
-    unpack_f32x2(xx, x0, x1);
-    x0 = fmaxf(x0, -125.f);
-    x1 = fmaxf(x1, -125.f);
-    const uint64_t x = pack_f32x2(x0, x1);
-    const uint64_t magic = pack_f32x2(12582912.f, 12582912.f), neg_magic = pack_f32x2(-12582912.f, -12582912.f);
-    const uint64_t t = add_f32x2(x, magic);
-    const uint64_t n = add_f32x2(t, neg_magic);
-    const uint64_t f = fma_f32x2(n, pack_f32x2(-1.f, -1.f), x);
-    uint64_t r = fma_f32x2(f, pack_f32x2(0.0551716685f, 0.0551716685f), pack_f32x2(0.242611125f, 0.242611125f));
-    r = fma_f32x2(r, f, pack_f32x2(0.693260968f, 0.693260968f));
-    r = fma_f32x2(r, f, pack_f32x2(0.999928057f, 0.999928057f));
-    float t0, t1, r0, r1;
-    unpack_f32x2(t, t0, t1);
-    unpack_f32x2(r, r0, r1);
-    p0 = __uint_as_float(__float_as_uint(r0) + (__float_as_uint(t0) << 23));
-    p1 = __uint_as_float(__float_as_uint(r1) + (__float_as_uint(t1) << 23));
-}
 
 // Writes a warp's 32 rows x 32 columns (lane = row, v = its 32 fp32 values) to global memory through a
 // per-warp staging area in shared memory, so that every store instruction covers whole 64- or 128-byte
@@ -677,9 +642,8 @@ __device__ __forceinline__ void softmax_loop(const AttnParams& p, Aux* aux, unsi
                 for (int j = 0; j < 32; ++j) {
                     float x0, x1;
                     const uint64_t xx = fma_f32x2(pack_f32x2(sv[hf * 64 + 2 * j], sv[hf * 64 + 2 * j + 1]), scale2_x2, neg_m_x2);
-                    float p0, p1;
-                    if (kPolyPeriod > 0 && j % (kPolyPeriod > 0 ? kPolyPeriod : 1) == 0) exp2_poly_x2(xx, p0, p1);
-                    else { unpack_f32x2(xx, x0, x1); p0 = fast_exp2(x0); p1 = fast_exp2(x1); }
+                    unpack_f32x2(xx, x0, x1);
+                    const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
                     __nv_bfloat162 b2 = __floats2bfloat162_rn(p0, p1);
                     const uint32_t u = *reinterpret_cast<uint32_t*>(&b2);
                     pk[j] = u;
