@@ -330,9 +330,9 @@ __device__ __forceinline__ void producer_loop(const AttnParams& p, const CUtenso
 //    the guard (`elected` lane, waits succeeded, work to do) themselves.  What steers the loop (the segment's tile
 //    range and mode, the verdicts of the waits) goes through a warp reduction or a vote first, so that trip counts,
 //    ring slots and descriptors are uniform by construction;
-//  * per stream and tile it waits on two hardware barriers (about 25 clocks each when the arrival is already in; a
-//    look at an mbarrier costs 70 to 130): on one the softmax warpgroup announces P, on the other that it has seen
-//    the stream's next key tile arrive;
+//  * per stream and tile of such a unit it waits on two hardware barriers (about 25 clocks each when the arrival is
+//    already in; a look at an mbarrier costs 70 to 130): on one the softmax warpgroup announces P, on the other
+//    that it has seen the stream's next key tile arrive (units of up to 128 rows wait for the tile itself);
 //  * the iterations in which both streams have both products to issue run in a loop of their own without
 //    per-product conditions; the first and the last ones of a segment take the general form.
 __device__ __forceinline__ void mma_loop(const AttnParams& p, Aux* aux, uint32_t smem_base, uint32_t tmem, Walker w) {
@@ -387,6 +387,40 @@ __device__ __forceinline__ void mma_loop(const AttnParams& p, Aux* aux, uint32_t
                     umma_ss_if(issue, tmem + s * 128, qdesc + (uint64_t)((hf * 16384 + ks * 32) >> 4),
                                kdesc + (uint64_t)((hf * 1024 + ks * 32) >> 4), idesc_qk, (hf | ks) ? 1u : 0u);
         };
+        // Before S = Q K^T of the stream's tile i + 1.  M > 128: the issue loop is what bounds the unit, and the
+        // softmax warpgroup, which has time to spare, looks at the tile's arrival barrier and passes the news on
+        // through hardware barrier 6 + s (about 25 clocks here).  M <= 128: the tile itself is what the warp
+        // usually waits for, and it waits on the arrival barrier directly, one wake-up instead of two.
+        auto wait_next_k = [&](int s, int i) {
+            if (shared) {
+                asm volatile("bar.sync %0, 64;" ::"r"(6 + s) : "memory");
+            } else {
+                const uint32_t seq = (item_base >> 1) + (uint32_t)(2 * (i + 1) + s);
+                ok = __all_sync(kAll, mbar_wait(smem_u32(&aux->full[seq % kTilesInFlight]), (seq / kTilesInFlight) & 1u,
+                                                abort_flag)) && ok;
+            }
+        };
+        // The same two products with the k-steps in a loop, for the few iterations of the general form below (they
+        // are too rare to be worth the code size of another thirty-two unrolled instructions)
+        auto issue_pv_rolled = [&](int s, uint32_t issue, uint32_t acc0) {
+            uint64_t vdesc = v_desc0 + (uint64_t)(v_slot[s] * (uint32_t)(kSlotBytes >> 4));
+            const uint32_t tO = tmem + 256 + s * 128;
+            uint32_t tP = tmem + s * 128;
+#pragma unroll 1
+            for (int ks = 0; ks < 8; ++ks, vdesc += 4096 >> 4, tP += 8)
+                umma_ts_if(issue, tO, tP, vdesc, idesc_pv, ks ? 1u : acc0);
+        };
+        auto issue_qk_rolled = [&](int s, uint32_t issue) {
+            uint64_t qdesc = q_desc0 + (uint64_t)((shared && s) ? (kQBytes >> 4) : 0);
+            uint64_t kdesc = k_desc0 + (uint64_t)(k_slot[s] * (uint32_t)(kSlotBytes >> 4));
+#pragma unroll 1
+            for (int j = 0; j < 8; ++j) {
+                umma_ss_if(issue, tmem + s * 128, qdesc, kdesc, idesc_qk, j ? 1u : 0u);
+                // four k-steps of 32 bytes inside a 128-byte swizzle row, then the other half of the head dimension
+                qdesc += j == 3 ? (uint64_t)((16384 - 96) >> 4) : 2u;
+                kdesc += j == 3 ? (uint64_t)((1024 - 96) >> 4) : 2u;
+            }
+        };
         // General form of one iteration: O += P V of tile i, then S = Q K^T of tile i + 1 (which overwrites the P just
         // consumed; the tensor pipe runs them in order), each where the stream has such a tile.  i = -1 issues the
         // first S of both streams, after this warp's own look at the arrival barrier of their first tiles.
@@ -403,13 +437,13 @@ __device__ __forceinline__ void mma_loop(const AttnParams& p, Aux* aux, uint32_t
                 }
                 tc_fence_after();
                 uint32_t issue = (ok && do_pv) ? elected : 0u;
-                issue_pv(s, issue, i > 0 ? 1u : 0u);
+                issue_pv_rolled(s, issue, i > 0 ? 1u : 0u);
                 umma_commit_if(i == n_it[s] - 1 ? issue : 0u, smem_u32(&aux->o_done[s]));   // only the segment end waits for it
                 umma_commit_if(last_reader ? issue : 0u, smem_u32(&aux->empty[v_slot[s]]));
                 if (do_pv) advance(v_slot[s]);
-                if (i >= 0 && do_qk) { asm volatile("bar.sync %0, 64;" ::"r"(6 + s) : "memory"); tc_fence_after(); }
+                if (i >= 0 && do_qk) { wait_next_k(s, i); tc_fence_after(); }
                 issue = (ok && do_qk) ? elected : 0u;
-                issue_qk(s, issue);
+                issue_qk_rolled(s, issue);
                 umma_commit_if(issue, smem_u32(&aux->s_full[s]));
                 umma_commit_if(last_reader ? issue : 0u, smem_u32(&aux->empty[k_slot[s]]));
                 if (do_qk) advance(k_slot[s]);
@@ -427,8 +461,8 @@ __device__ __forceinline__ void mma_loop(const AttnParams& p, Aux* aux, uint32_t
                 issue_pv(s, issue, i > 0 ? 1u : 0u);
                 umma_commit_if(issue_last, smem_u32(&aux->empty[v_slot[s]]));
                 advance(v_slot[s]);
-                asm volatile("bar.sync %0, 64;" ::"r"(6 + s) : "memory");   // the next K tile has landed
-                issue_qk(s, issue);
+                wait_next_k(s, i);                                          // the next K tile has landed
+                issue_qk(s, ok ? issue : 0u);
                 umma_commit_if(issue, smem_u32(&aux->s_full[s]));
                 umma_commit_if(issue_last, smem_u32(&aux->empty[k_slot[s]]));
                 advance(k_slot[s]);
@@ -664,12 +698,13 @@ __device__ __forceinline__ void softmax_loop(const AttnParams& p, Aux* aux, unsi
             tmem_wait_st();
             tc_fence_before();
             asm volatile("bar.arrive %0, 160;" ::"r"(4 + s) : "memory");
-            // The MMA warp polls no mbarrier between O += P V of this tile and S = Q K^T of the stream's next one: the
-            // first warp of the warpgroup looks at that tile's arrival barrier for it (after P is announced, so that
-            // nothing this tile holds is released any later) and passes the news on through hardware barrier 6 + s.
-            // A wait that gives up raises the abort flag; the arrival happens all the same.
-            if (wtid < 32 && i + 1 < n_it) {
-                const uint32_t seq = tile_base + (uint32_t)(g.shared ? i + 1 : 2 * (i + 1) + s);
+            // In a unit of more than 128 rows the MMA warp polls no mbarrier between O += P V of this tile and
+            // S = Q K^T of the next one: the first warp of the warpgroup looks at that tile's arrival barrier for it
+            // (after P is announced, so that nothing this tile holds is released any later) and passes the news on
+            // through hardware barrier 6 + s.  A wait that gives up raises the abort flag; the arrival happens all
+            // the same.
+            if (g.shared && wtid < 32 && i + 1 < n_it) {
+                const uint32_t seq = tile_base + (uint32_t)(i + 1);
                 mbar_wait(smem_u32(&aux->full[seq % kTilesInFlight]), (seq / kTilesInFlight) & 1u, abort_flag);
                 asm volatile("bar.arrive %0, 64;" ::"r"(6 + s) : "memory");
             }
