@@ -205,7 +205,13 @@ int owl_create(owl_ctx** out, int device, const owl_dims* max_dims) {
     if (ok && attn) {
         ok = cudaFuncSetAttribute(mma_path::verify_attn_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                   mma_path::kSmemBytes) == cudaSuccess &&
-             cudaFuncSetAttribute(umma_path::verify_attn_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+             cudaFuncSetAttribute(umma_path::verify_attn_umma_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  umma_path::kSmemBytes) == cudaSuccess &&
+             cudaFuncSetAttribute(umma_path::verify_attn_umma_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  umma_path::kSmemBytes) == cudaSuccess &&
+             cudaFuncSetAttribute(umma_path::verify_attn_umma_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  umma_path::kSmemBytes) == cudaSuccess &&
+             cudaFuncSetAttribute(umma_path::verify_attn_umma_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                   umma_path::kSmemBytes) == cudaSuccess;
     }
     if (!ok || cudaDeviceSynchronize() != cudaSuccess) {
@@ -316,7 +322,12 @@ int owl_verify_attn(owl_ctx* ctx, const owl_dims* d, const void* q, const void* 
             attr[0].val.programmaticStreamSerializationAllowed = 1;
             cfg.attrs = attr;
             cfg.numAttrs = 1;
-            cudaLaunchKernelEx(&cfg, umma_path::verify_attn_umma_kernel, p, ctx->kmap, ctx->vmap);
+            // the instance that holds only this call's case: block-wide schedule above 32 sequences, the two-row-block
+            // mode only if a unit (G * max_nodes rows at most) can exceed 128 rows
+            const bool many = d->batch > 32, wide = G * d->max_nodes > 128;
+            auto kernel = many ? (wide ? umma_path::verify_attn_umma_kernel<true, true> : umma_path::verify_attn_umma_kernel<true, false>)
+                               : (wide ? umma_path::verify_attn_umma_kernel<false, true> : umma_path::verify_attn_umma_kernel<false, false>);
+            cudaLaunchKernelEx(&cfg, kernel, p, ctx->kmap, ctx->vmap);
         }
         ++ctx->launches;
         if (ctx->profiling) cudaEventRecord(ctx->ev[1], stream);

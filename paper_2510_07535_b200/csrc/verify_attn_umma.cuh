@@ -103,6 +103,9 @@ struct Walker {
         cur_node_base = seq_node_base(p, b);
         cur_b = b;
     }
+    // kWide = false: the caller knows that no unit has more than 128 rows (G * max_nodes <= 128, and sequences with
+    // more nodes than max_nodes are rejected), so `shared` is a constant and the code of that mode is not generated.
+    template <bool kWide>
     __device__ __forceinline__ bool next(const AttnParams& p, Segment& g) {
         if (t >= t_end) return false;
         while (b < p.batch) {
@@ -124,7 +127,7 @@ struct Walker {
         g.unit = unit_begin + g.h;
         g.node_base = cur_node_base;
         g.M = cur_n * p.group;
-        g.shared = g.M > 128;
+        g.shared = kWide && g.M > 128;
         t += g.tile1 - g.tile0;
         return true;
     }
@@ -272,6 +275,7 @@ __device__ __forceinline__ void build_walk_small(const AttnParams& p, Walker& w)
 }
 
 // ------------------------------------------------------------------------------------------ producer
+template <bool kWide>
 __device__ __forceinline__ void producer_loop(const AttnParams& p, const CUtensorMap* kmap, const CUtensorMap* vmap,
                                               Aux* aux, uint32_t ring, Walker w, uint32_t& items_out) {
     const int lane = threadIdx.x & 31;
@@ -283,7 +287,7 @@ __device__ __forceinline__ void producer_loop(const AttnParams& p, const CUtenso
     // K/V are read once: let them leave L2 first, so that Q, the partials, the tables and the code stay
     const uint64_t stream_policy = l2_policy_evict_first();
     Segment g;
-    while (w.next(p, g)) {
+    while (w.template next<kWide>(p, g)) {
         const int keys = g.L + g.n;
         const int pages_valid = (keys + p.page_size - 1) >> p.page_shift;
         const int32_t* table = p.block_table + (long long)g.b * p.max_pages_per_seq;
@@ -335,6 +339,7 @@ __device__ __forceinline__ void producer_loop(const AttnParams& p, const CUtenso
 //    that it has seen the stream's next key tile arrive (units of up to 128 rows wait for the tile itself);
 //  * the iterations in which both streams have both products to issue run in a loop of their own without
 //    per-product conditions; the first and the last ones of a segment take the general form.
+template <bool kWide>
 __device__ __forceinline__ void mma_loop(const AttnParams& p, Aux* aux, uint32_t smem_base, uint32_t tmem, Walker w) {
     constexpr unsigned kAll = 0xffffffffu;
     volatile int* abort_flag = &aux->abort_flag;
@@ -350,10 +355,10 @@ __device__ __forceinline__ void mma_loop(const AttnParams& p, Aux* aux, uint32_t
     Segment g;
 
     for (;;) {
-        const bool more = w.next(p, g);
+        const bool more = w.template next<kWide>(p, g);
         if (!__any_sync(kAll, more)) break;
         const int tile0 = __reduce_max_sync(kAll, g.tile0), tile1 = __reduce_max_sync(kAll, g.tile1);
-        const bool shared = __reduce_max_sync(kAll, g.shared ? 1 : 0) != 0;
+        const bool shared = kWide && __reduce_max_sync(kAll, g.shared ? 1 : 0) != 0;
         bool ok = __all_sync(kAll, mbar_wait(smem_u32(&aux->q_full), seg_no & 1u, abort_flag));
         const int T = tile1 - tile0;
         const int n_it[2] = {shared ? T : (T + 1) >> 1, shared ? T : T >> 1};
@@ -522,6 +527,7 @@ __device__ __forceinline__ void store_rows32(const AttnParams& p, float* stage, 
     }
 }
 
+template <bool kWide>
 __device__ __forceinline__ void softmax_loop(const AttnParams& p, Aux* aux, unsigned char* smem, uint32_t tmem, Walker w,
                                              const int s /*stream*/) {
     const int wtid = threadIdx.x - 128 - s * 128;          // 0..127 inside the warpgroup
@@ -535,7 +541,7 @@ __device__ __forceinline__ void softmax_loop(const AttnParams& p, Aux* aux, unsi
     uint32_t tile_base = 0;                      // key tiles of the CTA's earlier segments (the ring counts them through)
     Segment g;
 
-    while (w.next(p, g)) {
+    while (w.template next<kWide>(p, g)) {
         // ---- Q rows (16-byte asynchronous copies, rows beyond M zero-filled) and, in stream 0's warpgroup, the
         // ancestor masks; every global read of the segment start is in flight at the same time
         int parent_i = -1;
@@ -780,6 +786,10 @@ __device__ __forceinline__ void softmax_loop(const AttnParams& p, Aux* aux, unsi
 }
 
 // ------------------------------------------------------------------------------------------ kernel
+// kManySeqs: more than 32 sequences (the block-wide schedule); kWide: some unit may have more than 128 rows.  Four
+// instances, so that a launch carries only the code of its own case: the text of the paths a launch never takes
+// still costs it time (3 us of 39 on a 32K-context, 32-node step when the block-wide schedule was compiled in).
+template <bool kManySeqs, bool kWide>
 __global__ void __launch_bounds__(kThreads, 1)
 verify_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap vmap) {
     extern __shared__ __align__(1024) unsigned char smem[];
@@ -813,23 +823,23 @@ verify_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap 
     // before this one in the stream has completed (a no-op in an ordinary launch)
     asm volatile("griddepcontrol.wait;" ::: "memory");
     Walker w;
-    if (p.batch <= 32) build_walk_small(p, w);     // its global loads overlap the set-up above
+    if (!kManySeqs) build_walk_small(p, w);        // its global loads overlap the set-up above
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = aux->tmem_base;
-    if (p.batch > 32) build_walk(p, aux, w);
+    if (kManySeqs) build_walk(p, aux, w);
 
     // registers move from the warpgroup of the producer / MMA warps to the two softmax warpgroups,
     // whose threads each hold a 128-column row of S: 128 x 72 + 256 x 216 = 384 x 168, the registers the CTA was launched with
     uint32_t items = 0;
     if (warp < 4) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
-        if (warp == 0) producer_loop(p, &kmap, &vmap, aux, smem_base + kRingOff, w, items);
-        else if (warp == 1) mma_loop(p, aux, smem_base, tmem, w);
+        if (warp == 0) producer_loop<kWide>(p, &kmap, &vmap, aux, smem_base + kRingOff, w, items);
+        else if (warp == 1) mma_loop<kWide>(p, aux, smem_base, tmem, w);
     } else {
         asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
-        softmax_loop(p, aux, smem, tmem, w, warp >= 8 ? 1 : 0);
+        softmax_loop<kWide>(p, aux, smem, tmem, w, warp >= 8 ? 1 : 0);
     }
 
     tc_fence_before();
