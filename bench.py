@@ -306,7 +306,11 @@ def run_gpu(args, rank, world, local_rank):
 
     if rank == 0:
         peak, peak_kind = measured_peaks()
-        achieved = attn_b / kt[0] / 1e9 if kt[0] > 0 else None
+        # a step with a small acceptance scan has no arg-max kernel: the attention kernel's spare warps read the logits,
+        # so those bytes belong to that launch
+        fused = kt[2] == 0 and logit_b > 0
+        attn_launch_b = attn_b + (logit_b if fused else 0)
+        achieved = attn_launch_b / kt[0] / 1e9 if kt[0] > 0 else None
         line = {
             "metric": METRIC, "value": world * step_bytes / step_s / 1e9, "unit": "GB/s", "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": step_s * 1e3, "higher_is_better": True,
@@ -319,7 +323,8 @@ def run_gpu(args, rank, world, local_rank):
             "frac_of_hbm_peak": step_bytes / step_s / 1e9 / peak,
             "kernel_us": {"verify_attn": kt[0] * 1e6, "combine": kt[1] * 1e6, "argmax_accept": kt[2] * 1e6},
             "bytes_per_step": {"attention": attn_b, "logits": logit_b},
-            "roofline": {"bound": "hbm", "kernel": "verify_attn", "achieved": achieved, "peak": peak, "unit": "GB/s",
+            "roofline": {"bound": "hbm", "kernel": "verify_attn" + (" (+ logits scan)" if fused else ""),
+                         "bytes_per_launch": attn_launch_b, "achieved": achieved, "peak": peak, "unit": "GB/s",
                          "frac": achieved / peak if achieved else None, "peak_kind": f"of {peak_kind}",
                          "traffic": ncu_traffic(spec.name)},
             "accept_gbs": logit_b / kt[2] / 1e9 if kt[2] > 0 else None,

@@ -143,11 +143,12 @@ int owl_tree_accept(owl_ctx* ctx, const owl_dims* dims, const float* logits,
 /*
  * One whole verify step on device buffers: owl_verify_attn and owl_tree_accept of the same batch
  * (Section 3.2.2 "Decode Stage" followed by the acceptance of the Introduction), arguments as in those
- * two calls.  The two halves do not depend on each other (the logits are an input), so a small acceptance
- * scan (about one wave of CTAs or less) is queued on a stream of the context's own and runs beside the
- * tail of the attention pass; the call forks from `stream` and joins it again, i.e. for the caller
- * everything happens in stream order.  Larger scans follow the attention pass on `stream`.
- * Asynchronous; errors as in the two calls.
+ * two calls, results bit for bit those of the two calls.  The two halves do not depend on each other (the
+ * logits are an input), so a small acceptance (total_nodes * ceil(vocab / 8192) <= 1024) costs no launch
+ * of its own: spare warps of the attention kernel scan the logits while K/V stream in, and the kernel
+ * that merges the attention partials also walks the trees.  Larger scans follow the attention pass as a
+ * kernel of their own.  Everything runs on `stream`, in stream order.  Asynchronous; errors as in the
+ * two calls (argument errors of either half are reported before anything is launched).
  */
 int owl_verify_step(owl_ctx* ctx, const owl_dims* dims, const void* q, const void* k_cache, const void* v_cache,
                     const int32_t* block_table, const int32_t* ctx_lens, const int32_t* node_offsets,

@@ -13,6 +13,10 @@
 // (draft token == parent's arg-max), picks the deepest matching node (lowest index among equals) and
 // writes accept_len / accept_path / bonus_token.  Calls alternate between two sets of counters and clear the
 // idle one, so no separate clearing pass is needed.
+//
+// Inside a verify step with a small scan both halves run as guests of the attention kernels: the scan in warps
+// the attention pass does not use (argmax_scan_chunk_warp), the walk in extra CTAs of the merge kernel, after
+// the pass has completed; no counters are involved there.
 #pragma once
 
 #include "owl_common.cuh"
@@ -101,6 +105,65 @@ __device__ __forceinline__ void accept_walk_seq(const AcceptParams& p, const int
         int k = len - 1;
         for (int c = win; c >= 0 && k >= 0; c = s_parent[c]) path[k--] = c;
     }
+}
+
+// The same scan of one (row, vocabulary chunk) by a single warp, for callers that have warps to spare inside
+// another kernel (the verify step's attention pass scans the logits with its two idle warps while it streams K/V).
+// Stores the same key argmax_partial_kernel would: the maximum over (value, ~index) does not depend on how the
+// chunk's elements are dealt out to threads.
+__device__ __forceinline__ void argmax_scan_chunk_warp(const AcceptParams& p, const int row, const int chunk) {
+    const int lane = threadIdx.x & 31;
+    const long long V = p.vocab;
+    const long long c0 = (long long)chunk * kArgmaxChunk;
+    const long long c1 = c0 + kArgmaxChunk < V ? c0 + kArgmaxChunk : V;
+    const float* base = p.logits + row * V;
+    // [c0, a0) scalar head up to 16-byte alignment, [a0, a1) float4 body, [a1, c1) scalar tail
+    const uintptr_t addr = reinterpret_cast<uintptr_t>(base + c0);
+    long long a0 = c0 + (long long)(((16 - (addr & 15)) & 15) >> 2);
+    if (a0 > c1) a0 = c1;
+    const long long a1 = a0 + ((c1 - a0) & ~3ll);
+
+    float bv = -INFINITY;
+    uint32_t bi = 0xffffffffu;   // "no candidate yet"
+    const float4* body = reinterpret_cast<const float4*>(base + a0);
+    const int nvec = (int)((a1 - a0) >> 2);
+    for (int v0 = 0; v0 < nvec; v0 += 32 * 8) {
+        float4 x[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {            // eight independent 16-byte loads per lane in flight
+            const int v = v0 + j * 32 + lane;
+            x[j] = v < nvec ? __ldg(body + v) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int v = v0 + j * 32 + lane;
+            if (v < nvec) {
+                const uint32_t i0 = (uint32_t)(a0 + 4ll * v);
+                // NaN reads as -inf; strict '>' keeps the first maximum (indices grow along this lane's walk)
+                const float e0 = x[j].x != x[j].x ? -INFINITY : x[j].x, e1 = x[j].y != x[j].y ? -INFINITY : x[j].y;
+                const float e2 = x[j].z != x[j].z ? -INFINITY : x[j].z, e3 = x[j].w != x[j].w ? -INFINITY : x[j].w;
+                if (bi == 0xffffffffu || e0 > bv) { bv = e0; bi = i0; }
+                if (e1 > bv) { bv = e1; bi = i0 + 1; }
+                if (e2 > bv) { bv = e2; bi = i0 + 2; }
+                if (e3 > bv) { bv = e3; bi = i0 + 3; }
+            }
+        }
+    }
+    unsigned long long key = bi != 0xffffffffu ? argmax_key(bv, bi) : 0ull;
+    if (lane < 8) {              // ragged ends: at most 3 + 3 elements per chunk
+        const long long j = lane < 4 ? c0 + lane : a1 + (lane - 4);
+        const long long lim = lane < 4 ? a0 : c1;
+        if (j < lim) {
+            const unsigned long long k2 = argmax_key(base[j], (uint32_t)j);
+            key = k2 > key ? k2 : key;
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const unsigned long long other = __shfl_xor_sync(0xffffffffu, key, o);
+        key = other > key ? other : key;
+    }
+    if (lane == 0) p.part_keys[(long long)row * p.chunks + chunk] = key;
 }
 
 __global__ void __launch_bounds__(kArgmaxThreads) argmax_partial_kernel(const AcceptParams p) {

@@ -4,6 +4,7 @@
 #pragma once
 
 #include "owl_common.cuh"
+#include "accept.cuh"
 
 namespace owl {
 
@@ -73,45 +74,88 @@ __global__ void __launch_bounds__(kCombineWarps * 32) combine_kernel(const AttnP
 }
 
 
-// LSE merge for the tcgen05 split-KV pass.  That pass leaves its schedule in global memory (first flat
-// tile of every sequence, totals, choice of partition), so this kernel rebuilds nothing: one warp per
-// output row finds the CTAs whose pieces cut the row's unit and merges their partials in CTA order.
-// A CTA stores at most two partials: slot 2c if its piece starts inside the unit, else 2c + 1.
-__global__ void __launch_bounds__(kCombineWarps * 32) combine_sched_kernel(const AttnParams p) {
-    // launched as a programmatic dependent of the split-KV pass: wait here until that grid has completed and
-    // its writes are visible (a no-op in an ordinary launch), then let the next kernel in the stream queue up
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+// LSE merge for the tcgen05 split-KV pass: one warp per output row finds the CTAs whose pieces cut the row's unit
+// and merges their partials in CTA order.  A CTA stores at most two partials: slot 2c if its piece starts inside
+// the unit, else 2c + 1.
+//
+// The kernel is launched as a programmatic dependent of that pass and its time after the pass has ended is pure
+// latency, so everything that needs no output of the pass comes before the wait: for batches of at most 32
+// sequences the warp derives the schedule from the inputs exactly as the pass did (warp_schedule) and knows its
+// row's partial slots when the wait returns; what is left is one round of loads.  Larger batches read the
+// schedule the pass left in global memory (first flat tile of every sequence, totals, choice of partition).
+//
+// kFused (verify step): the grid has one more CTA per sequence after the row CTAs; each of those runs one
+// sequence's acceptance walk over the arg-max keys that the pass's spare warps left (`ap`).
+template <bool kFused>
+__global__ void __launch_bounds__(kCombineWarps * 32) combine_sched_kernel(const AttnParams p, const AcceptParams ap) {
+    if (kFused) {
+        const long long rows = (long long)p.total_nodes * p.num_q_heads;
+        const unsigned row_ctas = (unsigned)((rows + kCombineWarps - 1) / kCombineWarps);
+        if (blockIdx.x >= row_ctas) {
+            static_assert(kCombineWarps * 32 >= kMaxNodes, "the walk needs one thread per node");
+            asm volatile("griddepcontrol.wait;" ::: "memory");
+            asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+            accept_walk_seq(ap, (int)(blockIdx.x - row_ctas));
+            return;
+        }
+    }
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const long long row_id = (long long)blockIdx.x * kCombineWarps + warp;
-    if (row_id >= (long long)p.total_nodes * p.num_q_heads) return;
-    const int n = (int)(row_id / p.num_q_heads), hq = (int)(row_id % p.num_q_heads);
-    int b;
-    if (p.node_offsets) {
-        int lo = 0, hi = p.batch;  // largest b with node_offsets[b] <= n
-        while (hi - lo > 1) { int mid = (lo + hi) >> 1; if (p.node_offsets[mid] <= n) lo = mid; else hi = mid; }
-        b = lo;
-    } else {
-        b = n / p.nodes_uniform;
-    }
-    // independent loads first, tests afterwards: one round trip instead of four
-    const int bad_epoch = p.seq_bad[b];
-    const long long seq_begin = p.sched_seq_begin[b], seq_end = p.sched_seq_begin[b + 1];
-    const SchedHeader hdr = *p.sched_header;
-    const int node_base = seq_node_base(p, b);
-    if (bad_epoch == p.epoch) return;
-    const int tiles = (int)((seq_end - seq_begin) / p.num_kv_heads);
-    if (tiles == 0) return;
+    const bool row_valid = row_id < (long long)p.total_nodes * p.num_q_heads;
+    const int n = row_valid ? (int)(row_id / p.num_q_heads) : 0, hq = row_valid ? (int)(row_id % p.num_q_heads) : 0;
+    const bool small = p.batch <= 32;
+    int b = 0, node_base = 0, tiles = 0;
+    long long seq_begin = 0;
     Partition part;
-    part.init(hdr.total_tiles, p.num_ctas, hdr.units, hdr.uniform_tiles);
-    const int G = p.group;
-    const int lrow = (n - node_base) * G + hq % G;
-    const long long t0 = seq_begin + (long long)(hq / G) * tiles;
-    const int c0 = part.owner(t0), c1 = part.owner(t0 + tiles - 1);
+    if (small) {
+        const WarpSchedule ws = warp_schedule(p);
+        const unsigned hit = __ballot_sync(0xffffffffu, lane < p.batch && ws.tiles > 0 && n >= ws.node_base && n < ws.node_base + ws.n);
+        b = hit ? __ffs(hit) - 1 : 0;
+        node_base = __shfl_sync(0xffffffffu, ws.node_base, b);
+        tiles = hit ? __shfl_sync(0xffffffffu, ws.tiles, b) : 0;
+        seq_begin = __shfl_sync(0xffffffffu, ws.excl_t, b);
+        part.init(ws.total, p.num_ctas, ws.units, ws.uniform_tiles);
+    }
+    // the CTAs c0..c1 whose pieces cut the row's unit, and the slot row of the partial this lane fetches first
+    int lrow = 0, c0 = 0, c1 = 0;
+    long long t0 = 0, prow_first = 0;
+    auto row_of = [&](int c) -> long long { return (2ll * c + (part.begin(c) < t0 ? 1 : 0)) * p.rows_per_slot + lrow; };
+    auto plan = [&]() {
+        if (tiles == 0) return;
+        const int G = p.group;
+        lrow = (n - node_base) * G + hq % G;
+        t0 = seq_begin + (long long)(hq / G) * tiles;
+        c0 = part.owner(t0);
+        c1 = part.owner(t0 + tiles - 1);
+        prow_first = row_of(c0 + min(lane & 15, c1 - c0));
+    };
+    if (small) plan();
+    // from here on the split-KV pass has completed and its writes are visible (a no-op in an ordinary launch)
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next kernel in the stream may queue up
+    if (!row_valid) return;
+    if (!small) {
+        int lo = 0, hi = p.batch;  // largest b with node_offsets[b] <= n
+        if (p.node_offsets) {
+            while (hi - lo > 1) { int mid = (lo + hi) >> 1; if (p.node_offsets[mid] <= n) lo = mid; else hi = mid; }
+            b = lo;
+        } else {
+            b = n / p.nodes_uniform;
+        }
+        // independent loads first, tests afterwards: one round trip instead of four
+        const long long sb = p.sched_seq_begin[b], se = p.sched_seq_begin[b + 1];
+        const SchedHeader hdr = *p.sched_header;
+        node_base = seq_node_base(p, b);
+        seq_begin = sb;
+        tiles = (int)((se - sb) / p.num_kv_heads);
+        part.init(hdr.total_tiles, p.num_ctas, hdr.units, hdr.uniform_tiles);
+        plan();
+    }
+    if (tiles == 0) return;
     if (c0 == c1) return;  // a single CTA saw every key of this unit and wrote the result itself
+    const int bad_epoch = __ldcg(p.seq_bad + b);   // (its round trip overlaps the partial loads below)
     const int count = c1 - c0 + 1;
 
-    auto row_of = [&](int c) -> long long { return (2ll * c + (part.begin(c) < t0 ? 1 : 0)) * p.rows_per_slot + lrow; };
     // Partials are taken 16 at a time: lane j (< 16) of a group owns partial base + j.  The row loads do not
     // depend on the LSE values, so both go out together: one memory round trip per group, and units cut into
     // at most 16 pieces - the usual case - need a single group.  Groups are folded online (running maximum).
@@ -120,7 +164,7 @@ __global__ void __launch_bounds__(kCombineWarps * 32) combine_sched_kernel(const
     for (int base = 0; base < count; base += 16) {
         const int mine = base + (lane & 15);
         const bool have = mine < count;
-        const long long prow = row_of(c0 + (have ? mine : 0));
+        const long long prow = base == 0 ? prow_first : row_of(c0 + (have ? mine : 0));
         const float my_lse = have ? __ldcg(p.part_lse + prow) : -INFINITY;
         float4 v[16];
 #pragma unroll
@@ -146,6 +190,7 @@ __global__ void __launch_bounds__(kCombineWarps * 32) combine_sched_kernel(const
             mx = mx_new;
         }
     }
+    if (bad_epoch == p.epoch) return;              // the pass found a bad tree or page in this sequence: no output
     const float inv = sum > 0.f ? 1.f / sum : 0.f;
     __nv_bfloat162 lo2 = __floats2bfloat162_rn(acc.x * inv, acc.y * inv);
     __nv_bfloat162 hi2 = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);

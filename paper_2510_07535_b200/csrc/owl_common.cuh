@@ -148,6 +148,51 @@ __device__ __forceinline__ bool seq_shape_ok(const AttnParams& p, int b, int n, 
     return keys <= (long long)p.max_pages_per_seq * p.page_size;
 }
 
+// Schedule of a batch of at most 32 sequences, derived by one warp on its own: lane b holds sequence b, prefix sums
+// by shuffle, no shared memory.  The split-KV pass (every warp of it) and the merge that follows it call the same
+// function on the same inputs, so the merge needs nothing from the pass but its partials.
+constexpr int kSchedTileKeys = 128;      // key tile of the tcgen05 split-KV pass
+struct WarpSchedule {
+    int n, L, node_base, tiles;          // this lane's sequence (tiles = 0 if it is not schedulable)
+    bool ok;
+    long long my_tiles, excl_t, total;   // flat tiles of this sequence (all KV heads), of the ones before it, of all
+    int my_units, excl_u, units;
+    int uniform_tiles;                   // tiles per unit if every schedulable sequence has the same count, else 0
+};
+__device__ __forceinline__ WarpSchedule warp_schedule(const AttnParams& p) {
+    const int lane = threadIdx.x & 31;
+    WarpSchedule ws;
+    ws.n = 0; ws.L = 0; ws.node_base = 0; ws.tiles = 0; ws.ok = false;
+    if (lane < p.batch) {
+        ws.n = seq_nodes(p, lane);
+        ws.L = p.ctx_lens[lane];
+        ws.node_base = seq_node_base(p, lane);
+        ws.ok = seq_shape_ok(p, lane, ws.n, ws.L);
+        ws.tiles = ws.ok ? (ws.L + ws.n + kSchedTileKeys - 1) / kSchedTileKeys : 0;
+    }
+    ws.my_tiles = (long long)ws.tiles * p.num_kv_heads;
+    ws.my_units = ws.ok ? p.num_kv_heads : 0;
+    long long inc_t = ws.my_tiles;
+    int inc_u = ws.my_units, tmin = ws.ok ? ws.tiles : 0x7fffffff, tmax = ws.ok ? ws.tiles : 0;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const long long vt = __shfl_up_sync(0xffffffffu, inc_t, o);
+        const int vu = __shfl_up_sync(0xffffffffu, inc_u, o);
+        if (lane >= o) { inc_t += vt; inc_u += vu; }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        tmin = min(tmin, __shfl_xor_sync(0xffffffffu, tmin, o));
+        tmax = max(tmax, __shfl_xor_sync(0xffffffffu, tmax, o));
+    }
+    ws.total = __shfl_sync(0xffffffffu, inc_t, 31);
+    ws.units = __shfl_sync(0xffffffffu, inc_u, 31);
+    ws.uniform_tiles = (ws.units > 0 && tmin == tmax) ? tmin : 0;
+    ws.excl_t = inc_t - ws.my_tiles;
+    ws.excl_u = inc_u - ws.my_units;
+    return ws;
+}
+
 // Every CTA derives the same per-sequence schedule into shared memory.
 // s_tile[b], s_unit[b] are exclusive prefix sums; entries [batch] hold the totals.
 template <int TileKeys, int RowsPerBlock>

@@ -46,9 +46,6 @@ struct owl_ctx {
     int64_t launches = 0;
     bool profiling = false;
     cudaEvent_t ev[6] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
-    // owl_verify_step: acceptance runs on a stream of its own beside the attention's tail and the combine
-    cudaStream_t side = nullptr;
-    cudaEvent_t fork = nullptr, join = nullptr;
     bool ev_attn_valid = false, ev_accept_valid = false;
     char err[256] = {0};
     // device staging of owl_verify_step_host (grown on demand)
@@ -73,8 +70,8 @@ int cuda_fail(owl_ctx* ctx, cudaError_t e, const char* what) {
 
 // Launch `kernel(arg)` so that it may be scheduled while the kernel before it in the stream is still running
 // (programmatic dependent launch); the kernel itself waits (griddepcontrol.wait) before it reads anything.
-template <typename Arg>
-cudaError_t launch_dependent(void (*kernel)(Arg), dim3 grid, dim3 block, cudaStream_t stream, const Arg& arg) {
+template <typename... Args>
+cudaError_t launch_dependent(void (*kernel)(Args...), dim3 grid, dim3 block, cudaStream_t stream, const Args&... args) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
     cfg.blockDim = block;
@@ -85,7 +82,25 @@ cudaError_t launch_dependent(void (*kernel)(Arg), dim3 grid, dim3 block, cudaStr
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, kernel, arg);
+    return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
+// The attention kernel's instances: [more than 32 sequences][units above 128 rows][logits scan fused in]
+using UmmaKernel = void (*)(AttnParams, CUtensorMap, CUtensorMap, AcceptParams);
+UmmaKernel umma_kernel(bool many, bool wide, bool fused) {
+    static const UmmaKernel table[2][2][2] = {
+        {{umma_path::verify_attn_umma_kernel<false, false, false>, umma_path::verify_attn_umma_kernel<false, false, true>},
+         {umma_path::verify_attn_umma_kernel<false, true, false>, umma_path::verify_attn_umma_kernel<false, true, true>}},
+        {{umma_path::verify_attn_umma_kernel<true, false, false>, umma_path::verify_attn_umma_kernel<true, false, true>},
+         {umma_path::verify_attn_umma_kernel<true, true, false>, umma_path::verify_attn_umma_kernel<true, true, true>}}};
+    return table[many][wide][fused];
+}
+bool set_umma_smem_attr() {
+    bool ok = true;
+    for (int i = 0; i < 8; ++i)
+        ok = ok && cudaFuncSetAttribute(umma_kernel(i & 4, i & 2, i & 1), cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        umma_path::kSmemBytes) == cudaSuccess;
+    return ok;
 }
 
 int log2_exact(int v) {
@@ -199,20 +214,10 @@ int owl_create(owl_ctx** out, int device, const owl_dims* max_dims) {
              cudaMemset(ctx->seq_bad, 0, (size_t)max_dims->batch * sizeof(int32_t)) == cudaSuccess;
     }
     for (int i = 0; ok && i < 6; ++i) ok = cudaEventCreate(&ctx->ev[i]) == cudaSuccess;
-    if (ok) ok = cudaStreamCreateWithFlags(&ctx->side, cudaStreamNonBlocking) == cudaSuccess &&
-                 cudaEventCreateWithFlags(&ctx->fork, cudaEventDisableTiming) == cudaSuccess &&
-                 cudaEventCreateWithFlags(&ctx->join, cudaEventDisableTiming) == cudaSuccess;
     if (ok && attn) {
         ok = cudaFuncSetAttribute(mma_path::verify_attn_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                   mma_path::kSmemBytes) == cudaSuccess &&
-             cudaFuncSetAttribute(umma_path::verify_attn_umma_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                  umma_path::kSmemBytes) == cudaSuccess &&
-             cudaFuncSetAttribute(umma_path::verify_attn_umma_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                  umma_path::kSmemBytes) == cudaSuccess &&
-             cudaFuncSetAttribute(umma_path::verify_attn_umma_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                  umma_path::kSmemBytes) == cudaSuccess &&
-             cudaFuncSetAttribute(umma_path::verify_attn_umma_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                  umma_path::kSmemBytes) == cudaSuccess;
+             set_umma_smem_attr();
     }
     if (!ok || cudaDeviceSynchronize() != cudaSuccess) {
         cudaGetLastError();
@@ -237,16 +242,15 @@ int owl_destroy(owl_ctx* ctx) {
     for (auto& s : ctx->stg) cudaFree(s.p);
     for (auto& ev : ctx->ev)
         if (ev) cudaEventDestroy(ev);
-    if (ctx->fork) cudaEventDestroy(ctx->fork);
-    if (ctx->join) cudaEventDestroy(ctx->join);
-    if (ctx->side) cudaStreamDestroy(ctx->side);
     delete ctx;
     return OWL_OK;
 }
 
-int owl_verify_attn(owl_ctx* ctx, const owl_dims* d, const void* q, const void* k_cache, const void* v_cache,
-                    const int32_t* block_table, const int32_t* ctx_lens, const int32_t* node_offsets,
-                    const int32_t* tree_parent, void* out, float* lse, void* stream_) {
+// Attention of a verify step.  `ap` non-null (tcgen05 path only): the logits scan rides in the attention kernel's
+// spare warps and the acceptance walk in the merge kernel, two launches for the whole step.
+static int verify_attn_impl(owl_ctx* ctx, const owl_dims* d, const void* q, const void* k_cache, const void* v_cache,
+                            const int32_t* block_table, const int32_t* ctx_lens, const int32_t* node_offsets,
+                            const int32_t* tree_parent, void* out, float* lse, void* stream_, const AcceptParams* ap) {
     if (!ctx) return OWL_ERR_INVALID_ARG;
     int rc = check_dims(d, true, false);
     if (rc != OWL_OK) return rc;
@@ -323,15 +327,14 @@ int owl_verify_attn(owl_ctx* ctx, const owl_dims* d, const void* q, const void* 
             cfg.attrs = attr;
             cfg.numAttrs = 1;
             // the instance that holds only this call's case: block-wide schedule above 32 sequences, the two-row-block
-            // mode only if a unit (G * max_nodes rows at most) can exceed 128 rows
+            // mode only if a unit (G * max_nodes rows at most) can exceed 128 rows, the logits scan only in a step
             const bool many = d->batch > 32, wide = G * d->max_nodes > 128;
-            auto kernel = many ? (wide ? umma_path::verify_attn_umma_kernel<true, true> : umma_path::verify_attn_umma_kernel<true, false>)
-                               : (wide ? umma_path::verify_attn_umma_kernel<false, true> : umma_path::verify_attn_umma_kernel<false, false>);
-            cudaLaunchKernelEx(&cfg, kernel, p, ctx->kmap, ctx->vmap);
+            cudaLaunchKernelEx(&cfg, umma_kernel(many, wide, ap != nullptr), p, ctx->kmap, ctx->vmap, ap ? *ap : AcceptParams{});
         }
         ++ctx->launches;
         if (ctx->profiling) cudaEventRecord(ctx->ev[1], stream);
-        launch_dependent(combine_sched_kernel, dim3(grid), dim3(kCombineWarps * 32), stream, p);
+        if (ap) launch_dependent(combine_sched_kernel<true>, dim3(grid + (unsigned)d->batch), dim3(kCombineWarps * 32), stream, p, *ap);
+        else launch_dependent(combine_sched_kernel<false>, dim3(grid), dim3(kCombineWarps * 32), stream, p, AcceptParams{});
     } else {
         mma_path::verify_attn_mma_kernel<<<ctx->num_ctas, mma_path::kThreads, mma_path::kSmemBytes, stream>>>(p);
         ++ctx->launches;
@@ -345,9 +348,17 @@ int owl_verify_attn(owl_ctx* ctx, const owl_dims* d, const void* q, const void* 
     return OWL_OK;
 }
 
-int owl_tree_accept(owl_ctx* ctx, const owl_dims* d, const float* logits, const int32_t* draft_tokens,
-                    const int32_t* node_offsets, const int32_t* tree_parent, int32_t* accept_len,
-                    int32_t* accept_path, int32_t* bonus_token, int32_t* node_argmax, void* stream_) {
+int owl_verify_attn(owl_ctx* ctx, const owl_dims* d, const void* q, const void* k_cache, const void* v_cache,
+                    const int32_t* block_table, const int32_t* ctx_lens, const int32_t* node_offsets,
+                    const int32_t* tree_parent, void* out, float* lse, void* stream_) {
+    return verify_attn_impl(ctx, d, q, k_cache, v_cache, block_table, ctx_lens, node_offsets, tree_parent, out, lse, stream_,
+                            nullptr);
+}
+
+// Argument checks of the acceptance and its kernel parameters (everything but the counters of the stand-alone kernel).
+static int accept_params(owl_ctx* ctx, const owl_dims* d, const float* logits, const int32_t* draft_tokens,
+                         const int32_t* node_offsets, const int32_t* tree_parent, int32_t* accept_len,
+                         int32_t* accept_path, int32_t* bonus_token, int32_t* node_argmax, AcceptParams& p) {
     if (!ctx) return OWL_ERR_INVALID_ARG;
     int rc = check_dims(d, false, true);
     if (rc != OWL_OK) return rc;
@@ -357,10 +368,7 @@ int owl_tree_accept(owl_ctx* ctx, const owl_dims* d, const float* logits, const 
     if (d->total_nodes > 65535) return OWL_ERR_UNSUPPORTED;
     const int chunks = (d->vocab + kArgmaxChunk - 1) / kArgmaxChunk;
     if (!ctx->part_keys || (long long)d->total_nodes * chunks > ctx->part_keys_len) return OWL_ERR_TOO_LARGE;
-
-    DeviceGuard guard(ctx->device);
-    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-    AcceptParams p{};
+    p = AcceptParams{};
     p.logits = logits;
     p.draft_tokens = draft_tokens;
     p.node_offsets = node_offsets;
@@ -378,7 +386,19 @@ int owl_tree_accept(owl_ctx* ctx, const owl_dims* d, const float* logits, const 
     p.max_nodes = d->max_nodes;
     p.vocab = d->vocab;
     p.path_stride = d->path_stride;
+    return OWL_OK;
+}
 
+int owl_tree_accept(owl_ctx* ctx, const owl_dims* d, const float* logits, const int32_t* draft_tokens,
+                    const int32_t* node_offsets, const int32_t* tree_parent, int32_t* accept_len,
+                    int32_t* accept_path, int32_t* bonus_token, int32_t* node_argmax, void* stream_) {
+    AcceptParams p;
+    const int rc = accept_params(ctx, d, logits, draft_tokens, node_offsets, tree_parent, accept_len, accept_path, bonus_token,
+                                 node_argmax, p);
+    if (rc != OWL_OK) return rc;
+    DeviceGuard guard(ctx->device);
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const int chunks = p.chunks;
     p.seq_counter = ctx->seq_counter;
     p.counter_stride = ctx->max_dims.batch;
     p.epoch = ++ctx->accept_epoch;
@@ -400,33 +420,23 @@ int owl_verify_step(owl_ctx* ctx, const owl_dims* d, const void* q, const void* 
     if (!ctx) return OWL_ERR_INVALID_ARG;
     int rc = check_dims(d, true, true);
     if (rc != OWL_OK) return rc;
-    DeviceGuard guard(ctx->device);
-    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-    // A scan of at most about one wave of CTAs hides in the tail of the attention pass; a larger one would
-    // take SMs from the persistent attention CTAs at their start, so it simply follows in stream order.
-    const long long scan_ctas = (long long)d->total_nodes * ((d->vocab + kArgmaxChunk - 1) / kArgmaxChunk);
-    if (scan_ctas > 1024) {
+    // A scan of up to about a thousand (row, chunk) items - a few per spare warp - rides inside the attention kernel;
+    // a larger one slows the attention down by more than its own kernel costs (measured: 4 x 64 nodes of a 128K
+    // vocabulary, 570 -> 605 us), so it follows as a kernel of its own in stream order.
+    const long long scan_items = (long long)d->total_nodes * ((d->vocab + kArgmaxChunk - 1) / kArgmaxChunk);
+    if (!ctx->use_umma || scan_items > 1024) {
         rc = owl_verify_attn(ctx, d, q, k_cache, v_cache, block_table, ctx_lens, node_offsets, tree_parent, out, lse, stream_);
         if (rc != OWL_OK) return rc;
         return owl_tree_accept(ctx, d, logits, draft_tokens, node_offsets, tree_parent, accept_len, accept_path, bonus_token,
                                node_argmax, stream_);
     }
-    // fork: what the caller queued before this call is complete before either half starts
-    cudaError_t e = cudaEventRecord(ctx->fork, stream);
-    if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->side, ctx->fork, 0);
-    if (e != cudaSuccess) return cuda_fail(ctx, e, "owl_verify_step fork");
-    rc = owl_verify_attn(ctx, d, q, k_cache, v_cache, block_table, ctx_lens, node_offsets, tree_parent, out, lse, stream_);
-    int rc2 = OWL_OK;
-    if (rc == OWL_OK)
-        rc2 = owl_tree_accept(ctx, d, logits, draft_tokens, node_offsets, tree_parent, accept_len, accept_path, bonus_token,
-                              node_argmax, ctx->side);
-    // join (always, so that the side stream never runs ahead of the caller's)
-    e = cudaEventRecord(ctx->join, ctx->side);
-    if (e == cudaSuccess) e = cudaStreamWaitEvent(stream, ctx->join, 0);
+    // Two launches: the attention kernel, whose two spare warps per CTA scan the logits while K/V stream in, and the
+    // merge kernel, which also walks the trees.
+    AcceptParams ap;
+    rc = accept_params(ctx, d, logits, draft_tokens, node_offsets, tree_parent, accept_len, accept_path, bonus_token, node_argmax, ap);
     if (rc != OWL_OK) return rc;
-    if (rc2 != OWL_OK) return rc2;
-    if (e != cudaSuccess) return cuda_fail(ctx, e, "owl_verify_step join");
-    return OWL_OK;
+    ctx->ev_accept_valid = false;
+    return verify_attn_impl(ctx, d, q, k_cache, v_cache, block_table, ctx_lens, node_offsets, tree_parent, out, lse, stream_, &ap);
 }
 
 int owl_verify_step_host(owl_ctx* ctx, const owl_dims* d, const void* q_h, const void* k_h, const void* v_h,

@@ -34,6 +34,7 @@
 
 #include "kv_tensor_map.cuh"
 #include "owl_common.cuh"
+#include "accept.cuh"
 #include "sm100_ptx.cuh"
 
 namespace owl {
@@ -213,40 +214,16 @@ __device__ __forceinline__ void build_walk(const AttnParams& p, Aux* aux, Walker
 // b, prefix sums by shuffle), with no shared memory and no CTA-wide barrier, so that each role can start
 // as soon as its own loads have returned.
 __device__ __forceinline__ void build_walk_small(const AttnParams& p, Walker& w) {
+    static_assert(kTileKeys == kSchedTileKeys, "the merge kernel derives the same schedule");
     const int lane = threadIdx.x & 31;
-    int n = 0, L = 0, node_base = 0, tiles = 0;
-    bool ok = false;
-    if (lane < p.batch) {
-        n = seq_nodes(p, lane);
-        L = p.ctx_lens[lane];
-        node_base = seq_node_base(p, lane);
-        ok = seq_shape_ok(p, lane, n, L);
-        tiles = ok ? (L + n + kTileKeys - 1) / kTileKeys : 0;
-        if (!ok && threadIdx.x < 32) {
-            report(p.status, seq_tree_shape_ok(p, lane, n) ? kErrBadPage : kErrBadTree);
-            p.seq_bad[lane] = p.epoch;
-        }
+    const WarpSchedule ws = warp_schedule(p);
+    const int n = ws.n, L = ws.L, node_base = ws.node_base, tiles = ws.tiles;
+    if (lane < p.batch && !ws.ok && threadIdx.x < 32) {
+        report(p.status, seq_tree_shape_ok(p, lane, n) ? kErrBadPage : kErrBadTree);
+        p.seq_bad[lane] = p.epoch;
     }
-    const long long my_tiles = (long long)tiles * p.num_kv_heads;
-    const int my_units = ok ? p.num_kv_heads : 0;
-    long long inc_t = my_tiles;
-    int inc_u = my_units, tmin = ok ? tiles : 0x7fffffff, tmax = ok ? tiles : 0;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const long long vt = __shfl_up_sync(0xffffffffu, inc_t, o);
-        const int vu = __shfl_up_sync(0xffffffffu, inc_u, o);
-        if (lane >= o) { inc_t += vt; inc_u += vu; }
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        tmin = min(tmin, __shfl_xor_sync(0xffffffffu, tmin, o));
-        tmax = max(tmax, __shfl_xor_sync(0xffffffffu, tmax, o));
-    }
-    const long long total = __shfl_sync(0xffffffffu, inc_t, 31);
-    const int units = __shfl_sync(0xffffffffu, inc_u, 31);
-    const int uniform_tiles = (units > 0 && tmin == tmax) ? tmin : 0;
-    const long long excl_t = inc_t - my_tiles;
-    const int excl_u = inc_u - my_units;
+    const long long my_tiles = ws.my_tiles, total = ws.total, excl_t = ws.excl_t;
+    const int units = ws.units, uniform_tiles = ws.uniform_tiles, excl_u = ws.excl_u;
     Partition part;
     part.init(total, gridDim.x, units, uniform_tiles);
     const long long t_begin = part.begin(blockIdx.x), t_end = part.begin(blockIdx.x + 1);
@@ -786,12 +763,16 @@ __device__ __forceinline__ void softmax_loop(const AttnParams& p, Aux* aux, unsi
 }
 
 // ------------------------------------------------------------------------------------------ kernel
-// kManySeqs: more than 32 sequences (the block-wide schedule); kWide: some unit may have more than 128 rows.  Four
-// instances, so that a launch carries only the code of its own case: the text of the paths a launch never takes
+// kManySeqs: more than 32 sequences (the block-wide schedule); kWide: some unit may have more than 128 rows.
+// Separate instances, so that a launch carries only the code of its own case: the text of the paths a launch never takes
 // still costs it time (3 us of 39 on a 32K-context, 32-node step when the block-wide schedule was compiled in).
-template <bool kManySeqs, bool kWide>
+// kFused: the verify step's logits scan rides along.  Warps 2 and 3 have no part in the attention; they take the
+// (row, vocabulary chunk) items of the arg-max scan in turn, 2 x gridDim.x warps in all, and leave one key per item
+// for the acceptance walk, which the merge kernel runs after this grid (`ap` is not looked at otherwise).
+template <bool kManySeqs, bool kWide, bool kFused>
 __global__ void __launch_bounds__(kThreads, 1)
-verify_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap vmap) {
+verify_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap vmap,
+                        const AcceptParams ap) {
     extern __shared__ __align__(1024) unsigned char smem[];
     Aux* aux = reinterpret_cast<Aux*>(smem + kAuxOff);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -837,6 +818,11 @@ verify_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap 
         asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
         if (warp == 0) producer_loop<kWide>(p, &kmap, &vmap, aux, smem_base + kRingOff, w, items);
         else if (warp == 1) mma_loop<kWide>(p, aux, smem_base, tmem, w);
+        else if (kFused) {
+            const long long items = (long long)ap.total_nodes * ap.chunks;
+            for (long long it = 2ll * blockIdx.x + (warp - 2); it < items; it += 2ll * gridDim.x)
+                argmax_scan_chunk_warp(ap, (int)(it / ap.chunks), (int)(it % ap.chunks));
+        }
     } else {
         asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
         softmax_loop<kWide>(p, aux, smem, tmem, w, warp >= 8 ? 1 : 0);
