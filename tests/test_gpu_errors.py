@@ -89,6 +89,15 @@ def test_bad_tree_is_reported_and_isolated():
     alen = dw.accept_len.cpu().numpy()
     assert alen[1] == -5 and alen[0] == r_alen[0] and alen[2] == r_alen[2]
     assert ctx.owl_get_status() == 0                            # reading the status clears it
+    # the whole step in one call (scan and walk inside the attention kernels): same verdict, same isolation
+    dw.out.fill_(7.0); dw.accept_len.fill_(-5)
+    dw.step(ctx)
+    assert ctx.owl_get_status() == -4
+    out = dw.out_f32()
+    assert np.all(out[8:12] == 7.0)
+    assert np.abs(out[:8] - ref_out[:8]).max() <= 1e-2 and np.abs(out[12:] - ref_out[12:]).max() <= 1e-2
+    alen = dw.accept_len.cpu().numpy()
+    assert alen[1] == -5 and alen[0] == r_alen[0] and alen[2] == r_alen[2]
     # the context stays usable
     dw2 = DeviceWorkload.upload(wl)
     dw2.step(ctx)

@@ -211,9 +211,15 @@ def test_other_page_sizes(page):
     check_attention(wl)
 
 
-def test_verify_step_equals_the_two_calls():
-    """owl_verify_step (acceptance beside the attention pass) gives bit for bit what the two calls give."""
-    wl = W.generate(W.Spec("step", 32, 8, [1500, 40], [("tree", 32, 6), ("chain", 8)], shuffle_pages=True, seed=411, vocab=20000))
+@pytest.mark.parametrize("vocab", [
+    20000,     # rows 16-byte aligned, three chunks per row: the scan rides in the attention kernel's spare warps
+    1003,      # rows not 16-byte aligned: scalar head and tail of every chunk
+    8193,      # a second chunk of one element
+    250000,    # 40 nodes x 31 chunks > 1024 items: the scan follows as a kernel of its own
+])
+def test_verify_step_equals_the_two_calls(vocab):
+    """owl_verify_step (acceptance inside the attention kernels, or after them) gives bit for bit what the two calls give."""
+    wl = W.generate(W.Spec("step", 32, 8, [1500, 40], [("tree", 32, 6), ("chain", 8)], shuffle_pages=True, seed=411, vocab=vocab))
     dw = DeviceWorkload.upload(wl)
     ctx = OwlContext(dims_of(wl))
     dw.attn(ctx)
