@@ -5,6 +5,7 @@
 //   warp 0        TMA producer: per 128-key tile, one box per (page, head) for K and for V into a
 //                 ring of 32 KB shared-memory slots (layout in kv_tensor_map.cuh)
 //   warp 1        issues every tcgen05.mma (one lane) and the commits that signal their completion
+//   warps 2-3     no part in the attention; in a verify step with a small logits scan they do that scan
 //   warps 4-7     softmax warpgroup of stream 0   (one thread per packed row)
 //   warps 8-11    softmax warpgroup of stream 1
 // A unit is one (sequence, KV head) with M = G * n packed rows (row = node * G + head in group).
@@ -59,7 +60,7 @@ constexpr float kLazyRescale = 8.0f;       // log2 units
 struct Aux {
     uint64_t full[kTilesInFlight];   // one per tile: its K and its V slot complete the same barrier
     uint64_t empty[kSlots];
-    uint64_t s_full[2], p_full[2], o_done[2];
+    uint64_t s_full[2], o_done[2];
     uint64_t q_full;
     uint32_t tmem_base;
     int abort_flag;
@@ -788,7 +789,6 @@ verify_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap 
         for (int i = 0; i < kTilesInFlight; ++i) mbar_init(smem_u32(&aux->full[i]), 1);
         for (int s = 0; s < 2; ++s) {
             mbar_init(smem_u32(&aux->s_full[s]), 1);
-            mbar_init(smem_u32(&aux->p_full[s]), 128);
             mbar_init(smem_u32(&aux->o_done[s]), 1);
         }
         mbar_init(smem_u32(&aux->q_full), 256);
