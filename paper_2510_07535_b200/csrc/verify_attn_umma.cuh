@@ -33,6 +33,8 @@
 // the status word reports OWL_ERR_TIMEOUT.
 #pragma once
 
+#include <type_traits>
+
 #include "kv_tensor_map.cuh"
 #include "owl_common.cuh"
 #include "accept.cuh"
@@ -312,9 +314,10 @@ __device__ __forceinline__ void producer_loop(const AttnParams& p, const CUtenso
 //    the guard (`elected` lane, waits succeeded, work to do) themselves.  What steers the loop (the segment's tile
 //    range and mode, the verdicts of the waits) goes through a warp reduction or a vote first, so that trip counts,
 //    ring slots and descriptors are uniform by construction;
-//  * per stream and tile of such a unit it waits on two hardware barriers (about 25 clocks each when the arrival is
-//    already in; a look at an mbarrier costs 70 to 130): on one the softmax warpgroup announces P, on the other
-//    that it has seen the stream's next key tile arrive (units of up to 128 rows wait for the tile itself);
+//  * per tile of such a unit it waits on hardware barriers only (about 25 clocks each when the arrival is already
+//    in; a look at an mbarrier costs 70 to 130): one per stream, on which the softmax warpgroup announces P, and
+//    one on which stream 0's warpgroup tells that it has seen the next key tile arrive (units of up to 128 rows
+//    wait for the tile itself);
 //  * the iterations in which both streams have both products to issue run in a loop of their own without
 //    per-product conditions; the first and the last ones of a segment take the general form.
 template <bool kWide>
@@ -372,11 +375,12 @@ __device__ __forceinline__ void mma_loop(const AttnParams& p, Aux* aux, uint32_t
         };
         // Before S = Q K^T of the stream's tile i + 1.  M > 128: the issue loop is what bounds the unit, and the
         // softmax warpgroup, which has time to spare, looks at the tile's arrival barrier and passes the news on
-        // through hardware barrier 6 + s (about 25 clocks here).  M <= 128: the tile itself is what the warp
+        // through hardware barrier 6 (about 25 clocks here).  M <= 128: the tile itself is what the warp
         // usually waits for, and it waits on the arrival barrier directly, one wake-up instead of two.
         auto wait_next_k = [&](int s, int i) {
             if (shared) {
-                asm volatile("bar.sync %0, 64;" ::"r"(6 + s) : "memory");
+                // (both streams read the tile: stream 1 finds what stream 0 has just made sure of)
+                if (s == 0) asm volatile("bar.sync 6, 64;" ::: "memory");
             } else {
                 const uint32_t seq = (item_base >> 1) + (uint32_t)(2 * (i + 1) + s);
                 ok = __all_sync(kAll, mbar_wait(smem_u32(&aux->full[seq % kTilesInFlight]), (seq / kTilesInFlight) & 1u,
@@ -436,20 +440,26 @@ __device__ __forceinline__ void mma_loop(const AttnParams& p, Aux* aux, uint32_t
         for (int i = -1; i < n_it[0]; ++i) {
             if (i < 0 || i >= n_it[1] - 1) { general(i); continue; }
             const uint32_t issue = ok ? elected : 0u;
+            // one body per mode, so that what a mode does not need (stream 0's slot releases and stream 1's tile
+            // barrier when both streams read every tile) is not even a predicated-off instruction
+            auto steady = [&](auto mode) {
+                constexpr bool kBoth = decltype(mode)::value;
 #pragma unroll
-            for (int s = 0; s < 2; ++s) {
-                const uint32_t issue_last = (shared && s == 0) ? 0u : issue;
-                asm volatile("bar.sync %0, 160;" ::"r"(4 + s) : "memory");
-                tc_fence_after();
-                issue_pv(s, issue, i > 0 ? 1u : 0u);
-                umma_commit_if(issue_last, smem_u32(&aux->empty[v_slot[s]]));
-                advance(v_slot[s]);
-                wait_next_k(s, i);                                          // the next K tile has landed
-                issue_qk(s, ok ? issue : 0u);
-                umma_commit_if(issue, smem_u32(&aux->s_full[s]));
-                umma_commit_if(issue_last, smem_u32(&aux->empty[k_slot[s]]));
-                advance(k_slot[s]);
-            }
+                for (int s = 0; s < 2; ++s) {
+                    constexpr bool kRelease = !kBoth;   // (for s == 1 see below)
+                    asm volatile("bar.sync %0, 160;" ::"r"(4 + s) : "memory");
+                    tc_fence_after();
+                    issue_pv(s, issue, i > 0 ? 1u : 0u);
+                    if (kRelease || s == 1) umma_commit_if(issue, smem_u32(&aux->empty[v_slot[s]]));
+                    advance(v_slot[s]);
+                    wait_next_k(s, i);                                      // the next K tile has landed
+                    issue_qk(s, ok ? issue : 0u);
+                    umma_commit_if(issue, smem_u32(&aux->s_full[s]));
+                    if (kRelease || s == 1) umma_commit_if(issue, smem_u32(&aux->empty[k_slot[s]]));
+                    advance(k_slot[s]);
+                }
+            };
+            if (kWide && shared) steady(std::true_type{}); else steady(std::false_type{});
         }
         item_base += 2u * (uint32_t)T;
         ++seg_no;
@@ -685,12 +695,12 @@ __device__ __forceinline__ void softmax_loop(const AttnParams& p, Aux* aux, unsi
             // In a unit of more than 128 rows the MMA warp polls no mbarrier between O += P V of this tile and
             // S = Q K^T of the next one: the first warp of the warpgroup looks at that tile's arrival barrier for it
             // (after P is announced, so that nothing this tile holds is released any later) and passes the news on
-            // through hardware barrier 6 + s.  A wait that gives up raises the abort flag; the arrival happens all
-            // the same.
-            if (g.shared && wtid < 32 && i + 1 < n_it) {
+            // through hardware barrier 6 (stream 0's warpgroup does; the tile is the same for both streams).  A wait
+            // that gives up raises the abort flag; the arrival happens all the same.
+            if (g.shared && s == 0 && wtid < 32 && i + 1 < n_it) {
                 const uint32_t seq = tile_base + (uint32_t)(i + 1);
                 mbar_wait(smem_u32(&aux->full[seq % kTilesInFlight]), (seq / kTilesInFlight) & 1u, abort_flag);
-                asm volatile("bar.arrive %0, 64;" ::"r"(6 + s) : "memory");
+                asm volatile("bar.arrive 6, 64;" ::: "memory");
             }
             ++it;
         }
