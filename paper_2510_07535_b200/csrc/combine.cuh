@@ -86,7 +86,12 @@ __global__ void __launch_bounds__(kCombineWarps * 32) combine_kernel(const AttnP
 //
 // kFused (verify step): the grid has one more CTA per sequence after the row CTAs; each of those runs one
 // sequence's acceptance walk over the arg-max keys that the pass's spare warps left (`ap`).
-template <bool kFused>
+//
+// kGroup: partials fetched per round, 16 or 32.  A unit cut into 17 to 32 pieces (8 units of a 32K context over 148
+// CTAs: 18 or 19) costs a second round of loads with 16, which is a whole memory round trip of a kernel that is
+// all latency; with 32 the registers of a thread double, which costs occupancy where there are rows enough to
+// fill the machine.  The host takes 32 up to 4096 output rows.
+template <bool kFused, int kGroup>
 __global__ void __launch_bounds__(kCombineWarps * 32) combine_sched_kernel(const AttnParams p, const AcceptParams ap) {
     if (kFused) {
         const long long rows = (long long)p.total_nodes * p.num_q_heads;
@@ -127,7 +132,7 @@ __global__ void __launch_bounds__(kCombineWarps * 32) combine_sched_kernel(const
         t0 = seq_begin + (long long)(hq / G) * tiles;
         c0 = part.owner(t0);
         c1 = part.owner(t0 + tiles - 1);
-        prow_first = row_of(c0 + min(lane & 15, c1 - c0));
+        prow_first = row_of(c0 + min(lane & (kGroup - 1), c1 - c0));
     };
     if (small) plan();
     // from here on the split-KV pass has completed and its writes are visible (a no-op in an ordinary launch)
@@ -156,25 +161,26 @@ __global__ void __launch_bounds__(kCombineWarps * 32) combine_sched_kernel(const
     const int bad_epoch = __ldcg(p.seq_bad + b);   // (its round trip overlaps the partial loads below)
     const int count = c1 - c0 + 1;
 
-    // Partials are taken 16 at a time: lane j (< 16) of a group owns partial base + j.  The row loads do not
-    // depend on the LSE values, so both go out together: one memory round trip per group, and units cut into
-    // at most 16 pieces - the usual case - need a single group.  Groups are folded online (running maximum).
+    // Partials are taken kGroup at a time: lane j (< kGroup) of a group owns partial base + j.  The row loads do
+    // not depend on the LSE values, so both go out together: one memory round trip per group.  Groups are folded
+    // online (running maximum).
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     float sum = 0.f, mx = -INFINITY;
-    for (int base = 0; base < count; base += 16) {
-        const int mine = base + (lane & 15);
+    for (int base = 0; base < count; base += kGroup) {
+        const int mine = base + (lane & (kGroup - 1));
         const bool have = mine < count;
         const long long prow = base == 0 ? prow_first : row_of(c0 + (have ? mine : 0));
         const float my_lse = have ? __ldcg(p.part_lse + prow) : -INFINITY;
-        float4 v[16];
+        float4 v[kGroup];
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {
+        for (int j = 0; j < kGroup; ++j) {
             const long long pj = __shfl_sync(0xffffffffu, prow, j);
-            v[j] = __ldcg(reinterpret_cast<const float4*>(p.part_o + pj * kHeadDim + lane * 4));
+            v[j] = base + j < count ? __ldcg(reinterpret_cast<const float4*>(p.part_o + pj * kHeadDim + lane * 4))
+                                    : make_float4(0.f, 0.f, 0.f, 0.f);
         }
         float gmx = my_lse;
 #pragma unroll
-        for (int o = 8; o > 0; o >>= 1) gmx = fmaxf(gmx, __shfl_xor_sync(0xffffffffu, gmx, o));
+        for (int o = kGroup / 2; o > 0; o >>= 1) gmx = fmaxf(gmx, __shfl_xor_sync(0xffffffffu, gmx, o));
         const float mx_new = fmaxf(mx, gmx);
         if (mx_new > -INFINITY) {
             const float rescale = mx > -INFINITY ? __expf(mx - mx_new) : 0.f;
@@ -182,7 +188,7 @@ __global__ void __launch_bounds__(kCombineWarps * 32) combine_sched_kernel(const
             sum *= rescale;
             const float w = have ? __expf(my_lse - mx_new) : 0.f;     // -inf partial: weight 0
 #pragma unroll
-            for (int j = 0; j < 16; ++j) {
+            for (int j = 0; j < kGroup; ++j) {
                 const float wj = __shfl_sync(0xffffffffu, w, j);
                 acc.x += wj * v[j].x; acc.y += wj * v[j].y; acc.z += wj * v[j].z; acc.w += wj * v[j].w;
                 sum += wj;

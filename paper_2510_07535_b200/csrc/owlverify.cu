@@ -333,8 +333,13 @@ static int verify_attn_impl(owl_ctx* ctx, const owl_dims* d, const void* q, cons
         }
         ++ctx->launches;
         if (ctx->profiling) cudaEventRecord(ctx->ev[1], stream);
-        if (ap) launch_dependent(combine_sched_kernel<true>, dim3(grid + (unsigned)d->batch), dim3(kCombineWarps * 32), stream, p, *ap);
-        else launch_dependent(combine_sched_kernel<false>, dim3(grid), dim3(kCombineWarps * 32), stream, p, AcceptParams{});
+        const bool few_rows = rows <= 4096;      // latency-bound merge: 32 partials per round (see combine.cuh)
+        if (ap)
+            launch_dependent(few_rows ? combine_sched_kernel<true, 32> : combine_sched_kernel<true, 16>,
+                             dim3(grid + (unsigned)d->batch), dim3(kCombineWarps * 32), stream, p, *ap);
+        else
+            launch_dependent(few_rows ? combine_sched_kernel<false, 32> : combine_sched_kernel<false, 16>, dim3(grid),
+                             dim3(kCombineWarps * 32), stream, p, AcceptParams{});
     } else {
         mma_path::verify_attn_mma_kernel<<<ctx->num_ctas, mma_path::kThreads, mma_path::kSmemBytes, stream>>>(p);
         ++ctx->launches;
