@@ -84,8 +84,16 @@ struct Partition {
     long long total, q;
     int rem, ctas;
     int unit_tiles, base, urem;   // aligned mode iff unit_tiles > 0
+    // (Every CTA runs this once, on its critical path and with cold instruction caches, where each instruction costs
+    // tens of nanoseconds: one 32-bit division where the numbers allow it instead of 64-bit ones.)
     __device__ __host__ void init(long long total_, int ctas_) {
-        total = total_; ctas = ctas_; q = total_ / ctas_; rem = (int)(total_ % ctas_);
+        total = total_; ctas = ctas_;
+        if (total_ >= 0 && total_ <= 0x7fffffffll) {
+            const unsigned qq = (unsigned)total_ / (unsigned)ctas_;
+            q = qq; rem = (int)((unsigned)total_ - qq * (unsigned)ctas_);
+        } else {
+            q = total_ / ctas_; rem = (int)(total_ % ctas_);
+        }
         unit_tiles = 0; base = 0; urem = 0;
     }
     __device__ __host__ void init(long long total_, int ctas_, int units, int uniform_tiles) {
@@ -93,9 +101,25 @@ struct Partition {
         if (uniform_tiles > 0 && units > 1 && units <= ctas_) {
             const int b = ctas_ / units;
             const long long cost_aligned = (uniform_tiles + b - 1) / b;
-            const long long cost_flat = (total_ + ctas_ - 1) / ctas_ + kBoundaryPenaltyTiles;
-            if (cost_aligned < cost_flat) { unit_tiles = uniform_tiles; base = b; urem = ctas_ % units; }
+            const long long cost_flat = q + (rem ? 1 : 0) + kBoundaryPenaltyTiles;   // ceil(total / ctas) + penalty
+            if (cost_aligned < cost_flat) { unit_tiles = uniform_tiles; base = b; urem = ctas_ - b * units; }
         }
+    }
+    // [begin(c), begin(c + 1)) with one set of divisions (the pieces of a unit tile it exactly, so a piece's end is
+    // its begin plus its length in either mode)
+    __device__ __host__ void range(int c, long long& t_begin, long long& t_end) const {
+        if (unit_tiles == 0) {
+            t_begin = (long long)c * q + (c < rem ? c : rem);
+            t_end = t_begin + q + (c < rem ? 1 : 0);
+            return;
+        }
+        const int big = urem * (base + 1);
+        int u, k, cu;
+        if (c < big) { u = c / (base + 1); k = c - u * (base + 1); cu = base + 1; }
+        else { u = urem + (c - big) / base; k = (c - big) - (u - urem) * base; cu = base; }
+        const int qq = unit_tiles / cu, rr = unit_tiles - qq * cu;
+        t_begin = (long long)u * unit_tiles + (long long)k * qq + (k < rr ? k : rr);
+        t_end = t_begin + qq + (k < rr ? 1 : 0);
     }
     __device__ __host__ long long begin(int c) const {
         if (unit_tiles == 0) return (long long)c * q + (c < rem ? c : rem);

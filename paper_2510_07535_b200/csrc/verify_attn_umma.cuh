@@ -185,7 +185,8 @@ __device__ __forceinline__ void build_walk(const AttnParams& p, Aux* aux, Walker
     const int excl_u = off_u + inc_u - my_units;
     Partition part;
     part.init(total, gridDim.x, units, uniform_tiles);
-    const long long t_begin = part.begin(blockIdx.x), t_end = part.begin(blockIdx.x + 1);
+    long long t_begin, t_end;
+    part.range(blockIdx.x, t_begin, t_end);
     if (t_begin < t_end && my_tiles > 0 && t_begin >= excl_t && t_begin < excl_t + my_tiles) {
         aux->sched_b0 = b_lo;                 // the walker skips ahead from the first sequence of this thread
         aux->sched_tile_begin = excl_t;
@@ -229,7 +230,8 @@ __device__ __forceinline__ void build_walk_small(const AttnParams& p, Walker& w)
     const int units = ws.units, uniform_tiles = ws.uniform_tiles, excl_u = ws.excl_u;
     Partition part;
     part.init(total, gridDim.x, units, uniform_tiles);
-    const long long t_begin = part.begin(blockIdx.x), t_end = part.begin(blockIdx.x + 1);
+    long long t_begin, t_end;
+    part.range(blockIdx.x, t_begin, t_end);
     const unsigned owner = __ballot_sync(0xffffffffu, my_tiles > 0 && t_begin >= excl_t && t_begin < excl_t + my_tiles);
     if (blockIdx.x == 0 && threadIdx.x < 32) {
         if (lane < p.batch) p.sched_seq_begin[lane] = excl_t;
