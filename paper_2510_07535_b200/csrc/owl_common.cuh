@@ -198,19 +198,26 @@ __device__ __forceinline__ WarpSchedule warp_schedule(const AttnParams& p) {
     ws.my_units = ws.ok ? p.num_kv_heads : 0;
     long long inc_t = ws.my_tiles;
     int inc_u = ws.my_units, tmin = ws.ok ? ws.tiles : 0x7fffffff, tmax = ws.ok ? ws.tiles : 0;
+    // as many rounds as the batch needs (one sequence: none): this runs once per launch on every CTA's critical
+    // path, where an instruction costs tens of nanoseconds.  Lanes >= batch hold zeros / neutral elements.
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
+        if (o >= p.batch) break;
         const long long vt = __shfl_up_sync(0xffffffffu, inc_t, o);
         const int vu = __shfl_up_sync(0xffffffffu, inc_u, o);
         if (lane >= o) { inc_t += vt; inc_u += vu; }
     }
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        tmin = min(tmin, __shfl_xor_sync(0xffffffffu, tmin, o));
-        tmax = max(tmax, __shfl_xor_sync(0xffffffffu, tmax, o));
+    for (int o = 1; o < 32; o <<= 1) {               // after the rounds with o < batch, lane 0 covers [0, batch)
+        if (o >= p.batch) break;
+        tmin = min(tmin, __shfl_down_sync(0xffffffffu, tmin, o));
+        tmax = max(tmax, __shfl_down_sync(0xffffffffu, tmax, o));
     }
-    ws.total = __shfl_sync(0xffffffffu, inc_t, 31);
-    ws.units = __shfl_sync(0xffffffffu, inc_u, 31);
+    tmin = __shfl_sync(0xffffffffu, tmin, 0);
+    tmax = __shfl_sync(0xffffffffu, tmax, 0);
+    const int last = p.batch < 32 ? p.batch - 1 : 31;
+    ws.total = __shfl_sync(0xffffffffu, inc_t, last);
+    ws.units = __shfl_sync(0xffffffffu, inc_u, last);
     ws.uniform_tiles = (ws.units > 0 && tmin == tmax) ? tmin : 0;
     ws.excl_t = inc_t - ws.my_tiles;
     ws.excl_u = inc_u - ws.my_units;
