@@ -491,8 +491,9 @@ __device__ __forceinline__ void store_rows32(const AttnParams& p, float* stage, 
     for (int j = 0; j < 8; ++j)
         *reinterpret_cast<float4*>(stage + lane * kStageStride + 4 * j) = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
     __syncwarp();
+    // (rolled: this code runs a few times per launch, with cold instruction caches, where its length counts)
     if (kFinal) {
-#pragma unroll
+#pragma unroll 1
         for (int k = 0; k < 4; ++k) {                 // 8 rows x 64 bytes per instruction
             const int row = 8 * k + (lane >> 2), piece = lane & 3;
             const long long orow = __shfl_sync(0xffffffffu, out_row, row);
@@ -507,7 +508,7 @@ __device__ __forceinline__ void store_rows32(const AttnParams& p, float* stage, 
             if (ok) *reinterpret_cast<uint4*>(p.out + orow * kHeadDim + col + piece * 8) = u;
         }
     } else {
-#pragma unroll
+#pragma unroll 2
         for (int k = 0; k < 8; ++k) {                 // 4 rows x 128 bytes per instruction
             const int row = 4 * k + (lane >> 3), piece = lane & 7;
             const bool ok = __shfl_sync(0xffffffffu, row_ok ? 1 : 0, row) != 0;
