@@ -45,8 +45,8 @@
  *                 of sequence b are already stored at logical position L_b + i, so the
  *                 cache holds L_b + n_b valid positions.  Q and K arrive with their
  *                 rotary position (the paper's position-id manipulation) applied.
- *                 Cache slots of a sequence's last page beyond L_b + n_b must hold
- *                 finite values (they are multiplied by an exact zero weight).
+ *                 Cache slots of a sequence's last page beyond L_b + n_b are never
+ *                 visible and may hold anything (uninitialised memory, NaN, Inf).
  *  - node_offsets int32 [B+1], packed offsets of each sequence's nodes; NULL means
  *                 every sequence has N/B nodes.
  *  - tree_parent  int32 [N]: parent of each node as an index local to its sequence,
@@ -69,7 +69,8 @@ typedef enum owl_status {
     OWL_ERR_INVALID_ARG = -1, /* null pointer, batch < 1, total_nodes < 1, Hq % Hkv != 0, ...       */
     OWL_ERR_UNSUPPORTED = -2, /* head_dim != 128, max_nodes > 64, G*max_nodes > 256, page size, ... */
     OWL_ERR_CUDA = -3,        /* a CUDA call failed; see owl_last_error                             */
-    OWL_ERR_BAD_TREE = -4,    /* device-detected: parent[i] >= i, parent < -1, node 0 not the root  */
+    OWL_ERR_BAD_TREE = -4,    /* device-detected: parent[i] >= i, parent < -1, node 0 not the root,
+                                 a sequence with no or too many nodes, inconsistent node_offsets    */
     OWL_ERR_BAD_PAGE = -5,    /* device-detected: block_table entry outside [0, num_pages)          */
     OWL_ERR_TIMEOUT = -6,     /* device-detected: a bounded wait inside a kernel expired            */
     OWL_ERR_TOO_LARGE = -7    /* dims exceed what the context was created for                       */
@@ -159,7 +160,7 @@ int owl_verify_step(owl_ctx* ctx, const owl_dims* dims, const void* q, const voi
 /*
  * One whole verify step from HOST memory: copies every input to device staging buffers owned by
  * the context (grown on demand, so the first call at a given size allocates), runs
- * owl_verify_attn and owl_tree_accept, copies the results back and synchronises `stream`.
+ * owl_verify_step, copies the results back and synchronises `stream`.
  * Every tensor pointer here is a HOST pointer (page-locked memory makes the copies asynchronous
  * and fast; pageable memory works).  Shapes and meanings are those of the two calls above;
  * lse_h may be NULL.  Returns a host-detected error, else the device status word (as
@@ -192,9 +193,9 @@ int owl_verify_step_host(owl_ctx* ctx, const owl_dims* dims, const void* q_h, co
  *
  * Arguments are those of owl_tree_accept (device pointers, caller-owned), without the context, plus
  * device_status: a device int32 the call first clears and the kernels then set to OWL_ERR_BAD_TREE
- * if a tree is malformed (that sequence's outputs stay unwritten).  NULL keeps the status in the
- * library's own array, where nobody can read it.  The work runs on the CURRENT device, on `stream`,
- * asynchronously.
+ * if a tree is malformed (that sequence's outputs stay unwritten) or node_offsets does not describe
+ * total_nodes rows.  With NULL the verdict is dropped: pass a word if malformed input is possible.
+ * The work runs on the CURRENT device, on `stream`, asynchronously.
  *
  * Sharing: all calls on a device use the same array.  Calls queued on one stream are safe one after
  * another (a call overwrites every key before it reads it, so stale contents never matter); calls
@@ -214,6 +215,19 @@ int owl_tree_accept_static(const owl_dims* dims, const float* logits, const int3
  * context since the last owl_get_status (OWL_OK, OWL_ERR_BAD_TREE, OWL_ERR_BAD_PAGE,
  * OWL_ERR_TIMEOUT; the first error wins) and clear it. */
 int owl_get_status(owl_ctx* ctx, void* stream);
+
+/*
+ * Self-test of the kernels' bounded waits.  Every wait inside the kernels (on a TMA arrival, on a
+ * tensor-core commit) gives up after a time limit, raises its CTA's abort flag and reports
+ * OWL_ERR_TIMEOUT instead of hanging the GPU.  This call runs that very wait routine in a
+ * one-warp kernel on a barrier that nothing ever completes, with the limit given here
+ * (1 .. 1e9 ns), then synchronises `stream`.  Returns the device status word and clears it:
+ * OWL_ERR_TIMEOUT is the expected answer.  waited_ns (host, may be NULL) receives the nanoseconds
+ * the first wait took (about limit_ns) and those of a second wait on the same barrier, which
+ * must return at once because the abort flag is up.  Nothing faults or traps; the context stays
+ * usable.
+ */
+int owl_selftest_wait(owl_ctx* ctx, uint64_t limit_ns, uint64_t waited_ns[2], void* stream);
 
 /* Text for a status code; never NULL. */
 const char* owl_status_string(int status);

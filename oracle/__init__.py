@@ -44,6 +44,12 @@ def _load():
         lib.owl_oracle_accept.restype = ctypes.c_int
         lib.owl_oracle_accept.argtypes = [ctypes.c_int, i32p, i32p, i32p, i32p, ctypes.c_int, i32p, i32p, i32p]
         lib.owl_oracle_num_threads.restype = ctypes.c_int
+        lib.owl_oracle_prepare_spec.restype = ctypes.c_int
+        lib.owl_oracle_prepare_spec.argtypes = [ctypes.c_int, i32p, i32p, i32p, i32p, ctypes.c_int32] + [i32p] * 5
+        lib.owl_oracle_spec_leaf.restype = ctypes.c_int
+        lib.owl_oracle_spec_leaf.argtypes = [ctypes.c_int, i32p, i32p, i32p, i32p, i32p, ctypes.c_int, i32p]
+        lib.owl_oracle_kv_commit.restype = ctypes.c_int
+        lib.owl_oracle_kv_commit.argtypes = [ctypes.c_int] * 6 + [u16p, u16p, i32p, i32p, i32p, i32p, i32p, ctypes.c_int]
         _lib = lib
     return _lib
 
@@ -135,3 +141,54 @@ def tree_accept(logits, draft_tokens, node_offsets, tree_parent, path_stride: in
     am = row_argmax(logits)
     alen, path, bonus = accept_from_argmax(node_offsets, tree_parent, draft_tokens, am, path_stride)
     return alen, path, bonus, am
+
+
+def prepare_spec_tree(node_offsets, tree_parent, draft_tokens, ctx_lens, spec_token: int):
+    """Prepare(d): one [SPEC] leaf after every tree path.  Returns (node_offsets, tree_parent, draft_tokens,
+    input_ids, position_ids) of the augmented trees (twice the nodes; leaves carry draft token -1)."""
+    lib = _load()
+    node_offsets = _c(node_offsets, np.int32); tree_parent = _c(tree_parent, np.int32)
+    draft_tokens = _c(draft_tokens, np.int32); ctx_lens = _c(ctx_lens, np.int32)
+    B = node_offsets.shape[0] - 1
+    N = int(node_offsets[-1])
+    offs = np.empty(B + 1, np.int32)
+    par, drf, ids, pos = (np.empty(2 * N, np.int32) for _ in range(4))
+    i32 = ctypes.c_int32
+    rc = lib.owl_oracle_prepare_spec(B, _p(node_offsets, i32), _p(tree_parent, i32), _p(draft_tokens, i32), _p(ctx_lens, i32),
+                                     int(spec_token), _p(offs, i32), _p(par, i32), _p(drf, i32), _p(ids, i32), _p(pos, i32))
+    if rc != 0:
+        raise ValueError(f"owl_oracle_prepare_spec failed with code {rc}")
+    return offs, par, drf, ids, pos
+
+
+def spec_leaf(node_offsets, tree_parent, draft_tokens, accept_len, accept_path) -> np.ndarray:
+    """Index of the [SPEC] leaf hanging off the last accepted node of every sequence (-1 if none)."""
+    lib = _load()
+    node_offsets = _c(node_offsets, np.int32); tree_parent = _c(tree_parent, np.int32)
+    draft_tokens = _c(draft_tokens, np.int32); accept_len = _c(accept_len, np.int32); accept_path = _c(accept_path, np.int32)
+    B = node_offsets.shape[0] - 1
+    out = np.empty(B, np.int32)
+    i32 = ctypes.c_int32
+    rc = lib.owl_oracle_spec_leaf(B, _p(node_offsets, i32), _p(tree_parent, i32), _p(draft_tokens, i32), _p(accept_len, i32),
+                                  _p(accept_path, i32), accept_path.shape[1], _p(out, i32))
+    if rc != 0:
+        raise ValueError(f"owl_oracle_spec_leaf failed with code {rc}")
+    return out
+
+
+def kv_commit(k_cache, v_cache, block_table, ctx_lens, node_offsets, accept_len, accept_path) -> None:
+    """Moves the accepted nodes' K/V from L + path[k] to L + k and adds accept_len to ctx_lens, IN PLACE
+    (k_cache, v_cache: contiguous uint16 [pages, Hkv, page, D]; ctx_lens: contiguous int32 [B])."""
+    lib = _load()
+    for a, dt in ((k_cache, np.uint16), (v_cache, np.uint16), (ctx_lens, np.int32)):
+        assert a.dtype == dt and a.flags["C_CONTIGUOUS"], "in-place arguments must be contiguous arrays of the exact type"
+    block_table = _c(block_table, np.int32); node_offsets = _c(node_offsets, np.int32)
+    accept_len = _c(accept_len, np.int32); accept_path = _c(accept_path, np.int32)
+    num_pages, Hkv, page, D = k_cache.shape
+    B = ctx_lens.shape[0]
+    i32, u16 = ctypes.c_int32, ctypes.c_uint16
+    rc = lib.owl_oracle_kv_commit(B, Hkv, D, page, block_table.shape[1], num_pages, _p(k_cache, u16), _p(v_cache, u16),
+                                  _p(block_table, i32), _p(ctx_lens, i32), _p(node_offsets, i32), _p(accept_len, i32),
+                                  _p(accept_path, i32), accept_path.shape[1])
+    if rc != 0:
+        raise ValueError(f"owl_oracle_kv_commit failed with code {rc}")

@@ -18,14 +18,20 @@
  *    tokens accepted per verification step.  Under greedy decoding a drafted token
  *    keeps the distribution iff it equals the target's own arg-max continuation of
  *    its parent.
- *  - Non-tree verification (Section 3.2.3, Algorithm 1 line 8) is the same pass with
+ *  - Non-tree verification (Section 3.2.3, NonTreeVerify of Algorithm 1) is the same pass with
  *    a chain-shaped tree.
+ *  - Around that pass (Algorithm 1): Prepare(d) appends the [SPEC] leaves and fixes mask and
+ *    position ids; the accepted path names the [SPEC] whose hidden state the drafter gets; the
+ *    accepted tokens are then committed to the cache ("l <- l; d").
  *
  * Parity pins (tests, CPU only): brute-force dense-mask softmax in numpy fp64,
  * single-node == decode attention and chain == causal attention against a library
  * SDPA in fp64, the paper's worked mask example, softmax invariants, hand-worked
  * acceptance cases, losslessness on a toy model, a closed-form expectation, and
- * the acceptance-length bounds the paper states.  No function here is unpinned.
+ * the acceptance-length bounds the paper states; for the steps around the pass the
+ * paper's [SPEC] example extended to leaf indices and position ids, hand-worked
+ * commits on shuffled page tables, the same commit on a gathered logical view, and
+ * the multi-step lossless loop with the cache contents checked.  No function here is unpinned.
  *
  * Arithmetic: bf16 inputs are decoded exactly to double; dot products, the
  * two-pass softmax and the weighted sum run in double; nothing is blocked, fused
@@ -230,6 +236,110 @@ int owl_oracle_accept(int B, const int32_t* node_offsets, const int32_t* tree_pa
         int k = win_depth;
         for (int c = win; c >= 0; c = parent[c]) accept_path[(int64_t)b * path_stride + k--] = c;
         bonus_token[b] = am[base + win];
+    }
+    return ORACLE_OK;
+}
+
+/*
+ * Prepare(d) of Algorithm 1 / Section 3.2.2 "Decode Stage": one [SPEC] token is appended after every
+ * tree path, i.e. every drafted node j (the end of the path root..j) gets one [SPEC] child, "the same
+ * number of [SPEC] as the number of tree nodes", in node order (the paper's example: the first [SPEC]
+ * follows (t_{N+1}), the second (t_{N+1}, t_{N+2}), the third (t_{N+1}, t_{N+2'})).  The attention mask
+ * follows from the parent array; the manipulated position id of a token is the number of context tokens
+ * plus its depth in the tree (a token on a path sits where it would sit if that path were the text).
+ *
+ * In: B trees (node_offsets, tree_parent, draft_tokens; the root's token is t_{N+1}), ctx_lens,
+ * the token id of [SPEC].  Out, for sequence b with n nodes, 2n nodes at out_offsets[b] = 2 * node_offsets[b]:
+ *   nodes 0..n-1   the drafted tree as given; nodes n..2n-1 the [SPEC] leaves, leaf n + j child of j
+ *   out_draft      drafted token, -1 for a [SPEC] leaf (never a candidate of the acceptance)
+ *   out_input_ids  what the verifier embeds: drafted token, spec_token for a leaf
+ *   out_position   ctx_lens[b] + depth
+ */
+int owl_oracle_prepare_spec(int B, const int32_t* node_offsets, const int32_t* tree_parent,
+                            const int32_t* draft_tokens, const int32_t* ctx_lens, int32_t spec_token,
+                            int32_t* out_offsets, int32_t* out_parent, int32_t* out_draft,
+                            int32_t* out_input_ids, int32_t* out_position) {
+    out_offsets[0] = 0;
+    for (int b = 0; b < B; ++b) {
+        const int base = node_offsets[b], n = node_offsets[b + 1] - base;
+        const int32_t* parent = tree_parent + base;
+        if (!tree_ok(parent, n)) return ORACLE_BAD_TREE;
+        const int ob = 2 * base;
+        out_offsets[b + 1] = ob + 2 * n;
+        for (int j = 0; j < n; ++j) {
+            int depth = 0;
+            for (int c = j; parent[c] >= 0; c = parent[c]) ++depth;
+            out_parent[ob + j] = parent[j];
+            out_draft[ob + j] = draft_tokens[base + j];
+            out_input_ids[ob + j] = draft_tokens[base + j];
+            out_position[ob + j] = ctx_lens[b] + depth;
+            out_parent[ob + n + j] = j;                 /* the [SPEC] after the path that ends in j */
+            out_draft[ob + n + j] = -1;
+            out_input_ids[ob + n + j] = spec_token;
+            out_position[ob + n + j] = ctx_lens[b] + depth + 1;
+        }
+    }
+    return ORACLE_OK;
+}
+
+/*
+ * "When a path is accepted, we take the hidden state of the corresponding [SPEC]" (Section 3.2.2, Decode
+ * Stage): the [SPEC] leaf (a child with a negative draft token) of the last node of the accepted path;
+ * the lowest index if there were several, -1 if the node has none (a tree verified without [SPEC]).
+ */
+int owl_oracle_spec_leaf(int B, const int32_t* node_offsets, const int32_t* tree_parent,
+                         const int32_t* draft_tokens, const int32_t* accept_len, const int32_t* accept_path,
+                         int path_stride, int32_t* spec_node) {
+    for (int b = 0; b < B; ++b) {
+        const int base = node_offsets[b], n = node_offsets[b + 1] - base;
+        if (accept_len[b] < 1 || accept_len[b] > path_stride) return ORACLE_BAD_ARG;
+        const int last = accept_path[(int64_t)b * path_stride + accept_len[b] - 1];
+        if (last < 0 || last >= n) return ORACLE_BAD_ARG;
+        spec_node[b] = -1;
+        for (int c = n - 1; c >= 0; --c)
+            if (tree_parent[base + c] == last && draft_tokens[base + c] < 0) spec_node[b] = c;
+    }
+    return ORACLE_OK;
+}
+
+/*
+ * Commit of the accepted tokens to the cache: Algorithm 1, "l <- l; d" and "N <- N + |d|".  During the
+ * verification the K/V of drafted node i sit at logical position L + i.  After it the accepted path
+ * p_0 = 0 < p_1 < ... < p_{a-1} becomes text: the token at L + p_k moves to L + k for every KV head, K and
+ * V alike, everything else that was drafted is dropped, and the committed length grows by a.
+ * All rows are read before any is written (a position may be both a source and a destination).
+ */
+int owl_oracle_kv_commit(int B, int Hkv, int D, int page_size, int max_pages_per_seq, int num_pages,
+                         uint16_t* k_cache, uint16_t* v_cache, const int32_t* block_table, int32_t* ctx_lens,
+                         const int32_t* node_offsets, const int32_t* accept_len, const int32_t* accept_path,
+                         int path_stride) {
+    for (int b = 0; b < B; ++b) {
+        const int n = node_offsets[b + 1] - node_offsets[b];
+        const int a = accept_len[b];
+        const int32_t* path = accept_path + (int64_t)b * path_stride;
+        if (a < 1 || a > n || a > path_stride || path[0] != 0) return ORACLE_BAD_ARG;
+        for (int k = 1; k < a; ++k)
+            if (path[k] <= path[k - 1] || path[k] >= n) return ORACLE_BAD_ARG;
+        const int64_t L = ctx_lens[b];
+        uint16_t* tmp = (uint16_t*)malloc((size_t)2 * a * Hkv * D * sizeof(uint16_t));
+        for (int k = 0; k < a; ++k)
+            for (int h = 0; h < Hkv; ++h) {
+                const uint16_t* ks = kv_row(k_cache, block_table, b, max_pages_per_seq, num_pages, Hkv, page_size, D, h, L + path[k]);
+                const uint16_t* vs = kv_row(v_cache, block_table, b, max_pages_per_seq, num_pages, Hkv, page_size, D, h, L + path[k]);
+                if (!ks || !vs) { free(tmp); return ORACLE_BAD_PAGE; }
+                memcpy(tmp + ((size_t)(2 * k) * Hkv + h) * D, ks, (size_t)D * sizeof(uint16_t));
+                memcpy(tmp + ((size_t)(2 * k + 1) * Hkv + h) * D, vs, (size_t)D * sizeof(uint16_t));
+            }
+        for (int k = 0; k < a; ++k)
+            for (int h = 0; h < Hkv; ++h) {
+                uint16_t* kd = (uint16_t*)kv_row(k_cache, block_table, b, max_pages_per_seq, num_pages, Hkv, page_size, D, h, L + k);
+                uint16_t* vd = (uint16_t*)kv_row(v_cache, block_table, b, max_pages_per_seq, num_pages, Hkv, page_size, D, h, L + k);
+                if (!kd || !vd) { free(tmp); return ORACLE_BAD_PAGE; }
+                memcpy(kd, tmp + ((size_t)(2 * k) * Hkv + h) * D, (size_t)D * sizeof(uint16_t));
+                memcpy(vd, tmp + ((size_t)(2 * k + 1) * Hkv + h) * D, (size_t)D * sizeof(uint16_t));
+            }
+        free(tmp);
+        ctx_lens[b] = (int32_t)(L + a);
     }
     return ORACLE_OK;
 }

@@ -58,6 +58,8 @@ def load_library() -> ctypes.CDLL:
     lib.owl_verify_step_host.argtypes = [vp, dp] + [vp] * 15
     lib.owl_get_status.restype = i32
     lib.owl_get_status.argtypes = [vp, vp]
+    lib.owl_selftest_wait.restype = i32
+    lib.owl_selftest_wait.argtypes = [vp, ctypes.c_uint64, ctypes.POINTER(ctypes.c_uint64), vp]
     lib.owl_status_string.restype = ctypes.c_char_p
     lib.owl_status_string.argtypes = [i32]
     lib.owl_last_error.restype = ctypes.c_char_p
@@ -173,6 +175,13 @@ class OwlContext:
 
     def owl_get_status(self) -> int:
         return int(self.lib.owl_get_status(self._h, _stream(self.device)))
+
+    def owl_selftest_wait(self, limit_ns: int):
+        """Runs the kernels' bounded wait on a barrier nothing completes; returns (status, ns of the first wait,
+        ns of the second wait)."""
+        ns = (ctypes.c_uint64 * 2)()
+        rc = int(self.lib.owl_selftest_wait(self._h, ctypes.c_uint64(limit_ns), ns, _stream(self.device)))
+        return rc, int(ns[0]), int(ns[1])
 
     def last_error(self) -> str:
         return self.lib.owl_last_error(self._h).decode()

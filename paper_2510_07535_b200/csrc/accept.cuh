@@ -12,7 +12,7 @@
 // the chunk keys to arg-max tokens, evaluates for every node whether all edges on its root path match
 // (draft token == parent's arg-max), picks the deepest matching node (lowest index among equals) and
 // writes accept_len / accept_path / bonus_token.  Calls alternate between two sets of counters and clear the
-// idle one, so no separate clearing pass is needed.
+// idle one as a whole, so no separate clearing pass is needed.
 //
 // Inside a verify step with a small scan both halves run as guests of the attention kernels: the scan in warps
 // the attention pass does not use (argmax_scan_chunk_warp), the walk in extra CTAs of the merge kernel, after
@@ -26,6 +26,21 @@ namespace owl {
 constexpr int kArgmaxThreads = 256;
 static_assert(kArgmaxThreads >= kMaxNodes, "the walk needs one thread per node");
 constexpr int kArgmaxChunk = 8192;  // floats per CTA: 8 x float4 per thread
+static_assert(kArgmaxChunk == 8 * 4 * kArgmaxThreads, "argmax_partial_kernel reads its chunk in one round of 8 loads");
+
+// 16-byte load of data that is read once: no L1 allocation, first in line for eviction from L2
+// (`policy` from createpolicy.fractional.L2::evict_first).
+__device__ __forceinline__ uint64_t l2_evict_first_policy() {
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+__device__ __forceinline__ float4 ld_stream_f4(const float4* ptr, uint64_t policy) {
+    float4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.L2::cache_hint.v4.f32 {%0, %1, %2, %3}, [%4], %5;"
+                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(ptr), "l"(policy));
+    return v;
+}
 
 struct AcceptParams {
     const float* logits;
@@ -172,6 +187,22 @@ __global__ void __launch_bounds__(kArgmaxThreads) argmax_partial_kernel(const Ac
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next kernel may queue up; it waits likewise
     const int row = blockIdx.y;
+    if (blockIdx.x == 0 && blockIdx.y == 0) {
+        // Once per call: clear every counter of the idle set (the next call counts there, whatever its batch), and
+        // check that the packed offsets describe this call's rows: start at 0, end at total_nodes, 1..max_nodes
+        // nodes per sequence.  With inconsistent offsets a row would count for the wrong sequence and a walk could
+        // run on keys not yet stored; the status word says so (that call's outputs are then meaningless).
+        unsigned int* idle = p.seq_counter + (size_t)((p.epoch + 1u) & 1u) * p.counter_stride;
+        for (int b = threadIdx.x; b < p.counter_stride; b += kArgmaxThreads) idle[b] = 0u;
+        if (p.node_offsets) {
+            bool bad = false;
+            for (int b = threadIdx.x; b < p.batch; b += kArgmaxThreads) {
+                const int lo = p.node_offsets[b], n = p.node_offsets[b + 1] - lo;
+                bad = bad || n < 1 || n > p.max_nodes || (b == 0 && lo != 0) || (b == p.batch - 1 && lo + n != p.total_nodes);
+            }
+            if (bad) report(p.status, kErrBadTree);
+        }
+    }
     const long long V = p.vocab;
     const long long c0 = (long long)blockIdx.x * kArgmaxChunk;
     const long long c1 = c0 + kArgmaxChunk < V ? c0 + kArgmaxChunk : V;
@@ -188,16 +219,31 @@ __global__ void __launch_bounds__(kArgmaxThreads) argmax_partial_kernel(const Ac
     unsigned long long key = 0;
     const float4* body = reinterpret_cast<const float4*>(base + a0);
     const int nvec = (int)((a1 - a0) >> 2);
-    for (int v = threadIdx.x; v < nvec; v += kArgmaxThreads) {
-        const float4 x = __ldg(body + v);
-        const uint32_t i0 = (uint32_t)(a0 + 4ll * v);
-        // NaN reads as -inf; strict '>' keeps the first maximum (indices grow along this thread's walk)
-        const float e0 = x.x != x.x ? -INFINITY : x.x, e1 = x.y != x.y ? -INFINITY : x.y;
-        const float e2 = x.z != x.z ? -INFINITY : x.z, e3 = x.w != x.w ? -INFINITY : x.w;
-        if (bi == 0xffffffffu || e0 > bv) { bv = e0; bi = i0; }
-        if (e1 > bv) { bv = e1; bi = i0 + 1; }
-        if (e2 > bv) { bv = e2; bi = i0 + 2; }
-        if (e3 > bv) { bv = e3; bi = i0 + 3; }
+    // A chunk is 8 x 16 bytes per thread: all eight loads are issued before the first compare, so that a CTA has its
+    // whole 32 KB in flight at once (one load per iteration left the scan at about half of the memory bandwidth).
+    // The logits are read once: they bypass L1 and are the first to leave L2.
+    {
+        const uint64_t policy = l2_evict_first_policy();
+        float4 x[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int v = j * kArgmaxThreads + (int)threadIdx.x;
+            x[j] = v < nvec ? ld_stream_f4(body + v, policy) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int v = j * kArgmaxThreads + (int)threadIdx.x;
+            if (v < nvec) {
+                const uint32_t i0 = (uint32_t)(a0 + 4ll * v);
+                // NaN reads as -inf; strict '>' keeps the first maximum (indices grow along this thread's walk)
+                const float e0 = x[j].x != x[j].x ? -INFINITY : x[j].x, e1 = x[j].y != x[j].y ? -INFINITY : x[j].y;
+                const float e2 = x[j].z != x[j].z ? -INFINITY : x[j].z, e3 = x[j].w != x[j].w ? -INFINITY : x[j].w;
+                if (bi == 0xffffffffu || e0 > bv) { bv = e0; bi = i0; }
+                if (e1 > bv) { bv = e1; bi = i0 + 1; }
+                if (e2 > bv) { bv = e2; bi = i0 + 2; }
+                if (e3 > bv) { bv = e3; bi = i0 + 3; }
+            }
+        }
     }
     if (bi != 0xffffffffu) key = argmax_key(bv, bi);
     // ragged ends: at most 3 + 3 elements per chunk
@@ -234,10 +280,10 @@ __global__ void __launch_bounds__(kArgmaxThreads) argmax_partial_kernel(const Ac
             n_b = p.nodes_uniform;
         }
         __threadfence();
-        // two sets of counters: this call counts in set (epoch & 1) and clears the other one for the next call,
-        // so a counter left dirty by malformed input never survives
+        // two sets of counters: this call counts in set (epoch & 1); the other one is cleared as a whole (above)
+        // for the next call, so a counter left dirty by malformed input is gone two calls later at the latest and
+        // is never counted in
         unsigned int* ctr = p.seq_counter + (size_t)(p.epoch & 1u) * p.counter_stride + b;
-        p.seq_counter[(size_t)((p.epoch + 1u) & 1u) * p.counter_stride + b] = 0u;
         const unsigned int want = atomicAdd(ctr, 1u) + 1u;
         if ((long long)want == (long long)p.chunks * n_b) *ctr = 0u;   // a completed counter is left clean as well
         s_walk_b = ((long long)want == (long long)p.chunks * n_b) ? b : -1;

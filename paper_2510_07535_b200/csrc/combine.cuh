@@ -10,71 +10,7 @@ namespace owl {
 
 constexpr int kCombineWarps = 8;
 
-template <int TileKeys, int RowsPerBlock>
-__global__ void __launch_bounds__(kCombineWarps * 32) combine_kernel(const AttnParams p) {
-    __shared__ long long s_tile[kMaxBatch + 1];
-    __shared__ int s_unit[kMaxBatch + 1];
-    build_schedule<TileKeys, RowsPerBlock>(p, s_tile, s_unit);
-    Partition part;
-    part.init(s_tile[p.batch], p.num_ctas);
-
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const long long row_id = (long long)blockIdx.x * kCombineWarps + warp;
-    if (row_id >= (long long)p.total_nodes * p.num_q_heads) return;
-    const int n = (int)(row_id / p.num_q_heads), hq = (int)(row_id % p.num_q_heads);
-
-    int b;
-    if (p.node_offsets) {
-        int lo = 0, hi = p.batch;  // largest b with node_offsets[b] <= n
-        while (hi - lo > 1) { int mid = (lo + hi) >> 1; if (p.node_offsets[mid] <= n) lo = mid; else hi = mid; }
-        b = lo;
-    } else {
-        b = n / p.nodes_uniform;
-    }
-    if (p.seq_bad[b] == p.epoch || s_unit[b + 1] == s_unit[b]) return;
-
-    const SeqSched s = seq_sched<TileKeys, RowsPerBlock>(p, s_tile, s_unit, b);
-    const int G = p.group;
-    const int r = (n - s.node_base) * G + hq % G;
-    const int ul = (hq / G) * s.row_blocks + r / RowsPerBlock;
-    const int lrow = r % RowsPerBlock;
-    const int unit = s.unit_begin + ul;
-    const long long t0 = s.tile_begin + (long long)ul * s.tiles;
-    const int c0 = part.owner(t0), c1 = part.owner(t0 + s.tiles - 1);
-    if (c0 == c1) return;  // a single CTA saw every key of this unit and wrote the result itself
-
-    auto slot_of = [&](int c) -> long long {
-        return (long long)c + unit;   // the partial of (CTA c, unit u) sits in slot c + u
-    };
-    float mx = -INFINITY;
-    for (int c = c0 + lane; c <= c1; c += 32)
-        mx = fmaxf(mx, p.part_lse[slot_of(c) * p.rows_per_slot + lrow]);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    float sum = 0.f;
-    if (mx > -INFINITY) {
-        for (int c = c0; c <= c1; ++c) {
-            const long long prow = slot_of(c) * p.rows_per_slot + lrow;
-            const float w = __expf(p.part_lse[prow] - mx);
-            const float4 v = *reinterpret_cast<const float4*>(p.part_o + prow * kHeadDim + lane * 4);
-            acc.x += w * v.x; acc.y += w * v.y; acc.z += w * v.z; acc.w += w * v.w;
-            sum += w;
-        }
-    }
-    const float inv = sum > 0.f ? 1.f / sum : 0.f;
-    __nv_bfloat162 lo2 = __floats2bfloat162_rn(acc.x * inv, acc.y * inv);
-    __nv_bfloat162 hi2 = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
-    uint2 pk;
-    pk.x = *reinterpret_cast<uint32_t*>(&lo2);
-    pk.y = *reinterpret_cast<uint32_t*>(&hi2);
-    *reinterpret_cast<uint2*>(p.out + row_id * kHeadDim + lane * 4) = pk;
-    if (p.lse && lane == 0) p.lse[row_id] = sum > 0.f ? mx + logf(sum) : -INFINITY;
-}
-
-
-// LSE merge for the tcgen05 split-KV pass: one warp per output row finds the CTAs whose pieces cut the row's unit
+// One warp per output row finds the CTAs whose pieces cut the row's unit
 // and merges their partials in CTA order.  A CTA stores at most two partials: slot 2c if its piece starts inside
 // the unit, else 2c + 1.
 //

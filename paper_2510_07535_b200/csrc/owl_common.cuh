@@ -35,8 +35,8 @@ struct AttnParams {
     float* part_lse;              // [slots, rows_per_slot] fp32, natural-log partial LSE (-inf if empty)
     int32_t* status;              // device status word (0 = ok, first error wins)
     int32_t* seq_bad;             // [B] epoch of the call in which the sequence was found malformed
-    long long* sched_seq_begin;   // [B + 1] first flat tile of every sequence (tcgen05 path; written by its CTA 0)
-    SchedHeader* sched_header;    // (tcgen05 path)
+    long long* sched_seq_begin;   // [B + 1] first flat tile of every sequence (written by CTA 0 of the pass)
+    SchedHeader* sched_header;
     int32_t epoch;
     int32_t batch, total_nodes, nodes_uniform, max_nodes;
     int32_t num_q_heads, num_kv_heads, group;  // group = Hq / Hkv
@@ -58,21 +58,12 @@ __device__ __forceinline__ void report(int32_t* status, int code) { atomicCAS(st
 // ---------------------------------------------------------------------------------------------
 // Flat partition of the split-KV pass.
 //
-// A unit is (sequence b, KV head h, row block mb); it owns tiles_b = ceil((L_b + n_b) / TileKeys)
-// key tiles.  Units are laid out sequence-major, then head, then row block; all their tiles form
-// one flat range [0, total) which is cut into num_ctas contiguous, nearly equal pieces.  A CTA's
-// piece may start and end inside a unit; each (CTA, unit) intersection yields one partial
-// (o, lse) stored in slot cta + unit, which is unique because pieces and units are both ordered.
+// A unit is (sequence b, KV head h) with all its G * n_b packed rows; it owns
+// tiles_b = ceil((L_b + n_b) / TileKeys) key tiles.  Units are laid out sequence-major, then head;
+// all their tiles form one flat range [0, total) which is cut into num_ctas contiguous pieces.  A
+// CTA's piece may start and end inside a unit; only its first and its last unit can be cut, so a
+// CTA stores at most two partials (o, lse): slot 2c for the unit its piece starts in, 2c + 1 for a later one.
 // ---------------------------------------------------------------------------------------------
-struct SeqSched {
-    long long tile_begin;  // first flat tile of the sequence
-    int unit_begin;        // first unit of the sequence
-    int tiles;             // key tiles per unit
-    int row_blocks;        // row blocks per (sequence, head)
-    int n, L;              // drafted nodes, committed context length
-    int node_base;
-};
-
 // Cut of the flat tile range [0, total) into `ctas` pieces, one per CTA.
 //   flat:    contiguous, nearly equal pieces; a piece may start and end inside a unit.
 //   aligned: only when every unit has the same number of tiles (`unit_tiles`) and there are at least as
@@ -175,7 +166,7 @@ __device__ __forceinline__ bool seq_shape_ok(const AttnParams& p, int b, int n, 
 // Schedule of a batch of at most 32 sequences, derived by one warp on its own: lane b holds sequence b, prefix sums
 // by shuffle, no shared memory.  The split-KV pass (every warp of it) and the merge that follows it call the same
 // function on the same inputs, so the merge needs nothing from the pass but its partials.
-constexpr int kSchedTileKeys = 128;      // key tile of the tcgen05 split-KV pass
+constexpr int kSchedTileKeys = 128;      // key tile of the split-KV pass
 struct WarpSchedule {
     int n, L, node_base, tiles;          // this lane's sequence (tiles = 0 if it is not schedulable)
     bool ok;
@@ -222,70 +213,6 @@ __device__ __forceinline__ WarpSchedule warp_schedule(const AttnParams& p) {
     ws.excl_t = inc_t - ws.my_tiles;
     ws.excl_u = inc_u - ws.my_units;
     return ws;
-}
-
-// Every CTA derives the same per-sequence schedule into shared memory.
-// s_tile[b], s_unit[b] are exclusive prefix sums; entries [batch] hold the totals.
-template <int TileKeys, int RowsPerBlock>
-__device__ void build_schedule(const AttnParams& p, long long* s_tile, int* s_unit) {
-    // serial prefix by one thread per 32 sequences would be overkill: batch is at most 1024 and
-    // this runs once per CTA; thread 0 walks it after all threads staged the per-sequence counts.
-    for (int b = threadIdx.x; b < p.batch; b += blockDim.x) {
-        int n = seq_nodes(p, b), L = p.ctx_lens[b];
-        int units = 0, tiles = 0;
-        if (seq_shape_ok(p, b, n, L)) {
-            tiles = (L + n + TileKeys - 1) / TileKeys;
-            units = p.num_kv_heads * ((n * p.group + RowsPerBlock - 1) / RowsPerBlock);
-        } else {
-            report(p.status, seq_tree_shape_ok(p, b, n) ? kErrBadPage : kErrBadTree);
-            p.seq_bad[b] = p.epoch;
-        }
-        s_tile[b + 1] = (long long)tiles * units;
-        s_unit[b + 1] = units;
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        s_tile[0] = 0; s_unit[0] = 0;
-        for (int b = 0; b < p.batch; ++b) { s_tile[b + 1] += s_tile[b]; s_unit[b + 1] += s_unit[b]; }
-    }
-    __syncthreads();
-}
-
-template <int TileKeys, int RowsPerBlock>
-__device__ __forceinline__ SeqSched seq_sched(const AttnParams& p, const long long* s_tile, const int* s_unit, int b) {
-    SeqSched s;
-    s.tile_begin = s_tile[b];
-    s.unit_begin = s_unit[b];
-    s.n = seq_nodes(p, b);
-    s.L = p.ctx_lens[b];
-    s.node_base = seq_node_base(p, b);
-    s.tiles = (s.L + s.n + TileKeys - 1) / TileKeys;
-    s.row_blocks = (s.n * p.group + RowsPerBlock - 1) / RowsPerBlock;
-    return s;
-}
-
-// Ancestor-or-self bitmasks of one sequence's tree: bit j of anc[i] is set iff node j lies on the
-// root path of node i (Section 3.2.2 "Decode Stage": a token sees exactly its own tree path).
-// Returns false (and writes nothing useful) if the tree violates parent[i] < i / single root.
-__device__ __forceinline__ bool build_ancestors(const int32_t* parent, int n, unsigned long long* anc /*smem[64]*/,
-                                                int* s_flag /*smem*/) {
-    if (threadIdx.x == 0) *s_flag = 0;
-    __syncthreads();
-    if (threadIdx.x < n) {
-        int i = threadIdx.x;
-        int pi = parent[i];
-        if ((i == 0 && pi != -1) || (i > 0 && (pi < 0 || pi >= i))) atomicExch(s_flag, 1);
-    }
-    __syncthreads();
-    bool ok = (*s_flag == 0);
-    if (ok && threadIdx.x < n) {
-        int i = threadIdx.x;
-        unsigned long long m = 0;
-        for (int j = i, guard = 0; j >= 0 && guard < kMaxNodes; j = parent[j], ++guard) m |= 1ull << j;
-        anc[i] = m;
-    }
-    __syncthreads();
-    return ok;
 }
 
 }  // namespace owl

@@ -6,17 +6,17 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
-#include <atomic>
 #include <mutex>
 #include <new>
 
 #include "accept.cuh"
 #include "combine.cuh"
 #include "owl_common.cuh"
-#include "verify_attn_mma.cuh"
 #include "verify_attn_umma.cuh"
 
 using namespace owl;
+
+constexpr int kMapCacheEntries = 8;
 
 struct owl_ctx {
     int device = 0;
@@ -28,6 +28,7 @@ struct owl_ctx {
     float* part_o = nullptr;
     float* part_lse = nullptr;
     int32_t* status = nullptr;
+    unsigned long long* selftest_ns = nullptr;
     int32_t* seq_bad = nullptr;
     long long* sched_seq_begin = nullptr;
     SchedHeader* sched_header = nullptr;
@@ -35,13 +36,17 @@ struct owl_ctx {
     unsigned int* seq_counter = nullptr;
     uint32_t accept_epoch = 0;
     long long part_keys_len = 0;
-    // tcgen05 path: tensor maps over the caller's K and V caches, re-encoded when the cache changes
-    bool use_umma = true;
+    // tensor maps over the callers' K and V caches: a few most recently used (cache pointers, geometry) pairs
+    // are kept, so that a caller rotating over several caches does not pay two encodes per call
     EncodeTiledFn encode = nullptr;
-    CUtensorMap kmap{}, vmap{};
-    const void* map_k = nullptr;
-    const void* map_v = nullptr;
-    int map_pages = 0, map_heads = 0, map_page_size = 0;
+    struct MapEntry {
+        CUtensorMap kmap{}, vmap{};
+        const void* k = nullptr;
+        const void* v = nullptr;
+        int pages = 0, heads = 0, page_size = 0;
+        uint64_t used = 0;
+    } maps[kMapCacheEntries];
+    uint64_t map_clock = 0;
     int32_t epoch = 0;
     int64_t launches = 0;
     bool profiling = false;
@@ -131,6 +136,30 @@ int check_dims(const owl_dims* d, bool for_attn, bool for_accept) {
     return OWL_OK;
 }
 
+// One warp waits, with the kernels' own bounded wait, on an mbarrier that nothing ever completes.  The wait must
+// give up after `limit_ns`, raise the abort flag (so that a second wait returns at once) and report kErrTimeout;
+// the kernel then ends normally.  res[0]: nanoseconds the first wait took, res[1]: those of the second.
+__global__ void selftest_wait_kernel(int32_t* status, unsigned long long limit_ns, unsigned long long* res) {
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        sm100::mbar_init(sm100::smem_u32(&bar), 1);
+        abort_flag = 0;
+        sm100::fence_barrier_init();
+    }
+    __syncthreads();
+    const uint64_t t0 = sm100::global_timer_ns();
+    const bool first = sm100::mbar_wait_ns(sm100::smem_u32(&bar), 0u, &abort_flag, limit_ns);
+    const uint64_t t1 = sm100::global_timer_ns();
+    const bool second = sm100::mbar_wait_ns(sm100::smem_u32(&bar), 0u, &abort_flag, limit_ns);
+    const uint64_t t2 = sm100::global_timer_ns();
+    if (threadIdx.x == 0) {
+        if (!first && !second && abort_flag) report(status, kErrTimeout);
+        res[0] = t1 - t0;
+        res[1] = t2 - t1;
+    }
+}
+
 }  // namespace
 
 extern "C" {
@@ -174,9 +203,7 @@ int owl_create(owl_ctx** out, int device, const owl_dims* max_dims) {
     ctx->sm_count = prop.multiProcessorCount;
     ctx->num_ctas = ctx->sm_count;
 
-    const char* path_env = getenv("OWL_ATTN_PATH");     // "mma" selects the warp-level MMA kernel (for comparison)
-    ctx->use_umma = !(path_env && strcmp(path_env, "mma") == 0);
-    if (ctx->use_umma && attn) {
+    if (attn) {
         ctx->encode = load_encode_tiled();
         if (!ctx->encode) { delete ctx; return OWL_ERR_CUDA; }
     }
@@ -186,20 +213,13 @@ int owl_create(owl_ctx** out, int device, const owl_dims* max_dims) {
         if (ok && (e = cudaMalloc(p, bytes ? bytes : 16)) != cudaSuccess) ok = false;
     };
     if (attn) {
-        const int G = max_dims->num_q_heads / max_dims->num_kv_heads;
-        const int M = G * max_dims->max_nodes;
-        const int row_blocks = (M + mma_path::kRows - 1) / mma_path::kRows;
-        if (ctx->use_umma) {
-            ctx->rows_per_slot = umma_path::kRows;
-            ctx->slots = 2ll * ctx->num_ctas;      // a CTA stores at most two partials per call
-        } else {
-            ctx->rows_per_slot = mma_path::kRows;
-            ctx->slots = (long long)ctx->num_ctas + (long long)max_dims->batch * max_dims->num_kv_heads * row_blocks;
-        }
+        ctx->rows_per_slot = umma_path::kRows;
+        ctx->slots = 2ll * ctx->num_ctas;      // a CTA stores at most two partials per call
         alloc((void**)&ctx->part_o, (size_t)ctx->slots * ctx->rows_per_slot * kHeadDim * sizeof(float));
         alloc((void**)&ctx->part_lse, (size_t)ctx->slots * ctx->rows_per_slot * sizeof(float));
     }
     alloc((void**)&ctx->status, sizeof(int32_t));
+    alloc((void**)&ctx->selftest_ns, 2 * sizeof(unsigned long long));
     alloc((void**)&ctx->seq_bad, (size_t)max_dims->batch * sizeof(int32_t));
     alloc((void**)&ctx->sched_seq_begin, ((size_t)max_dims->batch + 1) * sizeof(long long));
     alloc((void**)&ctx->sched_header, sizeof(SchedHeader));
@@ -215,9 +235,7 @@ int owl_create(owl_ctx** out, int device, const owl_dims* max_dims) {
     }
     for (int i = 0; ok && i < 6; ++i) ok = cudaEventCreate(&ctx->ev[i]) == cudaSuccess;
     if (ok && attn) {
-        ok = cudaFuncSetAttribute(mma_path::verify_attn_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                  mma_path::kSmemBytes) == cudaSuccess &&
-             set_umma_smem_attr();
+        ok = set_umma_smem_attr();
     }
     if (!ok || cudaDeviceSynchronize() != cudaSuccess) {
         cudaGetLastError();
@@ -234,6 +252,7 @@ int owl_destroy(owl_ctx* ctx) {
     cudaFree(ctx->part_o);
     cudaFree(ctx->part_lse);
     cudaFree(ctx->status);
+    cudaFree(ctx->selftest_ns);
     cudaFree(ctx->seq_bad);
     cudaFree(ctx->sched_seq_begin);
     cudaFree(ctx->sched_header);
@@ -246,7 +265,7 @@ int owl_destroy(owl_ctx* ctx) {
     return OWL_OK;
 }
 
-// Attention of a verify step.  `ap` non-null (tcgen05 path only): the logits scan rides in the attention kernel's
+// Attention of a verify step.  `ap` non-null: the logits scan rides in the attention kernel's
 // spare warps and the acceptance walk in the merge kernel, two launches for the whole step.
 static int verify_attn_impl(owl_ctx* ctx, const owl_dims* d, const void* q, const void* k_cache, const void* v_cache,
                             const int32_t* block_table, const int32_t* ctx_lens, const int32_t* node_offsets,
@@ -259,10 +278,7 @@ static int verify_attn_impl(owl_ctx* ctx, const owl_dims* d, const void* q, cons
     if (!ctx->part_o) return OWL_ERR_TOO_LARGE;
     const owl_dims& mx = ctx->max_dims;
     const int G = d->num_q_heads / d->num_kv_heads;
-    const int row_blocks = (G * d->max_nodes + mma_path::kRows - 1) / mma_path::kRows;
-    if (d->batch > mx.batch || d->total_nodes > mx.total_nodes ||
-        (!ctx->use_umma && (long long)ctx->num_ctas + (long long)d->batch * d->num_kv_heads * row_blocks > ctx->slots))
-        return OWL_ERR_TOO_LARGE;
+    if (d->batch > mx.batch || d->total_nodes > mx.total_nodes) return OWL_ERR_TOO_LARGE;
 
     DeviceGuard guard(ctx->device);
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
@@ -298,54 +314,58 @@ static int verify_attn_impl(owl_ctx* ctx, const owl_dims* d, const void* q, cons
     p.num_ctas = ctx->num_ctas;
     p.sm_scale = d->sm_scale;
 
-    if (ctx->use_umma && (ctx->map_k != k_cache || ctx->map_v != v_cache || ctx->map_pages != d->num_pages ||
-                          ctx->map_heads != d->num_kv_heads || ctx->map_page_size != d->page_size)) {
-        const int rk = make_kv_tensor_map(ctx->encode, &ctx->kmap, k_cache, d->num_pages, d->num_kv_heads, d->page_size);
-        const int rv = make_kv_tensor_map(ctx->encode, &ctx->vmap, v_cache, d->num_pages, d->num_kv_heads, d->page_size);
-        if (rk != 0 || rv != 0) {
-            ctx->map_k = ctx->map_v = nullptr;
-            snprintf(ctx->err, sizeof ctx->err, "cuTensorMapEncodeTiled failed (%d, %d): caches must be 16-byte aligned", rk, rv);
-            return OWL_ERR_CUDA;
+    owl_ctx::MapEntry* maps = nullptr;
+    {
+        owl_ctx::MapEntry* lru = &ctx->maps[0];
+        for (auto& m : ctx->maps) {
+            if (m.k == k_cache && m.v == v_cache && m.pages == d->num_pages && m.heads == d->num_kv_heads &&
+                m.page_size == d->page_size) { maps = &m; break; }
+            if (m.used < lru->used) lru = &m;
         }
-        ctx->map_k = k_cache; ctx->map_v = v_cache;
-        ctx->map_pages = d->num_pages; ctx->map_heads = d->num_kv_heads; ctx->map_page_size = d->page_size;
+        if (!maps) {
+            const int rk = make_kv_tensor_map(ctx->encode, &lru->kmap, k_cache, d->num_pages, d->num_kv_heads, d->page_size);
+            const int rv = make_kv_tensor_map(ctx->encode, &lru->vmap, v_cache, d->num_pages, d->num_kv_heads, d->page_size);
+            if (rk != 0 || rv != 0) {
+                lru->k = lru->v = nullptr;
+                lru->used = 0;
+                snprintf(ctx->err, sizeof ctx->err, "cuTensorMapEncodeTiled failed (%d, %d): caches must be 16-byte aligned", rk, rv);
+                return OWL_ERR_CUDA;
+            }
+            lru->k = k_cache; lru->v = v_cache;
+            lru->pages = d->num_pages; lru->heads = d->num_kv_heads; lru->page_size = d->page_size;
+            maps = lru;
+        }
+        maps->used = ++ctx->map_clock;
     }
 
     if (ctx->profiling) cudaEventRecord(ctx->ev[0], stream);
     const long long rows = (long long)d->total_nodes * d->num_q_heads;
     const unsigned grid = (unsigned)((rows + kCombineWarps - 1) / kCombineWarps);
-    if (ctx->use_umma) {
-        {
-            cudaLaunchConfig_t cfg = {};
-            cfg.gridDim = dim3(ctx->num_ctas);
-            cfg.blockDim = dim3(umma_path::kThreads);
-            cfg.dynamicSmemBytes = umma_path::kSmemBytes;
-            cfg.stream = stream;
-            cudaLaunchAttribute attr[1];
-            attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-            attr[0].val.programmaticStreamSerializationAllowed = 1;
-            cfg.attrs = attr;
-            cfg.numAttrs = 1;
-            // the instance that holds only this call's case: block-wide schedule above 32 sequences, the two-row-block
-            // mode only if a unit (G * max_nodes rows at most) can exceed 128 rows, the logits scan only in a step
-            const bool many = d->batch > 32, wide = G * d->max_nodes > 128;
-            cudaLaunchKernelEx(&cfg, umma_kernel(many, wide, ap != nullptr), p, ctx->kmap, ctx->vmap, ap ? *ap : AcceptParams{});
-        }
-        ++ctx->launches;
-        if (ctx->profiling) cudaEventRecord(ctx->ev[1], stream);
-        const bool few_rows = rows <= 4096;      // latency-bound merge: 32 partials per round (see combine.cuh)
-        if (ap)
-            launch_dependent(few_rows ? combine_sched_kernel<true, 32> : combine_sched_kernel<true, 16>,
-                             dim3(grid + (unsigned)d->batch), dim3(kCombineWarps * 32), stream, p, *ap);
-        else
-            launch_dependent(few_rows ? combine_sched_kernel<false, 32> : combine_sched_kernel<false, 16>, dim3(grid),
-                             dim3(kCombineWarps * 32), stream, p, AcceptParams{});
-    } else {
-        mma_path::verify_attn_mma_kernel<<<ctx->num_ctas, mma_path::kThreads, mma_path::kSmemBytes, stream>>>(p);
-        ++ctx->launches;
-        if (ctx->profiling) cudaEventRecord(ctx->ev[1], stream);
-        combine_kernel<mma_path::kTileKeys, mma_path::kRows><<<grid, kCombineWarps * 32, 0, stream>>>(p);
+    {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(ctx->num_ctas);
+        cfg.blockDim = dim3(umma_path::kThreads);
+        cfg.dynamicSmemBytes = umma_path::kSmemBytes;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        // the instance that holds only this call's case: block-wide schedule above 32 sequences, the two-row-block
+        // mode only if a unit (G * max_nodes rows at most) can exceed 128 rows, the logits scan only in a step
+        const bool many = d->batch > 32, wide = G * d->max_nodes > 128;
+        cudaLaunchKernelEx(&cfg, umma_kernel(many, wide, ap != nullptr), p, maps->kmap, maps->vmap, ap ? *ap : AcceptParams{});
     }
+    ++ctx->launches;
+    if (ctx->profiling) cudaEventRecord(ctx->ev[1], stream);
+    const bool few_rows = rows <= 4096;      // latency-bound merge: 32 partials per round (see combine.cuh)
+    if (ap)
+        launch_dependent(few_rows ? combine_sched_kernel<true, 32> : combine_sched_kernel<true, 16>,
+                         dim3(grid + (unsigned)d->batch), dim3(kCombineWarps * 32), stream, p, *ap);
+    else
+        launch_dependent(few_rows ? combine_sched_kernel<false, 32> : combine_sched_kernel<false, 16>, dim3(grid),
+                         dim3(kCombineWarps * 32), stream, p, AcceptParams{});
     ++ctx->launches;
     if (ctx->profiling) { cudaEventRecord(ctx->ev[2], stream); ctx->ev_attn_valid = true; }
     cudaError_t e = cudaGetLastError();
@@ -429,7 +449,7 @@ int owl_verify_step(owl_ctx* ctx, const owl_dims* d, const void* q, const void* 
     // a larger one slows the attention down by more than its own kernel costs (measured: 4 x 64 nodes of a 128K
     // vocabulary, 570 -> 605 us), so it follows as a kernel of its own in stream order.
     const long long scan_items = (long long)d->total_nodes * ((d->vocab + kArgmaxChunk - 1) / kArgmaxChunk);
-    if (!ctx->use_umma || scan_items > 1024) {
+    if (scan_items > 1024) {
         rc = owl_verify_attn(ctx, d, q, k_cache, v_cache, block_table, ctx_lens, node_offsets, tree_parent, out, lse, stream_);
         if (rc != OWL_OK) return rc;
         return owl_tree_accept(ctx, d, logits, draft_tokens, node_offsets, tree_parent, accept_len, accept_path, bonus_token,
@@ -477,13 +497,11 @@ int owl_verify_step_host(owl_ctx* ctx, const owl_dims* d, const void* q_h, const
     }
     auto dev = [&](int i) { return ctx->stg[i].p; };
     const int32_t* no_d = no_h ? static_cast<const int32_t*>(dev(5)) : nullptr;
-    rc = owl_verify_attn(ctx, d, dev(0), dev(1), dev(2), static_cast<const int32_t*>(dev(3)),
+    rc = owl_verify_step(ctx, d, dev(0), dev(1), dev(2), static_cast<const int32_t*>(dev(3)),
                          static_cast<const int32_t*>(dev(4)), no_d, static_cast<const int32_t*>(dev(6)), dev(9),
-                         static_cast<float*>(dev(10)), stream_);
-    if (rc != OWL_OK) return rc;
-    rc = owl_tree_accept(ctx, d, static_cast<const float*>(dev(7)), static_cast<const int32_t*>(dev(8)), no_d,
-                         static_cast<const int32_t*>(dev(6)), static_cast<int32_t*>(dev(11)),
-                         static_cast<int32_t*>(dev(12)), static_cast<int32_t*>(dev(13)), nullptr, stream_);
+                         static_cast<float*>(dev(10)), static_cast<const float*>(dev(7)), static_cast<const int32_t*>(dev(8)),
+                         static_cast<int32_t*>(dev(11)), static_cast<int32_t*>(dev(12)), static_cast<int32_t*>(dev(13)), nullptr,
+                         stream_);
     if (rc != OWL_OK) return rc;
     void* dst[5] = {out_h, lse_h, alen_h, apath_h, bonus_h};
     for (int i = 0; i < 5; ++i) {
@@ -503,6 +521,22 @@ int owl_get_status(owl_ctx* ctx, void* stream_) {
     if (e == cudaSuccess) e = cudaMemsetAsync(ctx->status, 0, sizeof st, stream);
     if (e == cudaSuccess) e = cudaStreamSynchronize(stream);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "owl_get_status");
+    return st;
+}
+
+int owl_selftest_wait(owl_ctx* ctx, uint64_t limit_ns, uint64_t waited_ns[2], void* stream_) {
+    if (!ctx || limit_ns == 0 || limit_ns > 1000000000ull) return OWL_ERR_INVALID_ARG;   // at most a second
+    DeviceGuard guard(ctx->device);
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    selftest_wait_kernel<<<1, 32, 0, stream>>>(ctx->status, limit_ns, ctx->selftest_ns);
+    ++ctx->launches;
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "owl_selftest_wait launch");
+    unsigned long long ns[2] = {0, 0};
+    e = cudaMemcpyAsync(ns, ctx->selftest_ns, sizeof ns, cudaMemcpyDeviceToHost, stream);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "owl_selftest_wait");
+    const int st = owl_get_status(ctx, stream_);    // synchronises the stream
+    if (waited_ns) { waited_ns[0] = ns[0]; waited_ns[1] = ns[1]; }
     return st;
 }
 
@@ -555,14 +589,16 @@ constexpr int kStaticCounterWords = kMaxBatch;                 // per-sequence p
 constexpr int kStaticMaxDevices = 64;
 
 static __device__ __align__(256) unsigned long long g_accept_scratch[kStaticMaxKeys + kStaticStatusWords + kStaticCounterWords];
-std::atomic<uint32_t> g_static_epoch{0};
-
+// Every device has its own copy of the array, hence its own call counter: the counter's parity selects the set of
+// progress counters a call counts in, and the set a call clears must be the one the next call ON THAT DEVICE uses.
 unsigned long long* g_static_addr[kStaticMaxDevices] = {nullptr};
 bool g_static_ready[kStaticMaxDevices] = {false};
+uint32_t g_static_epoch[kStaticMaxDevices] = {0};
 std::mutex g_static_mutex;
 
-// Device address of g_accept_scratch on the current device `dev`; looked up on first use.
-cudaError_t static_scratch(int dev, unsigned long long** out) {
+// Device address of g_accept_scratch on the current device `dev` (looked up on first use) and the number of this
+// call among the calls made on that device.
+cudaError_t static_scratch(int dev, unsigned long long** out, uint32_t* epoch) {
     std::lock_guard<std::mutex> lock(g_static_mutex);
     if (!g_static_ready[dev]) {
         void* p = nullptr;
@@ -572,6 +608,7 @@ cudaError_t static_scratch(int dev, unsigned long long** out) {
         g_static_ready[dev] = true;
     }
     *out = g_static_addr[dev];
+    *epoch = ++g_static_epoch[dev];
     return cudaSuccess;
 }
 
@@ -592,7 +629,9 @@ extern "C" int owl_tree_accept_static(const owl_dims* d, const float* logits, co
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kStaticMaxDevices) return OWL_ERR_CUDA;
     unsigned long long* scratch = nullptr;
-    if (static_scratch(dev, &scratch) != cudaSuccess) { cudaGetLastError(); return OWL_ERR_CUDA; }
+    uint32_t epoch = 0;
+    if (static_scratch(dev, &scratch, &epoch) != cudaSuccess) { cudaGetLastError(); return OWL_ERR_CUDA; }
+    // without a status word of the caller's the verdict goes to a word of the array that no call reports
     int32_t* status = device_status ? device_status : reinterpret_cast<int32_t*>(scratch + kStaticMaxKeys);
 
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
@@ -618,7 +657,7 @@ extern "C" int owl_tree_accept_static(const owl_dims* d, const float* logits, co
     p.path_stride = d->path_stride;
     p.seq_counter = reinterpret_cast<unsigned int*>(scratch + kStaticMaxKeys + kStaticStatusWords);   // 2 x kMaxBatch
     p.counter_stride = kMaxBatch;
-    p.epoch = ++g_static_epoch;
+    p.epoch = epoch;
     dim3 grid((unsigned)chunks, (unsigned)d->total_nodes);
     argmax_partial_kernel<<<grid, kArgmaxThreads, 0, stream>>>(p);
     if (cudaGetLastError() != cudaSuccess) return OWL_ERR_CUDA;

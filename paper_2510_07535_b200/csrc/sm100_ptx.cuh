@@ -64,11 +64,11 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
 
 // Bounded wait.  A phase that has already completed returns true after one poll; otherwise the wait
 // returns false at once if the CTA's abort flag is up, and else spins on try_wait;
-// every 256 failed polls it looks at the abort flag and at the wall clock, and after `kWaitLimitNs`
-// it raises the abort flag itself and gives up.  A false return means: do not touch what the wait
+// every 256 failed polls it looks at the abort flag and at the wall clock, and after the time limit
+// (`kWaitLimitNs` in the kernels; an argument in the self-test) it raises the abort flag itself and gives up.  A false return means: do not touch what the wait
 // guarded; carry on with the (finite) control flow so that every CTA-level barrier is still reached.
 constexpr uint64_t kWaitLimitNs = 2000000000ull;   // 2 s: three orders of magnitude above any real wait
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait_ns(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint64_t limit_ns) {
     if (mbar_try_wait(bar, parity)) return true;      // the common case costs one poll
     if (*abort_flag) return false;
     uint64_t t0 = 0;
@@ -78,9 +78,12 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
             if (*abort_flag) return false;
             const uint64_t now = global_timer_ns();
             if (t0 == 0) t0 = now;
-            else if (now - t0 > kWaitLimitNs || polls > 0x7fffff00u) { *abort_flag = 1; return false; }
+            else if (now - t0 > limit_ns || polls > 0x7fffff00u) { *abort_flag = 1; return false; }
         }
     }
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    return mbar_wait_ns(bar, parity, abort_flag, kWaitLimitNs);
 }
 
 // Makes generic-proxy writes to shared memory visible to the async proxy (TMA, tcgen05.mma).

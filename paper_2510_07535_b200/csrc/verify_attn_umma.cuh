@@ -619,6 +619,23 @@ __device__ __forceinline__ void softmax_loop(const AttnParams& p, Aux* aux, unsi
                     tmem_st32(tS + c4 * 32, r);
                 }
                 tmem_wait_st();
+                // Slots of the sequence's last page beyond L + n may hold anything, NaN and Inf included.  Their scores
+                // were just overwritten (weight exactly 0), but 0 * NaN would still reach O through P V: zero those
+                // V rows in the ring slot (pages wholly past the end were zero-filled by the copy itself).  The
+                // tile's arrival barrier covers V as well as K, so the rows have landed; the stores are ordered
+                // before the product by the proxy fence here and the hand-off of P below.  Both warpgroups of a
+                // 256-row unit do it (zeros over zeros); the slot is not released before both products are done.
+                const int kv_valid = g.L + g.n - t * kTileKeys;            // >= 1 valid keys in this tile
+                if (kv_valid < kTileKeys) {
+                    const int kv_end = min(kTileKeys, ((kv_valid + p.page_size - 1) >> p.page_shift) << p.page_shift);
+                    const uint32_t seq = tile_base + (uint32_t)(g.shared ? i : 2 * i + s);
+                    unsigned char* vslot = smem + kRingOff + ((2u * seq + 1u) % kSlots) * kSlotBytes;
+#pragma unroll 1
+                    for (int k = kv_valid + (wtid >> 4); k < kv_end; k += 8)   // 16 threads x 16 bytes per 256-byte row
+                        *reinterpret_cast<uint4*>(vslot + (k >> 3) * 2048 + ((wtid >> 3) & 1) * 1024 + (k & 7) * 128 +
+                                                  (wtid & 7) * 16) = make_uint4(0u, 0u, 0u, 0u);
+                    fence_proxy_async_smem();
+                }
             }
             float sv[128];
             {
@@ -791,8 +808,6 @@ verify_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap 
     Aux* aux = reinterpret_cast<Aux*>(smem + kAuxOff);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t smem_base = smem_u32(smem);
-    // the combine kernel is launched as a programmatic dependent: let it queue up behind this grid's CTAs
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (smem_base & 1023u) {                       // operand tiles must sit on swizzle-atom boundaries
         if (tid == 0) report(p.status, kErrTimeout);
         return;
@@ -816,6 +831,10 @@ verify_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap 
     // launched as a programmatic dependent itself: everything above touched no input; from here on the kernel
     // before this one in the stream has completed (a no-op in an ordinary launch)
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    // The combine kernel is launched as a programmatic dependent and may queue up behind this grid's CTAs from here
+    // on.  It reads the call's inputs (lengths, offsets) before its own wait: triggering only after this grid's wait
+    // keeps those reads ordered after whatever kernel wrote them earlier in the stream.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     Walker w;
     if (!kManySeqs) build_walk_small(p, w);        // its global loads overlap the set-up above
     tc_fence_before();

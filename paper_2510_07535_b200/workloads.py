@@ -330,3 +330,111 @@ def config_spec(idx: int, ctx_div: int = 1, vocab: Optional[int] = None, q_presc
         return Spec("cfg4_8b_16xmixed_hybrid", 32, 8, ctx, kinds, shuffle_pages=True, plant_prob=0.65,
                     vocab=V, seed=seed, q_prescaled=q_prescaled)
     raise ValueError(f"no such configuration: {idx}")
+
+
+# --------------------------------------------------------------------------- toy decoding loop (inputs only)
+
+class ToyLoop:
+    """Inputs of a multi-step speculative-decoding loop on a toy "language model".
+
+    The toy model is a fixed map ``f`` on token ids: the text of sequence b is s_0, s_1 = f(s_0), ... and the
+    target's logits row for a node holding token t has its maximum at f(t).  Every step draws, per sequence, a
+    chain (verified without [SPEC]) or a tree (verified with one [SPEC] leaf per node), whose drafted tokens are
+    right (= f of the parent's token) with probability ``p_right`` and wrong otherwise, at most one right child
+    per parent and all siblings distinct.  K/V rows are a fixed pattern of (token, position id, head), so that a
+    cache can be checked against the text it should hold.  Nothing here verifies, accepts or commits anything.
+    """
+
+    def __init__(self, batch: int, vocab: int = 1000, num_kv_heads: int = 2, page_size: int = PAGE_SIZE,
+                 ctx0: Sequence[int] = (), max_tokens: int = 2048, p_right: float = 0.7, spec_token: int = 999,
+                 seed: int = 7):
+        self.B, self.V, self.Hkv, self.P = batch, vocab, num_kv_heads, page_size
+        self.spec_token, self.p_right = spec_token, p_right
+        self.rng = _gen(np.random.SeedSequence(seed))
+        self.ctx0 = np.asarray(ctx0 if len(ctx0) else self.rng.integers(1, 40, size=batch), dtype=np.int32)
+        self.start = self.rng.integers(0, vocab, size=batch)
+        self.max_pages = (max_tokens + page_size - 1) // page_size
+        self.num_pages = batch * self.max_pages
+        self.block_table = self.rng.permutation(self.num_pages).astype(np.int32).reshape(batch, self.max_pages)
+        self.noise = self.rng.random((64 * batch, vocab), dtype=np.float32)
+
+    def f(self, t):
+        """The toy model's next token (works on ints and integer arrays)."""
+        return (t * 37 + 11) % self.V
+
+    def text(self, b: int, length: int) -> np.ndarray:
+        out = np.empty(length, dtype=np.int64)
+        t = int(self.start[b])
+        for j in range(length):
+            out[j] = t
+            t = int(self.f(t))
+        return out
+
+    @staticmethod
+    def kv_rows(tokens, positions, num_kv_heads: int, which: int) -> np.ndarray:
+        """bf16 bit patterns [len, Hkv, 128] of the K (which = 0) or V (1) rows of tokens at position ids."""
+        t = np.asarray(tokens, dtype=np.int64)[:, None, None]
+        p = np.asarray(positions, dtype=np.int64)[:, None, None]
+        h = np.arange(num_kv_heads, dtype=np.int64)[None, :, None]
+        d = np.arange(HEAD_DIM, dtype=np.int64)[None, None, :]
+        x = (t * 131 + p * 31 + h * 7 + which * 3 + d * 17) % 251 - 125
+        return f32_to_bf16_bits((x / 64.0).astype(np.float32))   # multiples of 1/64 below 2: exact in bf16
+
+    def initial_cache(self):
+        """Caches holding the first ctx0[b] tokens of every text; everything else is a recognisable filler."""
+        k = np.full((self.num_pages, self.Hkv, self.P, HEAD_DIM), 0x3F80, dtype=np.uint16)
+        v = np.full_like(k, 0x3F80)
+        for b in range(self.B):
+            L = int(self.ctx0[b])
+            pos = np.arange(L)
+            self.write_rows(k, v, b, pos, self.text(b, L), pos)
+        return k, v
+
+    def write_rows(self, k_cache, v_cache, b: int, slots, tokens, positions) -> None:
+        """Stores the rows of `tokens` (with position ids `positions`) at logical slots `slots` of sequence b."""
+        slots = np.asarray(slots, dtype=np.int64)
+        pg = self.block_table[b, slots // self.P]
+        k_cache[pg, :, slots % self.P, :] = self.kv_rows(tokens, positions, self.Hkv, 0)
+        v_cache[pg, :, slots % self.P, :] = self.kv_rows(tokens, positions, self.Hkv, 1)
+
+    def read_rows(self, cache, b: int, slots) -> np.ndarray:
+        slots = np.asarray(slots, dtype=np.int64)
+        return cache[self.block_table[b, slots // self.P], :, slots % self.P, :]
+
+    def draft(self, roots: Sequence[int]):
+        """One step's drafts: (kinds, node_offsets, tree_parent, draft_tokens); kinds[b] is "chain" or "tree"."""
+        kinds, parents, tokens = [], [], []
+        for b in range(self.B):
+            if self.rng.random() < 0.35:
+                kinds.append("chain")
+                par = chain_parents(int(self.rng.integers(1, 9)))
+            else:
+                kinds.append("tree")
+                par = random_tree_parents(self.rng, int(self.rng.integers(1, 31)), 8)
+            tok = np.zeros(len(par), dtype=np.int64)
+            tok[0] = int(roots[b])
+            kids = {}
+            for i in range(1, len(par)):
+                kids.setdefault(int(par[i]), []).append(i)
+            for p_, ch in kids.items():               # parents come in increasing order: tok[p_] is final
+                right = int(self.f(tok[p_]))
+                lucky = int(self.rng.integers(0, len(ch))) if self.rng.random() < self.p_right else -1
+                wrong = 0
+                for j, i in enumerate(ch):
+                    if j == lucky:
+                        tok[i] = right
+                    else:
+                        wrong += 1
+                        tok[i] = (right + wrong) % self.V
+            parents.append(par)
+            tokens.append(tok)
+        counts = np.array([len(p_) for p_ in parents])
+        offsets = np.concatenate([[0], np.cumsum(counts)]).astype(np.int32)
+        return kinds, offsets, np.concatenate(parents).astype(np.int32), np.concatenate(tokens).astype(np.int32)
+
+    def logits(self, input_ids) -> np.ndarray:
+        """fp32 [len, V]: fixed noise in [0, 1) plus 5 at f(token) of every row's token."""
+        ids = np.asarray(input_ids, dtype=np.int64)
+        lg = self.noise[:len(ids)].copy()
+        lg[np.arange(len(ids)), self.f(ids)] += np.float32(5.0)
+        return lg

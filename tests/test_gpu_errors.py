@@ -146,3 +146,56 @@ def test_scale_and_head_limits():
     assert DeviceWorkload.attn(dataclass_replace(dw, dims=bad), ctx, check=False) == -2
     assert ctx.launch_count() == n0
     ctx.close()
+
+
+def test_bounded_wait_gives_up_and_reports_timeout():
+    """The kernels' wait routine on a barrier nothing completes: gives up after the limit, reports
+    OWL_ERR_TIMEOUT, a second wait returns at once, and the next ordinary call on the context is clean."""
+    wl = _wl()
+    dw = DeviceWorkload.upload(wl)
+    ctx = OwlContext(dims_of(wl))
+    limit = 1_000_000                                   # 1 ms
+    st, first_ns, second_ns = ctx.owl_selftest_wait(limit)
+    assert st == -6
+    assert limit <= first_ns <= 50 * limit              # gave up after the limit, and soon after it
+    assert second_ns < limit // 2                       # abort flag up: no second spin
+    assert ctx.owl_get_status() == 0                    # reading the status cleared it
+    assert ctx.lib.owl_selftest_wait(ctx._h, 0, None, None) == -1          # limit out of range: nothing launched
+    assert ctx.lib.owl_selftest_wait(ctx._h, 2_000_000_000, None, None) == -1
+    dw.step(ctx)
+    assert ctx.owl_get_status() == 0
+    ref_out, _ = oracle.verify_attn(wl.q, wl.k_cache, wl.v_cache, wl.block_table, wl.ctx_lens, wl.node_offsets,
+                                    wl.tree_parent, wl.sm_scale)
+    assert np.abs(dw.out_f32() - ref_out).max() <= 1e-2
+    ctx.close()
+
+
+def _accept_equals_oracle(dw, wl):
+    alen, path, bonus, am = oracle.tree_accept(wl.logits, wl.draft_tokens, wl.node_offsets, wl.tree_parent, 64)
+    np.testing.assert_array_equal(dw.node_argmax.cpu().numpy(), am)
+    np.testing.assert_array_equal(dw.accept_len.cpu().numpy(), alen)
+    np.testing.assert_array_equal(dw.accept_path.cpu().numpy(), path)
+    np.testing.assert_array_equal(dw.bonus_token.cpu().numpy(), bonus)
+
+
+def test_inconsistent_node_offsets_are_reported_and_leave_no_trace():
+    """Offsets that do not describe the call's rows (a sequence with no nodes, a total that is not total_nodes) set
+    the status word; the per-sequence progress counters they leave dirty must not disturb later calls, also
+    when those have a smaller batch."""
+    big = W.generate(W.Spec("offs", 8, 2, [40] * 6, [("tree", 8, 3), ("chain", 4), ("tree", 6, 3)] * 2, seed=15, vocab=20000))
+    small = W.generate(W.Spec("offs2", 8, 2, [40] * 2, [("chain", 5), ("tree", 7, 3)], seed=16, vocab=20000))
+    ctx = OwlContext(dims_of(big))
+    dw_big, dw_small = DeviceWorkload.upload(big), DeviceWorkload.upload(small)
+    for bad_offsets in ([0, 8, 8, 18, 26, 30, 36],          # sequence 1 has no nodes
+                        [0, 8, 12, 18, 26, 30, 35],         # last offset is not total_nodes
+                        [2, 8, 12, 18, 26, 30, 36]):        # first offset is not 0
+        bad = dataclass_replace(dw_big, node_offsets=torch.tensor(bad_offsets, dtype=torch.int32, device="cuda"))
+        bad.accept(ctx)
+        assert ctx.owl_get_status() == -4
+        for dw, wl in ((dw_small, small), (dw_big, big), (dw_small, small), (dw_big, big)):
+            for t in (dw.accept_len, dw.accept_path, dw.bonus_token, dw.node_argmax):
+                t.fill_(-9)
+            dw.accept(ctx)
+            assert ctx.owl_get_status() == 0
+            _accept_equals_oracle(dw, wl)
+    ctx.close()

@@ -116,11 +116,24 @@ def test_uniform_node_offsets_null():
     ctx.close()
 
 
-def test_unused_tail_slots_may_hold_large_values():
-    """Slots past L+n in the last page are multiplied by zero weight: finite garbage must not leak."""
-    wl = W.generate(W.Spec("tail", 8, 2, [22], [("tree", 5, 2)], seed=80, with_logits=False))
-    wl.k_cache[1, :, 11:, :] = 0x7F00   # ~1.7e38
-    wl.v_cache[1, :, 11:, :] = 0x7F00
+@pytest.mark.parametrize("page,hq,hkv,trees,ctx", [
+    (16, 8, 2, [("tree", 5, 2)], [22]),                        # 27 keys: 5 dead slots in the second page
+    (16, 4, 1, [("tree", 64, 8)], [1000]),                     # 256-row unit (both warpgroups read the tile)
+    (64, 16, 4, [("chain", 3), ("tree", 9, 3)], [130, 255]),   # larger pages: up to 63 dead slots
+    (128, 8, 2, [("chain", 1)], [128]),                        # one live key in the last 128-token page
+])
+def test_unused_tail_slots_may_hold_anything(page, hq, hkv, trees, ctx):
+    """Slots of a sequence's last page past L + n are never visible: NaN, Inf and huge values there (what
+    uninitialised cache memory may hold) must not reach any output.  Same fill as the oracle's own pin."""
+    wl = W.generate(W.Spec("tail", hq, hkv, ctx, trees, page_size=page, shuffle_pages=True, seed=80 + page, with_logits=False))
+    fills = [0x7FC0, 0x7F80, 0xFF80, 0x7F00]     # NaN, +Inf, -Inf, 1.7e38
+    for b in range(wl.spec.batch):
+        keys = int(wl.ctx_lens[b]) + int(wl.node_offsets[b + 1] - wl.node_offsets[b])
+        last, used = (keys - 1) // page, (keys - 1) % page + 1
+        pg = int(wl.block_table[b, last])
+        for j in range(used, page):
+            wl.k_cache[pg, :, j, :] = fills[j % 4]
+            wl.v_cache[pg, :, j, :] = fills[(j + 1) % 4]
     check_attention(wl)
 
 

@@ -116,6 +116,13 @@ def test_lossless_on_toy_model():
     assert emitted == plain[:len(emitted)]
 
 
+def _truncated_geometric_variance(n, p):
+    k = np.arange(1, n + 1)
+    pk = np.array([p ** (j - 1) * (1 - p) for j in range(1, n)] + [p ** (n - 1)])
+    assert abs(pk.sum() - 1) < 1e-12
+    return float((pk * k * k).sum() - (pk * k).sum() ** 2)
+
+
 def test_chain_acceptance_closed_form():
     """Chain of n nodes with each edge planted w.p. p: E[accept_len] = (1 - p^n) / (1 - p)."""
     n, p, trials, V = 8, 0.7, 10000, 512
@@ -132,17 +139,20 @@ def test_chain_acceptance_closed_form():
     alen, _, _ = oracle.accept_from_argmax(offs, np.tile(par, trials), tok, am)
     mean = alen.mean()
     expect = (1 - p ** n) / (1 - p)
-    # variance of a truncated geometric count is below n^2; 4 sigma of the mean
-    assert abs(mean - expect) < 4 * np.sqrt(n * n / trials), (mean, expect)
+    # P(len = k) = p^(k-1) (1 - p) for k < n and p^(n-1) for k = n: variance 4.858 at n = 8, p = 0.7;
+    # the bound is 4 sigma of the mean of `trials` draws (0.088)
+    assert abs(mean - expect) < 4 * np.sqrt(_truncated_geometric_variance(n, p) / trials), (mean, expect)
     assert abs(expect - 3.1412) < 1e-3
 
 
 def test_planted_logits_generator_agrees_with_closed_form():
     """The workload generator's planting (+10 on the parent's row) drives acceptance as designed."""
-    spec = W.Spec("p8", 4, 1, [16] * 64, [("chain", 8)] * 64, plant_prob=0.7, vocab=4096, seed=11)
+    B = 1024
+    spec = W.Spec("p8", 4, 1, [16] * B, [("chain", 8)] * B, plant_prob=0.7, vocab=4096, seed=11)
     wl = W.generate(spec, threads=1)
     alen, _, _, _ = oracle.tree_accept(wl.logits, wl.draft_tokens, wl.node_offsets, wl.tree_parent)
-    assert abs(alen.mean() - 3.1412) < 4 * 8 / np.sqrt(64)
+    # 4 sigma of the mean of 1024 chains (0.28); an unplanted edge matches with probability ~ 1/4096 only
+    assert abs(alen.mean() - 3.1412) < 4 * np.sqrt(_truncated_geometric_variance(8, 0.7) / B), alen.mean()
     assert alen.min() >= 1 and alen.max() <= 8
 
 

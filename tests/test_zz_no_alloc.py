@@ -69,6 +69,37 @@ def test_static_scratch_reports_a_malformed_tree_and_recovers():
     assert rc == 0 and int(status.item()) == 0            # the call cleared the status word itself
 
 
+def test_static_scratch_survives_inconsistent_offsets():
+    """A call whose node_offsets do not describe its rows leaves progress counters dirty in the shared array; the
+    calls after it (a smaller batch first) must still agree with the context entry point."""
+    big = W.generate(W.Spec("na_offs", 8, 2, [30] * 4, [("tree", 8, 3), ("chain", 4)] * 2, seed=93, vocab=20000))
+    small = W.generate(W.Spec("na_offs2", 8, 2, [30], [("tree", 9, 3)], seed=94, vocab=20000))
+    want = {}
+    for name, wl in (("big", big), ("small", small)):
+        dw = DeviceWorkload.upload(wl)
+        ctx = OwlContext(dims_of(wl))
+        dw.accept(ctx)
+        assert ctx.owl_get_status() == 0
+        want[name] = (dw, _outputs(dw))
+        ctx.close()
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    dw_big = want["big"][0]
+    bad_offsets = torch.tensor([0, 8, 8, 20, 24], dtype=torch.int32, device="cuda")     # sequence 1 has no nodes
+    rc = owl_tree_accept_static(dw_big.dims, dw_big.logits, dw_big.draft_tokens, bad_offsets, dw_big.tree_parent,
+                                dw_big.accept_len, dw_big.accept_path, dw_big.bonus_token, None, status)
+    torch.cuda.synchronize()
+    assert rc == 0 and int(status.item()) == -4
+    for name in ("small", "big", "small", "big"):
+        dw, ref = want[name]
+        _clear(dw)
+        rc = owl_tree_accept_static(dw.dims, dw.logits, dw.draft_tokens, dw.node_offsets, dw.tree_parent,
+                                    dw.accept_len, dw.accept_path, dw.bonus_token, dw.node_argmax, status)
+        torch.cuda.synchronize()
+        assert rc == 0 and int(status.item()) == 0
+        for got, r in zip(_outputs(dw), ref):
+            assert torch.equal(got, r)
+
+
 def test_static_scratch_rejects_sizes_beyond_the_array():
     V = 128256
     chunks = (V + 8191) // 8192
