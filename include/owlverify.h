@@ -142,6 +142,57 @@ int owl_tree_accept(owl_ctx* ctx, const owl_dims* dims, const float* logits,
                     int32_t* bonus_token, int32_t* node_argmax, void* stream);
 
 /*
+ * owl_tree_accept with one more output for trees that carry [SPEC] leaves (Section 3.2.2 "Decode Stage":
+ * "when a path is accepted, we take the hidden state of the corresponding [SPEC]"; Algorithm 1, h_S returned
+ * by OurTreeVerify): spec_node[b] (device int32 [B], required) = local index of the [SPEC] leaf - a child with
+ * a negative draft token - of the last node of the accepted path, the lowest index if there are several, -1 if
+ * that node has none (a chain verified without [SPEC]).  Everything else as owl_tree_accept.
+ */
+int owl_tree_accept_spec(owl_ctx* ctx, const owl_dims* dims, const float* logits,
+                         const int32_t* draft_tokens, const int32_t* node_offsets,
+                         const int32_t* tree_parent, int32_t* accept_len, int32_t* accept_path,
+                         int32_t* bonus_token, int32_t* spec_node, int32_t* node_argmax, void* stream);
+
+/*
+ * Prepare(d) of Algorithm 1 (Section 3.2.2 "Decode Stage"): appends one [SPEC] token after every tree path - as
+ * many [SPEC] as the drafted tree has nodes - and derives what the verifier needs: the parents (from which
+ * owl_verify_attn builds the attention mask) and the manipulated position ids.
+ *
+ * In (device): the drafted trees as for owl_verify_attn (dims->batch, dims->total_nodes, dims->max_nodes <= 32;
+ * node_offsets [B+1] or NULL for uniform; tree_parent [N]; draft_tokens [N], the root's entry being the target's
+ * own token t_{N+1}); ctx_lens [B]; spec_token = token id of [SPEC].
+ * Out (device, caller-owned), sequence b with n nodes occupying [2*node_offsets[b], 2*node_offsets[b] + 2n):
+ *   out_node_offsets [B+1]  = 2 * node_offsets
+ *   out_tree_parent  [2N]   nodes 0..n-1 as drafted; node n + j is the [SPEC] after the path ending in node j
+ *   out_draft_tokens [2N]   drafted token; -1 for a [SPEC] leaf (never a candidate of the acceptance)
+ *   out_input_ids    [2N]   what the verifier embeds: drafted token; spec_token for a leaf
+ *   out_position_ids [2N]   ctx_lens[b] + depth of the node (root: depth 0)
+ * The prepared trees (2n <= 64 nodes, parent[i] < i) go to owl_verify_attn / owl_tree_accept_spec with
+ * total_nodes = 2N, max_nodes = 2 * dims->max_nodes.  Asynchronous on `stream`.  A malformed tree sets
+ * OWL_ERR_BAD_TREE in the status word and leaves that sequence's rows unwritten.
+ */
+int owl_prepare_spec_tree(owl_ctx* ctx, const owl_dims* dims, const int32_t* node_offsets,
+                          const int32_t* tree_parent, const int32_t* draft_tokens, const int32_t* ctx_lens,
+                          int32_t spec_token, int32_t* out_node_offsets, int32_t* out_tree_parent,
+                          int32_t* out_draft_tokens, int32_t* out_input_ids, int32_t* out_position_ids,
+                          void* stream);
+
+/*
+ * Commit of the accepted tokens to the cache (Algorithm 1: "l <- l; d", "N <- N + |d|").  During verification
+ * the K/V of drafted node i of sequence b sit at logical position L_b + i; for the accepted path p_0 = 0 < p_1 <
+ * ... < p_{a-1} (accept_path / accept_len as owl_tree_accept wrote them) the rows at L_b + p_k move to L_b + k,
+ * for every KV head, in k_cache and v_cache, IN PLACE, and ctx_lens[b] becomes L_b + a.  Whatever else was
+ * drafted stays behind as dead slots past the new length.  Uses dims->batch, total_nodes, max_nodes,
+ * num_kv_heads, head_dim, page_size, max_pages_per_seq, num_pages, path_stride.  All pointers device; k_cache,
+ * v_cache and ctx_lens are read and written.  Asynchronous on `stream` (two small kernels in stream order).  A
+ * path that is not a root path in node order sets OWL_ERR_BAD_TREE, a page id out of range OWL_ERR_BAD_PAGE;
+ * that sequence is then left untouched, length included.
+ */
+int owl_kv_commit(owl_ctx* ctx, const owl_dims* dims, void* k_cache, void* v_cache,
+                  const int32_t* block_table, int32_t* ctx_lens, const int32_t* node_offsets,
+                  const int32_t* accept_len, const int32_t* accept_path, void* stream);
+
+/*
  * One whole verify step on device buffers: owl_verify_attn and owl_tree_accept of the same batch
  * (Section 3.2.2 "Decode Stage" followed by the acceptance of the Introduction), arguments as in those
  * two calls, results bit for bit those of the two calls.  The two halves do not depend on each other (the

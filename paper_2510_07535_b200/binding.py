@@ -50,6 +50,12 @@ def load_library() -> ctypes.CDLL:
     lib.owl_verify_attn.argtypes = [vp, dp] + [vp] * 10
     lib.owl_tree_accept.restype = i32
     lib.owl_tree_accept.argtypes = [vp, dp] + [vp] * 9
+    lib.owl_tree_accept_spec.restype = i32
+    lib.owl_tree_accept_spec.argtypes = [vp, dp] + [vp] * 10
+    lib.owl_prepare_spec_tree.restype = i32
+    lib.owl_prepare_spec_tree.argtypes = [vp, dp] + [vp] * 4 + [ctypes.c_int32] + [vp] * 6
+    lib.owl_kv_commit.restype = i32
+    lib.owl_kv_commit.argtypes = [vp, dp] + [vp] * 8
     lib.owl_tree_accept_static.restype = i32
     lib.owl_tree_accept_static.argtypes = [dp] + [vp] * 10
     lib.owl_verify_step.restype = i32
@@ -142,6 +148,48 @@ class OwlContext:
             _ptr(node_argmax, torch.int32, dev, "node_argmax"), _stream(dev))
         if check and rc != OWL_OK:
             raise OwlError(rc, "owl_tree_accept", self.last_error())
+        return rc
+
+    def owl_tree_accept_spec(self, dims: OwlDims, logits, draft_tokens, node_offsets, tree_parent, accept_len, accept_path,
+                             bonus_token, spec_node, node_argmax=None, check: bool = True) -> int:
+        dev = self.device
+        i32 = torch.int32
+        rc = self.lib.owl_tree_accept_spec(
+            self._h, ctypes.byref(dims), _ptr(logits, torch.float32, dev, "logits"), _ptr(draft_tokens, i32, dev, "draft_tokens"),
+            _ptr(node_offsets, i32, dev, "node_offsets"), _ptr(tree_parent, i32, dev, "tree_parent"),
+            _ptr(accept_len, i32, dev, "accept_len"), _ptr(accept_path, i32, dev, "accept_path"),
+            _ptr(bonus_token, i32, dev, "bonus_token"), _ptr(spec_node, i32, dev, "spec_node"),
+            _ptr(node_argmax, i32, dev, "node_argmax"), _stream(dev))
+        if check and rc != OWL_OK:
+            raise OwlError(rc, "owl_tree_accept_spec", self.last_error())
+        return rc
+
+    def owl_prepare_spec_tree(self, dims: OwlDims, node_offsets, tree_parent, draft_tokens, ctx_lens, spec_token: int,
+                              out_node_offsets, out_tree_parent, out_draft_tokens, out_input_ids, out_position_ids,
+                              check: bool = True) -> int:
+        dev = self.device
+        i32 = torch.int32
+        rc = self.lib.owl_prepare_spec_tree(
+            self._h, ctypes.byref(dims), _ptr(node_offsets, i32, dev, "node_offsets"), _ptr(tree_parent, i32, dev, "tree_parent"),
+            _ptr(draft_tokens, i32, dev, "draft_tokens"), _ptr(ctx_lens, i32, dev, "ctx_lens"), int(spec_token),
+            _ptr(out_node_offsets, i32, dev, "out_node_offsets"), _ptr(out_tree_parent, i32, dev, "out_tree_parent"),
+            _ptr(out_draft_tokens, i32, dev, "out_draft_tokens"), _ptr(out_input_ids, i32, dev, "out_input_ids"),
+            _ptr(out_position_ids, i32, dev, "out_position_ids"), _stream(dev))
+        if check and rc != OWL_OK:
+            raise OwlError(rc, "owl_prepare_spec_tree", self.last_error())
+        return rc
+
+    def owl_kv_commit(self, dims: OwlDims, k_cache, v_cache, block_table, ctx_lens, node_offsets, accept_len, accept_path,
+                      check: bool = True) -> int:
+        dev = self.device
+        i32, bf = torch.int32, torch.bfloat16
+        rc = self.lib.owl_kv_commit(
+            self._h, ctypes.byref(dims), _ptr(k_cache, bf, dev, "k_cache"), _ptr(v_cache, bf, dev, "v_cache"),
+            _ptr(block_table, i32, dev, "block_table"), _ptr(ctx_lens, i32, dev, "ctx_lens"),
+            _ptr(node_offsets, i32, dev, "node_offsets"), _ptr(accept_len, i32, dev, "accept_len"),
+            _ptr(accept_path, i32, dev, "accept_path"), _stream(dev))
+        if check and rc != OWL_OK:
+            raise OwlError(rc, "owl_kv_commit", self.last_error())
         return rc
 
     def owl_verify_step(self, dims: OwlDims, q, k_cache, v_cache, block_table, ctx_lens, node_offsets, tree_parent, out, lse,

@@ -51,6 +51,7 @@ struct AcceptParams {
     int32_t* accept_path;
     int32_t* bonus_token;
     int32_t* node_argmax;
+    int32_t* spec_node;              // optional [B]: the [SPEC] leaf (negative draft token) under the last accepted node
     unsigned long long* part_keys;   // [total_nodes, chunks]
     unsigned int* seq_counter;       // [2, batch]: chunk keys of the sequence stored so far; set epoch & 1 is in use
     uint32_t epoch;                  // call number: the other set is cleared for the next call
@@ -73,8 +74,12 @@ __device__ __forceinline__ void accept_walk_seq(const AcceptParams& p, const int
     const int base = p.node_offsets ? p.node_offsets[b] : b * p.nodes_uniform;
     const int n = p.node_offsets ? p.node_offsets[b + 1] - base : p.nodes_uniform;
     __shared__ int s_parent[kMaxNodes], s_am[kMaxNodes], s_tok[kMaxNodes];
-    __shared__ int s_bad, s_win;
-    if (i == 0) { s_bad = (n < 1 || n > p.max_nodes || n > p.path_stride || base < 0 || base + n > p.total_nodes) ? 1 : 0; s_win = 0; }
+    __shared__ int s_bad, s_win, s_leaf;
+    if (i == 0) {
+        s_bad = (n < 1 || n > p.max_nodes || n > p.path_stride || base < 0 || base + n > p.total_nodes) ? 1 : 0;
+        s_win = 0;
+        s_leaf = kMaxNodes;
+    }
     __syncthreads();
     if (s_bad) { if (i == 0) report(p.status, kErrBadTree); return; }
     if (i < n) {
@@ -110,6 +115,14 @@ __device__ __forceinline__ void accept_walk_seq(const AcceptParams& p, const int
     }
     atomicMax(&s_win, key);
     __syncthreads();
+    if (p.spec_node) {
+        // Section 3.2.2 "Decode Stage": the hidden state handed to the drafter is that of the [SPEC] which follows
+        // the accepted path, i.e. the [SPEC] child of its last node (lowest index if several, -1 if none)
+        const int win = kMaxNodes - 1 - (s_win & 0xff);
+        if (i < n && s_parent[i] == win && s_tok[i] < 0) atomicMin(&s_leaf, i);
+        __syncthreads();
+        if (i == 0) p.spec_node[b] = s_leaf < kMaxNodes ? s_leaf : -1;
+    }
     if (i == 0) {
         const int win = kMaxNodes - 1 - (s_win & 0xff);
         const int len = s_win >> 8;

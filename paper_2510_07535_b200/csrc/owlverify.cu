@@ -12,6 +12,7 @@
 #include "accept.cuh"
 #include "combine.cuh"
 #include "owl_common.cuh"
+#include "spec_loop.cuh"
 #include "verify_attn_umma.cuh"
 
 using namespace owl;
@@ -383,7 +384,8 @@ int owl_verify_attn(owl_ctx* ctx, const owl_dims* d, const void* q, const void* 
 // Argument checks of the acceptance and its kernel parameters (everything but the counters of the stand-alone kernel).
 static int accept_params(owl_ctx* ctx, const owl_dims* d, const float* logits, const int32_t* draft_tokens,
                          const int32_t* node_offsets, const int32_t* tree_parent, int32_t* accept_len,
-                         int32_t* accept_path, int32_t* bonus_token, int32_t* node_argmax, AcceptParams& p) {
+                         int32_t* accept_path, int32_t* bonus_token, int32_t* node_argmax, AcceptParams& p,
+                         int32_t* spec_node = nullptr) {
     if (!ctx) return OWL_ERR_INVALID_ARG;
     int rc = check_dims(d, false, true);
     if (rc != OWL_OK) return rc;
@@ -402,6 +404,7 @@ static int accept_params(owl_ctx* ctx, const owl_dims* d, const float* logits, c
     p.accept_path = accept_path;
     p.bonus_token = bonus_token;
     p.node_argmax = node_argmax;
+    p.spec_node = spec_node;
     p.part_keys = ctx->part_keys;
     p.chunks = chunks;
     p.status = ctx->status;
@@ -414,12 +417,13 @@ static int accept_params(owl_ctx* ctx, const owl_dims* d, const float* logits, c
     return OWL_OK;
 }
 
-int owl_tree_accept(owl_ctx* ctx, const owl_dims* d, const float* logits, const int32_t* draft_tokens,
-                    const int32_t* node_offsets, const int32_t* tree_parent, int32_t* accept_len,
-                    int32_t* accept_path, int32_t* bonus_token, int32_t* node_argmax, void* stream_) {
+static int tree_accept_impl(owl_ctx* ctx, const owl_dims* d, const float* logits, const int32_t* draft_tokens,
+                            const int32_t* node_offsets, const int32_t* tree_parent, int32_t* accept_len,
+                            int32_t* accept_path, int32_t* bonus_token, int32_t* spec_node, int32_t* node_argmax,
+                            void* stream_) {
     AcceptParams p;
     const int rc = accept_params(ctx, d, logits, draft_tokens, node_offsets, tree_parent, accept_len, accept_path, bonus_token,
-                                 node_argmax, p);
+                                 node_argmax, p, spec_node);
     if (rc != OWL_OK) return rc;
     DeviceGuard guard(ctx->device);
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
@@ -435,6 +439,79 @@ int owl_tree_accept(owl_ctx* ctx, const owl_dims* d, const float* logits, const 
     if (ctx->profiling) ctx->ev_accept_valid = true;
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(ctx, e, "owl_tree_accept launch");
+    return OWL_OK;
+}
+
+int owl_tree_accept(owl_ctx* ctx, const owl_dims* d, const float* logits, const int32_t* draft_tokens,
+                    const int32_t* node_offsets, const int32_t* tree_parent, int32_t* accept_len,
+                    int32_t* accept_path, int32_t* bonus_token, int32_t* node_argmax, void* stream_) {
+    return tree_accept_impl(ctx, d, logits, draft_tokens, node_offsets, tree_parent, accept_len, accept_path, bonus_token,
+                            nullptr, node_argmax, stream_);
+}
+
+int owl_tree_accept_spec(owl_ctx* ctx, const owl_dims* d, const float* logits, const int32_t* draft_tokens,
+                         const int32_t* node_offsets, const int32_t* tree_parent, int32_t* accept_len,
+                         int32_t* accept_path, int32_t* bonus_token, int32_t* spec_node, int32_t* node_argmax,
+                         void* stream_) {
+    if (!spec_node) return OWL_ERR_INVALID_ARG;
+    return tree_accept_impl(ctx, d, logits, draft_tokens, node_offsets, tree_parent, accept_len, accept_path, bonus_token,
+                            spec_node, node_argmax, stream_);
+}
+
+int owl_prepare_spec_tree(owl_ctx* ctx, const owl_dims* d, const int32_t* node_offsets, const int32_t* tree_parent,
+                          const int32_t* draft_tokens, const int32_t* ctx_lens, int32_t spec_token,
+                          int32_t* out_node_offsets, int32_t* out_tree_parent, int32_t* out_draft_tokens,
+                          int32_t* out_input_ids, int32_t* out_position_ids, void* stream_) {
+    if (!ctx) return OWL_ERR_INVALID_ARG;
+    int rc = check_dims(d, false, false);
+    if (rc != OWL_OK) return rc;
+    if (2 * d->max_nodes > kMaxNodes) return OWL_ERR_UNSUPPORTED;        // the prepared tree has twice the nodes
+    if (!tree_parent || !draft_tokens || !ctx_lens || !out_node_offsets || !out_tree_parent || !out_draft_tokens ||
+        !out_input_ids || !out_position_ids)
+        return OWL_ERR_INVALID_ARG;
+    if (!node_offsets && d->total_nodes % d->batch != 0) return OWL_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    PrepareParams p{};
+    p.node_offsets = node_offsets; p.tree_parent = tree_parent; p.draft_tokens = draft_tokens; p.ctx_lens = ctx_lens;
+    p.out_offsets = out_node_offsets; p.out_parent = out_tree_parent; p.out_draft = out_draft_tokens;
+    p.out_input_ids = out_input_ids; p.out_position = out_position_ids;
+    p.status = ctx->status;
+    p.batch = d->batch; p.total_nodes = d->total_nodes; p.nodes_uniform = d->total_nodes / d->batch;
+    p.max_nodes = d->max_nodes; p.spec_token = spec_token;
+    prepare_spec_kernel<<<d->batch, kPrepareThreads, 0, static_cast<cudaStream_t>(stream_)>>>(p);
+    ++ctx->launches;
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "owl_prepare_spec_tree launch");
+    return OWL_OK;
+}
+
+int owl_kv_commit(owl_ctx* ctx, const owl_dims* d, void* k_cache, void* v_cache, const int32_t* block_table,
+                  int32_t* ctx_lens, const int32_t* node_offsets, const int32_t* accept_len, const int32_t* accept_path,
+                  void* stream_) {
+    if (!ctx) return OWL_ERR_INVALID_ARG;
+    int rc = check_dims(d, false, false);
+    if (rc != OWL_OK) return rc;
+    if (d->num_kv_heads < 1 || d->max_pages_per_seq < 1 || d->num_pages < 1 || d->path_stride < 1) return OWL_ERR_INVALID_ARG;
+    if (d->head_dim != kHeadDim || d->num_kv_heads > 128 ||
+        !(d->page_size == 16 || d->page_size == 32 || d->page_size == 64 || d->page_size == 128))
+        return OWL_ERR_UNSUPPORTED;
+    if (!k_cache || !v_cache || !block_table || !ctx_lens || !accept_len || !accept_path) return OWL_ERR_INVALID_ARG;
+    if (!node_offsets && d->total_nodes % d->batch != 0) return OWL_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    CommitParams p{};
+    p.k_cache = static_cast<__nv_bfloat16*>(k_cache); p.v_cache = static_cast<__nv_bfloat16*>(v_cache);
+    p.block_table = block_table; p.ctx_lens = ctx_lens; p.node_offsets = node_offsets;
+    p.accept_len = accept_len; p.accept_path = accept_path; p.status = ctx->status;
+    p.batch = d->batch; p.total_nodes = d->total_nodes; p.nodes_uniform = d->total_nodes / d->batch;
+    p.max_nodes = d->max_nodes; p.num_kv_heads = d->num_kv_heads;
+    p.page_size = d->page_size; p.page_shift = log2_exact(d->page_size);
+    p.max_pages_per_seq = d->max_pages_per_seq; p.num_pages = d->num_pages; p.path_stride = d->path_stride;
+    kv_commit_move_kernel<<<dim3(2u * (unsigned)d->num_kv_heads, (unsigned)d->batch), kCommitThreads, 0, stream>>>(p);
+    kv_commit_lens_kernel<<<d->batch, kCommitThreads, 0, stream>>>(p);
+    ctx->launches += 2;
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "owl_kv_commit launch");
     return OWL_OK;
 }
 
