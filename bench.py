@@ -3,14 +3,24 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 0..4] [--impl reference]
 
-One "step" is one pass of the whole hot path (owl_verify_attn + owl_tree_accept) over one batch
-of seeded synthetic input.  Prints ONE JSON line.  `value` is algorithmic HBM bytes of a step
-(K/V of every visible position + Q + out + LSE + logits) divided by the device time of a step,
-summed over ranks: the "achieved HBM GB/s" half of the headline metric; `verify_step_us` is the
-other half.  Inputs are resident in HBM when the timed region starts and rotate over enough
-copies that no step finds its inputs in L2.  `e2e` is the same metric through the host-buffer
-C-ABI call, host<->device copies inside the timed region.  `--impl reference` times the CPU
-oracle on bounded samples of the same workload instead.
+One "step" is one pass of the whole hot path (owl_verify_step = owl_verify_attn + owl_tree_accept) over one
+batch of seeded synthetic input.  Prints ONE JSON line.  The default run measures all five benchmark
+configurations one after the other and reports each under `per_config`; the top-level keys are those of the
+headline workload (configuration 1: 8B shape, 32K context, 32-node tree) and `headline_128k` repeats the
+128K-context workload's figures.  `--workload k` measures configuration k alone.
+
+`value` is algorithmic HBM bytes of a step (K/V of every visible position + Q + out + LSE + logits) divided by
+the device time of a step, summed over ranks: the "achieved HBM GB/s" half of the metric; `verify_step_us` is
+the other half.  A step's time is the median over `--regions` timed regions of exactly K steps each (CUDA
+events on the launching stream, barrier + synchronize on both sides of every region; min, max and the first
+region are reported too).  Inputs are resident in HBM and rotate over enough copies that no step finds its
+inputs in L2.  `kernel_us` times each half of the step in a loop of its own on the same inputs, so that every
+figure is a plain bytes / time of calls that ran back to back; `roofline` is the verify-attention call's.
+Clocks, power and throttle reasons are sampled through NVML across all regions of a workload; `us_x_sm_mhz`
+makes runs at different clocks comparable, and `sustained` repeats the step back to back for `--sustained`
+seconds (power-limited regime) with a clock record of its own.  `e2e` is the same metric through the
+host-buffer C-ABI call, host<->device copies inside the timed region.  `--impl reference` times the CPU oracle
+on bounded samples of the headline workload instead.
 """
 from __future__ import annotations
 
@@ -65,12 +75,12 @@ def ncu_traffic(workload_name):
 
 
 class ClockSampler(threading.Thread):
-    """Polls SM clock and throttle reasons through NVML (read-only) while the timed region runs."""
+    """Polls SM clock, power and throttle reasons through NVML (read-only) between begin() and end()."""
 
     def __init__(self, index: int, period: float = 0.001):
         super().__init__(daemon=True)
         self.index, self.period = index, period
-        self.samples, self.reasons = [], set()
+        self.samples, self.power, self.reasons = [], [], set()
         self.max_mhz = None
         self._stop_evt = threading.Event()
         self.active = threading.Event()
@@ -95,6 +105,7 @@ class ClockSampler(threading.Thread):
             if self.active.is_set():
                 try:
                     self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                    self.power.append(nv.nvmlDeviceGetPowerUsage(self.h) / 1000.0)
                     r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
                     for bit, name in names.items():
                         if r & bit:
@@ -103,12 +114,23 @@ class ClockSampler(threading.Thread):
                     pass
             time.sleep(self.period)
 
+    def begin(self, _label=""):
+        self.samples, self.power, self.reasons = [], [], set()
+        self.active.set()
+
+    def end(self):
+        self.active.clear()
+        time.sleep(2 * self.period)
+        return self.summary()
+
     def stop(self):
         self._stop_evt.set()
 
     def summary(self):
         med = int(np.median(self.samples)) if self.samples else None
-        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+        return {"sm_mhz": med, "sm_min_mhz": int(np.min(self.samples)) if self.samples else None, "sm_max_mhz": self.max_mhz,
+                "power_w_max": round(float(np.max(self.power)), 1) if self.power else None,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
 
 
 def physical_gpu_index(local_rank: int) -> int:
@@ -174,7 +196,7 @@ def run_reference(args, rank, world):
     from paper_2510_07535_b200 import workloads as W
     if rank != 0:
         return
-    spec = W.config_spec(args.workload)
+    spec = W.config_spec(1 if args.workload is None else args.workload)
     wl = W.generate(spec)
     attn_b, logit_b = algorithmic_bytes(wl)
     timer = OracleTimer(wl)
@@ -201,11 +223,128 @@ def run_reference(args, rank, world):
     print(json.dumps(line), flush=True)
 
 
+def _event_loop_us(fn, calls, barrier):
+    """Device microseconds per call of `calls` back-to-back calls of fn(i), CUDA events on the launching stream."""
+    import torch
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    ev0.record()
+    for i in range(calls):
+        fn(i)
+    ev1.record()
+    barrier()
+    return ev0.elapsed_time(ev1) * 1e3 / calls
+
+
+def measure_workload(idx, args, ctx_factory, dev, world, rank, barrier, max_over_ranks, sampler, headline):
+    """Times one benchmark configuration; returns its record (and, for the headline one, the extra legs)."""
+    import torch
+    from paper_2510_07535_b200 import replicas, workloads as W
+    from paper_2510_07535_b200.runner import DeviceWorkload, dims_of
+
+    spec = W.config_spec(idx)
+    if world > 1:
+        spec.seed = replicas.replica_seed(spec.seed, rank)   # replicas: every rank verifies its own batch
+    wl = W.generate(spec)
+    attn_b, logit_b = algorithmic_bytes(wl)
+    step_bytes = attn_b + logit_b
+    # rotate over enough input copies that a step never finds its K/V or logits in L2
+    copies = max(2, int(np.ceil(4 * L2_BYTES / step_bytes)) + 1) if step_bytes < 8 * L2_BYTES else 2
+    reps = [DeviceWorkload.upload(wl, dev) for _ in range(copies)]
+    ctx = ctx_factory(dims_of(wl))
+    peak, peak_kind = measured_peaks()
+    K = args.steps
+
+    for i in range(args.warmup):
+        reps[i % copies].step(ctx)
+    assert ctx.owl_get_status() == 0
+
+    # ---- the step: `regions` timed regions of exactly K steps each (barrier + synchronize on both sides of each)
+    sampler.begin(spec.name)
+    launches0 = ctx.launch_count()
+    region_us = [max_over_ranks(_event_loop_us(lambda i: reps[(r * K + i) % copies].step(ctx), K, barrier)) for r in range(args.regions)]
+    launches = (ctx.launch_count() - launches0) // args.regions
+    # ---- the two halves on their own, same inputs, same rotation: attention (split-KV kernel + merge) and acceptance
+    attn_us = max_over_ranks(np.median([_event_loop_us(lambda i: reps[(r * K + i) % copies].attn(ctx), K, barrier) for r in range(5)]))
+    accept_us = max_over_ranks(np.median([_event_loop_us(lambda i: reps[(r * K + i) % copies].accept(ctx), K, barrier) for r in range(5)]))
+    clocks = sampler.end()
+    assert ctx.owl_get_status() == 0
+    step_us = float(np.median(region_us))
+
+    fused = launches // K == 2 and logit_b > 0     # small scan: no arg-max kernel, the attention launch reads the logits too
+    rec = {
+        "workload": spec.name, "verify_step_us": step_us,
+        "step_us_regions": {"median": step_us, "min": float(np.min(region_us)), "max": float(np.max(region_us)),
+                            "first": float(region_us[0]), "regions": args.regions, "steps_per_region": K},
+        "hbm_gbs": step_bytes / step_us / 1e3, "frac_of_hbm_peak": step_bytes / step_us / 1e3 / peak,
+        "bytes_per_step": {"attention": attn_b, "logits": logit_b},
+        "kernel_us": {"verify_attn_call": attn_us, "tree_accept_call": accept_us,
+                      "note": "each call timed alone in a loop of its own (CUDA events around K back-to-back calls, same "
+                              "rotating inputs): owl_verify_attn = split-KV attention kernel + LSE merge; owl_tree_accept = "
+                              "arg-max scan + walk" + ("; inside the step the scan rides in the attention launch" if fused else "")},
+        "roofline": {"bound": "hbm", "kernel": "owl_verify_attn (verify_attn_umma_kernel + combine_sched_kernel, 2 launches)",
+                     "bytes_per_launch": attn_b, "achieved": attn_b / attn_us / 1e3, "peak": peak, "unit": "GB/s",
+                     "frac": attn_b / attn_us / 1e3 / peak, "peak_kind": f"of {peak_kind}", "traffic": ncu_traffic(spec.name)},
+        "accept_gbs": logit_b / accept_us / 1e3, "accept_frac_of_hbm_peak": logit_b / accept_us / 1e3 / peak,
+        "gpu_launches_per_step": launches // K, "clocks": clocks,
+        "us_x_sm_mhz": step_us * clocks["sm_mhz"] if clocks.get("sm_mhz") else None,
+        "l2": f"rotating {copies} input copies ({copies * step_bytes / 1e6:.0f} MB > L2)",
+        "config": {"batch": spec.batch, "ctx_lens": [int(min(spec.ctx_lens)), int(max(spec.ctx_lens))], "nodes": int(wl.total_nodes),
+                   "q_heads": spec.num_q_heads, "kv_heads": spec.num_kv_heads, "vocab": spec.vocab},
+    }
+    # ---- sustained: at least `--sustained` seconds of back-to-back steps with their own clock record
+    if args.sustained > 0 and step_us > 100:
+        n = int(np.ceil(args.sustained * 1e6 / step_us))
+        sampler.begin(spec.name + " sustained")
+        sus = max_over_ranks(_event_loop_us(lambda i: reps[i % copies].step(ctx), n, barrier))
+        c = sampler.end()
+        rec["sustained"] = {"verify_step_us": sus, "steps": n, "frac_of_hbm_peak": step_bytes / sus / 1e3 / peak, "clocks": c,
+                            "us_x_sm_mhz": sus * c["sm_mhz"] if c.get("sm_mhz") else None}
+
+    extra = {}
+    if headline:
+        extra["launches_region"] = launches
+        # ---- end to end through the host-buffer C-ABI call (pinned host memory)
+        pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+        bf = lambda a: torch.from_numpy(a.view(np.int16)).view(torch.bfloat16).pin_memory()
+        N, Hq, D = wl.q.shape
+        B = spec.batch
+        h_in = dict(q=bf(wl.q), k=bf(wl.k_cache), v=bf(wl.v_cache), bt=pin(wl.block_table), cl=pin(wl.ctx_lens),
+                    no=pin(wl.node_offsets), tp=pin(wl.tree_parent), lg=pin(wl.logits), dt=pin(wl.draft_tokens))
+        h_out = dict(out=torch.empty((N, Hq, D), dtype=torch.bfloat16).pin_memory(),
+                     lse=torch.empty((N, Hq), dtype=torch.float32).pin_memory(),
+                     alen=torch.empty(B, dtype=torch.int32).pin_memory(),
+                     path=torch.empty((B, 64), dtype=torch.int32).pin_memory(),
+                     bonus=torch.empty(B, dtype=torch.int32).pin_memory())
+        h2d = sum(t.numel() * t.element_size() for t in h_in.values())
+        d2h = sum(t.numel() * t.element_size() for t in h_out.values())
+
+        def host_step(_=0):
+            return ctx.owl_verify_step_host(reps[0].dims, h_in["q"], h_in["k"], h_in["v"], h_in["bt"], h_in["cl"], h_in["no"],
+                                            h_in["tp"], h_in["lg"], h_in["dt"], h_out["out"], h_out["lse"], h_out["alen"],
+                                            h_out["path"], h_out["bonus"])
+        e2e_steps = max(3, min(K, int(2.0 / max(h2d / 20e9, 1e-4))))
+        for _ in range(3):
+            assert host_step() == 0
+        e2e_us = max_over_ranks(_event_loop_us(host_step, e2e_steps, barrier))
+        extra["e2e"] = {"value": world * step_bytes / e2e_us / 1e3, "unit": "GB/s", "h2d_bytes_per_step": h2d,
+                        "d2h_bytes_per_step": d2h, "us_per_step": e2e_us, "steps": e2e_steps}
+        # ---- CPU oracle beside it (rank 0, N=1 only)
+        if rank == 0 and world == 1 and not args.no_cpu_baseline:
+            timer = OracleTimer(wl)
+            est, _, desc = timer.sample(args.cpu_budget)
+            extra["cpu_baseline"] = {"value": step_bytes / est / 1e9, "unit": "GB/s", "cores": timer.threads, "kind": "oracle",
+                                     "sample": desc, "est_step_s": est}
+    ctx.close()
+    del reps
+    torch.cuda.empty_cache()
+    return rec, extra
+
+
 def run_gpu(args, rank, world, local_rank):
     import torch
     import torch.distributed as dist
-    from paper_2510_07535_b200 import OwlContext, replicas, workloads as W
-    from paper_2510_07535_b200.runner import DeviceWorkload, dims_of
+    from paper_2510_07535_b200 import OwlContext, replicas
 
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
@@ -218,125 +357,40 @@ def run_gpu(args, rank, world, local_rank):
         torch.cuda.synchronize(dev)
 
     def max_over_ranks(x: float) -> float:
-        return replicas.aggregate(0.0, x, dev)[1]
-
-    spec = W.config_spec(args.workload)
-    if world > 1:
-        spec.seed = replicas.replica_seed(spec.seed, rank)   # replicas: every rank verifies its own batch
-    wl = W.generate(spec)
-    attn_b, logit_b = algorithmic_bytes(wl)
-    step_bytes = attn_b + logit_b
-    # rotate over enough input copies that a step never finds its K/V or logits in L2
-    copies = max(2, int(np.ceil(4 * L2_BYTES / step_bytes)) + 1) if step_bytes < 8 * L2_BYTES else 2
-    reps = [DeviceWorkload.upload(wl, dev) for _ in range(copies)]
-    ctx = OwlContext(dims_of(wl), dev)
+        return replicas.aggregate(0.0, float(x), dev)[1]
 
     sampler = ClockSampler(physical_gpu_index(local_rank))
     sampler.start()
-
-    def run_steps(k, first=0):
-        for i in range(k):
-            reps[(first + i) % copies].step(ctx)
-
-    # ---- device-resident timing
-    run_steps(args.warmup)
-    assert ctx.owl_get_status() == 0
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    launches0 = ctx.launch_count()
-    barrier()
-    sampler.active.set()
-    ev0.record()
-    run_steps(args.steps, args.warmup)
-    ev1.record()
-    barrier()
-    sampler.active.clear()
-    launches = ctx.launch_count() - launches0
-    assert ctx.owl_get_status() == 0
-    sec = max_over_ranks(ev0.elapsed_time(ev1) * 1e-3)
-    step_s = sec / args.steps
-
-    # ---- per-kernel device times of the same steps (events between the kernels, same stream)
-    ctx.set_profiling(True)
-    kt = np.zeros(4)
-    kn = min(args.steps, 200)
-    for i in range(kn):
-        reps[i % copies].step(ctx)
-        kt += np.array(ctx.last_kernel_times())
-    ctx.set_profiling(False)
-    kt /= kn
-
-    # ---- end to end through the host-buffer C-ABI call (pinned host memory)
-    pin = lambda a, dt=None: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
-    bf = lambda a: torch.from_numpy(a.view(np.int16)).view(torch.bfloat16).pin_memory()
-    N, Hq, D = wl.q.shape
-    B = spec.batch
-    h_in = dict(q=bf(wl.q), k=bf(wl.k_cache), v=bf(wl.v_cache), bt=pin(wl.block_table), cl=pin(wl.ctx_lens),
-                no=pin(wl.node_offsets), tp=pin(wl.tree_parent), lg=pin(wl.logits), dt=pin(wl.draft_tokens))
-    h_out = dict(out=torch.empty((N, Hq, D), dtype=torch.bfloat16).pin_memory(),
-                 lse=torch.empty((N, Hq), dtype=torch.float32).pin_memory(),
-                 alen=torch.empty(B, dtype=torch.int32).pin_memory(),
-                 path=torch.empty((B, 64), dtype=torch.int32).pin_memory(),
-                 bonus=torch.empty(B, dtype=torch.int32).pin_memory())
-    h2d = sum(t.numel() * t.element_size() for t in h_in.values())
-    d2h = sum(t.numel() * t.element_size() for t in h_out.values())
-
-    def host_step():
-        return ctx.owl_verify_step_host(reps[0].dims, h_in["q"], h_in["k"], h_in["v"], h_in["bt"], h_in["cl"], h_in["no"],
-                                        h_in["tp"], h_in["lg"], h_in["dt"], h_out["out"], h_out["lse"], h_out["alen"],
-                                        h_out["path"], h_out["bonus"])
-    e2e_steps = max(3, min(args.steps, int(2.0 / max(h2d / 20e9, 1e-4))))
-    for _ in range(3):
-        assert host_step() == 0
-    barrier()
-    ev0.record()
-    for _ in range(e2e_steps):
-        host_step()
-    ev1.record()
-    barrier()
-    e2e_s = max_over_ranks(ev0.elapsed_time(ev1) * 1e-3) / e2e_steps
+    workloads = [args.workload] if args.workload is not None else [1, 0, 2, 3, 4]
+    head_idx = workloads[0]
+    records, extra = {}, {}
+    for idx in workloads:
+        rec, ex = measure_workload(idx, args, lambda d: OwlContext(d, dev), dev, world, rank, barrier, max_over_ranks, sampler,
+                                   headline=(idx == head_idx))
+        records[rec["workload"]] = rec
+        if idx == head_idx:
+            head, extra = rec, ex
     sampler.stop()
 
-    # ---- CPU oracle beside it (rank 0, N=1 only)
-    cpu = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        timer = OracleTimer(wl)
-        est, _, desc = timer.sample(args.cpu_budget)
-        cpu = {"value": step_bytes / est / 1e9, "unit": "GB/s", "cores": timer.threads, "kind": "oracle", "sample": desc,
-               "est_step_s": est}
-
     if rank == 0:
-        peak, peak_kind = measured_peaks()
-        # a step with a small acceptance scan has no arg-max kernel: the attention kernel's spare warps read the logits,
-        # so those bytes belong to that launch
-        fused = kt[2] == 0 and logit_b > 0
-        attn_launch_b = attn_b + (logit_b if fused else 0)
-        achieved = attn_launch_b / kt[0] / 1e9 if kt[0] > 0 else None
+        step_bytes = head["bytes_per_step"]["attention"] + head["bytes_per_step"]["logits"]
         line = {
-            "metric": METRIC, "value": world * step_bytes / step_s / 1e9, "unit": "GB/s", "n_gpus": world,
-            "steps": args.steps, "warmup": args.warmup, "ms_per_step": step_s * 1e3, "higher_is_better": True,
+            "metric": METRIC, "value": world * step_bytes / head["verify_step_us"] / 1e3, "unit": "GB/s", "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": head["verify_step_us"] * 1e-3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": spec.name, "batch": B, "ctx_lens": [int(min(spec.ctx_lens)), int(max(spec.ctx_lens))],
-                       "nodes": int(wl.total_nodes), "q_heads": spec.num_q_heads, "kv_heads": spec.num_kv_heads,
-                       "vocab": spec.vocab, "parallelism": "replicas only" if world > 1 else "single GPU",
-                       "l2": f"rotating {copies} input copies ({copies * step_bytes / 1e6:.0f} MB > L2)"},
-            "verify_step_us": step_s * 1e6,
-            "frac_of_hbm_peak": step_bytes / step_s / 1e9 / peak,
-            "kernel_us": {"verify_attn": kt[0] * 1e6, "combine": kt[1] * 1e6, "argmax_accept": kt[2] * 1e6},
-            "bytes_per_step": {"attention": attn_b, "logits": logit_b},
-            "roofline": {"bound": "hbm", "kernel": "verify_attn" + (" (+ logits scan)" if fused else ""),
-                         "bytes_per_launch": attn_launch_b, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                         "frac": achieved / peak if achieved else None, "peak_kind": f"of {peak_kind}",
-                         "traffic": ncu_traffic(spec.name)},
-            "accept_gbs": logit_b / kt[2] / 1e9 if kt[2] > 0 else None,
-            "e2e": {"value": world * step_bytes / e2e_s / 1e9, "unit": "GB/s", "h2d_bytes_per_step": h2d,
-                    "d2h_bytes_per_step": d2h, "us_per_step": e2e_s * 1e6, "steps": e2e_steps},
-            "gpu_launches": launches,
-            "clocks": sampler.summary(),
+            "config": dict(head["config"], workload=head["workload"], parallelism="replicas only" if world > 1 else "single GPU",
+                           l2=head["l2"], timing=f"median of {args.regions} timed regions of {args.steps} steps each"),
+            "verify_step_us": head["verify_step_us"], "frac_of_hbm_peak": head["frac_of_hbm_peak"],
+            "kernel_us": head["kernel_us"], "bytes_per_step": head["bytes_per_step"], "roofline": head["roofline"],
+            "accept_gbs": head["accept_gbs"], "e2e": extra.get("e2e"), "gpu_launches": extra.get("launches_region"),
+            "clocks": head["clocks"], "per_config": records,
         }
-        if cpu:
-            line["cpu_baseline"] = cpu
+        big = next((r for n, r in records.items() if n.startswith("cfg2")), None)
+        if big:
+            line["headline_128k"] = {k: big[k] for k in ("workload", "verify_step_us", "hbm_gbs", "frac_of_hbm_peak", "roofline", "clocks")}
+        if "cpu_baseline" in extra:
+            line["cpu_baseline"] = extra["cpu_baseline"]
         print(json.dumps(line), flush=True)
-    ctx.close()
     if world > 1:
         dist.destroy_process_group()
 
@@ -344,9 +398,12 @@ def run_gpu(args, rank, world, local_rank):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=500)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=20)
-    ap.add_argument("--workload", type=int, default=1, help="benchmark configuration 0..4 (default 1: 8B shape, 32K context, 32-node tree)")
+    ap.add_argument("--workload", type=int, default=None,
+                    help="one benchmark configuration 0..4 only (default: all five, headline = 1: 8B shape, 32K context, 32-node tree)")
+    ap.add_argument("--regions", type=int, default=15, help="timed regions of --steps steps each; the headline is their median")
+    ap.add_argument("--sustained", type=float, default=2.0, help="seconds of back-to-back steps for the sustained record (0: skip)")
     ap.add_argument("--impl", default="owl", choices=["owl", "reference"])
     ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of CPU oracle work per sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -1,18 +1,17 @@
 // Greedy tree acceptance: row arg-max over the vocabulary, then the acceptance walk.
 //
-// Kernel 1 scans fp32 logits with 16-byte loads.  Every (value, index) candidate is folded into
-// one 64-bit key, high word = the float mapped to an unsigned integer that sorts like the float
-// (NaN mapped to -inf, -0 to +0), low word = ~index, so that an unsigned max picks the larger
-// value and, among equal values, the lower index.  Per-thread, warp (shuffle) and block maxima
-// give one key per (row, vocabulary chunk), stored to part_keys[row][chunk] (no atomics, nothing
-// to initialise).
+// The scan reads fp32 logits with 16-byte loads, one warp per (row, 8192-float vocabulary chunk) item.  Every
+// (value, index) candidate is folded into one 64-bit key, high word = the float mapped to an unsigned
+// integer that sorts like the float (NaN mapped to -inf, -0 to +0), low word = ~index, so that an unsigned
+// max picks the larger value and, among equal values, the lower index.  Per-lane and warp (shuffle) maxima
+// give one key per item, stored to part_keys[row][chunk] (no atomics, nothing to initialise).
 //
-// The CTA that stores the last chunk key of a sequence (a per-sequence counter, bumped after a
-// __threadfence; nobody waits for anybody) then does that sequence's walk in the same launch: it reduces
-// the chunk keys to arg-max tokens, evaluates for every node whether all edges on its root path match
-// (draft token == parent's arg-max), picks the deepest matching node (lowest index among equals) and
-// writes accept_len / accept_path / bonus_token.  Calls alternate between two sets of counters and clear the
-// idle one as a whole, so no separate clearing pass is needed.
+// The warp that stores the last chunk key of a sequence (a per-sequence counter, bumped after a
+// __threadfence; nobody waits for anybody) notes the sequence, and its CTA does that sequence's walk in the
+// same launch: it reduces the chunk keys to arg-max tokens, evaluates for every node whether all edges on its
+// root path match (draft token == parent's arg-max), picks the deepest matching node (lowest index among
+// equals) and writes accept_len / accept_path / bonus_token.  Calls alternate between two sets of counters and
+// clear the idle one as a whole, so no separate clearing pass is needed.
 //
 // Inside a verify step with a small scan both halves run as guests of the attention kernels: the scan in warps
 // the attention pass does not use (argmax_scan_chunk_warp), the walk in extra CTAs of the merge kernel, after
@@ -26,7 +25,6 @@ namespace owl {
 constexpr int kArgmaxThreads = 256;
 static_assert(kArgmaxThreads >= kMaxNodes, "the walk needs one thread per node");
 constexpr int kArgmaxChunk = 8192;  // floats per CTA: 8 x float4 per thread
-static_assert(kArgmaxChunk == 8 * 4 * kArgmaxThreads, "argmax_partial_kernel reads its chunk in one round of 8 loads");
 
 // 16-byte load of data that is read once: no L1 allocation, first in line for eviction from L2
 // (`policy` from createpolicy.fractional.L2::evict_first).
@@ -135,10 +133,15 @@ __device__ __forceinline__ void accept_walk_seq(const AcceptParams& p, const int
     }
 }
 
-// The same scan of one (row, vocabulary chunk) by a single warp, for callers that have warps to spare inside
-// another kernel (the verify step's attention pass scans the logits with its two idle warps while it streams K/V).
-// Stores the same key argmax_partial_kernel would: the maximum over (value, ~index) does not depend on how the
-// chunk's elements are dealt out to threads.
+// Scan of one (row, vocabulary chunk) item by a single warp: eight 16-byte loads per lane and round.  Per round a
+// lane first takes the maximum of its 32 values by a tree of fmaxf (NaN drops out: fmaxf returns the other operand,
+// and the final fmaxf with -inf turns an all-NaN round into -inf), and only if that beats its best so far - which
+// becomes rare quickly - looks for the first value that attains it.  Strict '>' and first-match keep the lowest
+// index among equal values, because a lane's indices grow along its walk; the maximum over (value, ~index) keys
+// then does not depend on how the chunk's elements are dealt out to lanes.
+// kPipelined: the next round's loads are issued before this round is reduced (twice the registers); the attention
+// kernel's guest warps, which run on 72 registers, use the plain form.
+template <bool kPipelined>
 __device__ __forceinline__ void argmax_scan_chunk_warp(const AcceptParams& p, const int row, const int chunk) {
     const int lane = threadIdx.x & 31;
     const long long V = p.vocab;
@@ -155,26 +158,48 @@ __device__ __forceinline__ void argmax_scan_chunk_warp(const AcceptParams& p, co
     uint32_t bi = 0xffffffffu;   // "no candidate yet"
     const float4* body = reinterpret_cast<const float4*>(base + a0);
     const int nvec = (int)((a1 - a0) >> 2);
-    for (int v0 = 0; v0 < nvec; v0 += 32 * 8) {
-        float4 x[8];
+    const uint64_t policy = l2_evict_first_policy();     // the logits are read once
+    const float4 none = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+    auto load_round = [&](int v0, float4 (&x)[8]) {
 #pragma unroll
         for (int j = 0; j < 8; ++j) {            // eight independent 16-byte loads per lane in flight
             const int v = v0 + j * 32 + lane;
-            x[j] = v < nvec ? __ldg(body + v) : make_float4(0.f, 0.f, 0.f, 0.f);
+            x[j] = v < nvec ? ld_stream_f4(body + v, policy) : none;
         }
+    };
+    auto reduce_round = [&](int v0, const float4 (&x)[8]) {
+        float m[8];
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            const int v = v0 + j * 32 + lane;
-            if (v < nvec) {
-                const uint32_t i0 = (uint32_t)(a0 + 4ll * v);
-                // NaN reads as -inf; strict '>' keeps the first maximum (indices grow along this lane's walk)
-                const float e0 = x[j].x != x[j].x ? -INFINITY : x[j].x, e1 = x[j].y != x[j].y ? -INFINITY : x[j].y;
-                const float e2 = x[j].z != x[j].z ? -INFINITY : x[j].z, e3 = x[j].w != x[j].w ? -INFINITY : x[j].w;
-                if (bi == 0xffffffffu || e0 > bv) { bv = e0; bi = i0; }
-                if (e1 > bv) { bv = e1; bi = i0 + 1; }
-                if (e2 > bv) { bv = e2; bi = i0 + 2; }
-                if (e3 > bv) { bv = e3; bi = i0 + 3; }
+        for (int j = 0; j < 8; ++j) m[j] = fmaxf(fmaxf(x[j].x, x[j].y), fmaxf(x[j].z, x[j].w));
+        const float mx = fmaxf(fmaxf(fmaxf(fmaxf(m[0], m[1]), fmaxf(m[2], m[3])), fmaxf(fmaxf(m[4], m[5]), fmaxf(m[6], m[7]))), -INFINITY);
+        if (v0 + lane < nvec && (bi == 0xffffffffu || mx > bv)) {
+            // a new best (or the first candidate): the first of this round's values that attains it; slots past
+            // the end hold -inf, which only an all -inf round matches, and then the round's first slot wins
+            bv = mx;
+#pragma unroll
+            for (int j = 7; j >= 0; --j) {
+                const uint32_t i0 = (uint32_t)(a0 + 4ll * (v0 + j * 32 + lane));
+                if (fmaxf(x[j].w, -INFINITY) == mx) bi = i0 + 3;
+                if (fmaxf(x[j].z, -INFINITY) == mx) bi = i0 + 2;
+                if (fmaxf(x[j].y, -INFINITY) == mx) bi = i0 + 1;
+                if (fmaxf(x[j].x, -INFINITY) == mx) bi = i0;
             }
+        }
+    };
+    if (kPipelined) {
+        float4 xa[8], xb[8];
+        if (nvec > 0) load_round(0, xa);
+        for (int v0 = 0; v0 < nvec; v0 += 2 * 32 * 8) {
+            if (v0 + 32 * 8 < nvec) load_round(v0 + 32 * 8, xb);
+            reduce_round(v0, xa);
+            if (v0 + 2 * 32 * 8 < nvec) load_round(v0 + 2 * 32 * 8, xa);
+            if (v0 + 32 * 8 < nvec) reduce_round(v0 + 32 * 8, xb);
+        }
+    } else {
+        for (int v0 = 0; v0 < nvec; v0 += 32 * 8) {
+            float4 x[8];
+            load_round(v0, x);
+            reduce_round(v0, x);
         }
     }
     unsigned long long key = bi != 0xffffffffu ? argmax_key(bv, bi) : 0ull;
@@ -194,13 +219,25 @@ __device__ __forceinline__ void argmax_scan_chunk_warp(const AcceptParams& p, co
     if (lane == 0) p.part_keys[(long long)row * p.chunks + chunk] = key;
 }
 
+// Persistent scan: the grid's warps take the (row, vocabulary chunk) items in turn (consecutive warps read
+// consecutive chunks), each with eight 16-byte loads per lane in flight, so that a warp streams without the
+// per-item cost of a CTA's launch, barriers and fences.  After storing an item's key, the warp counts it for
+// the row's sequence; the warp that counts a sequence's last item notes the sequence, and when the CTA has run
+// out of items it walks the trees of the sequences it noted.  (A CTA can note at most as many as it scanned items.)
+constexpr int kArgmaxWarps = kArgmaxThreads / 32;
+constexpr int kArgmaxCtasPerSm = 2;     // what fits at the kernel's register count
+constexpr int kArgmaxNoteMax = 64;
+
 __global__ void __launch_bounds__(kArgmaxThreads) argmax_partial_kernel(const AcceptParams p) {
     // may be launched as a programmatic dependent of the kernel before it in the stream: nothing is read
     // before that kernel has completed (a no-op in an ordinary launch)
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next kernel may queue up; it waits likewise
-    const int row = blockIdx.y;
-    if (blockIdx.x == 0 && blockIdx.y == 0) {
+    __shared__ int s_note[kArgmaxNoteMax];
+    __shared__ int s_notes;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) s_notes = 0;
+    if (blockIdx.x == 0) {
         // Once per call: clear every counter of the idle set (the next call counts there, whatever its batch), and
         // check that the packed offsets describe this call's rows: start at 0, end at total_nodes, 1..max_nodes
         // nodes per sequence.  With inconsistent offsets a row would count for the wrong sequence and a walk could
@@ -216,94 +253,56 @@ __global__ void __launch_bounds__(kArgmaxThreads) argmax_partial_kernel(const Ac
             if (bad) report(p.status, kErrBadTree);
         }
     }
-    const long long V = p.vocab;
-    const long long c0 = (long long)blockIdx.x * kArgmaxChunk;
-    const long long c1 = c0 + kArgmaxChunk < V ? c0 + kArgmaxChunk : V;
-    const float* base = p.logits + row * V;
-
-    // [c0, a0) scalar head up to 16-byte alignment, [a0, a1) float4 body, [a1, c1) scalar tail
-    const uintptr_t addr = reinterpret_cast<uintptr_t>(base + c0);
-    long long a0 = c0 + (long long)(((16 - (addr & 15)) & 15) >> 2);
-    if (a0 > c1) a0 = c1;
-    const long long a1 = a0 + ((c1 - a0) & ~3ll);
-
-    float bv = -INFINITY;
-    uint32_t bi = 0xffffffffu;   // "no candidate yet"
-    unsigned long long key = 0;
-    const float4* body = reinterpret_cast<const float4*>(base + a0);
-    const int nvec = (int)((a1 - a0) >> 2);
-    // A chunk is 8 x 16 bytes per thread: all eight loads are issued before the first compare, so that a CTA has its
-    // whole 32 KB in flight at once (one load per iteration left the scan at about half of the memory bandwidth).
-    // The logits are read once: they bypass L1 and are the first to leave L2.
-    {
-        const uint64_t policy = l2_evict_first_policy();
-        float4 x[8];
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            const int v = j * kArgmaxThreads + (int)threadIdx.x;
-            x[j] = v < nvec ? ld_stream_f4(body + v, policy) : make_float4(0.f, 0.f, 0.f, 0.f);
-        }
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            const int v = j * kArgmaxThreads + (int)threadIdx.x;
-            if (v < nvec) {
-                const uint32_t i0 = (uint32_t)(a0 + 4ll * v);
-                // NaN reads as -inf; strict '>' keeps the first maximum (indices grow along this thread's walk)
-                const float e0 = x[j].x != x[j].x ? -INFINITY : x[j].x, e1 = x[j].y != x[j].y ? -INFINITY : x[j].y;
-                const float e2 = x[j].z != x[j].z ? -INFINITY : x[j].z, e3 = x[j].w != x[j].w ? -INFINITY : x[j].w;
-                if (bi == 0xffffffffu || e0 > bv) { bv = e0; bi = i0; }
-                if (e1 > bv) { bv = e1; bi = i0 + 1; }
-                if (e2 > bv) { bv = e2; bi = i0 + 2; }
-                if (e3 > bv) { bv = e3; bi = i0 + 3; }
+    __syncthreads();
+    const long long items = (long long)p.total_nodes * p.chunks;
+    const long long stride = (long long)gridDim.x * kArgmaxWarps;
+    for (long long it = (long long)blockIdx.x * kArgmaxWarps + warp; it < items; it += stride) {
+        const int row = (int)(it / p.chunks), chunk = (int)(it - (long long)row * p.chunks);
+        argmax_scan_chunk_warp<true>(p, row, chunk);
+        if (lane == 0) {
+            // which sequence owns this row, and is this the last of its chunk keys?
+            int b, n_b;
+            if (p.node_offsets) {
+                int lo = 0, hi = p.batch;   // largest b with node_offsets[b] <= row
+                while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (p.node_offsets[mid] <= row) lo = mid; else hi = mid; }
+                b = lo;
+                n_b = p.node_offsets[b + 1] - p.node_offsets[b];
+            } else {
+                b = row / p.nodes_uniform;
+                n_b = p.nodes_uniform;
+            }
+            __threadfence();
+            // two sets of counters: this call counts in set (epoch & 1); the other one is cleared as a whole (above)
+            // for the next call, so a counter left dirty by malformed input is gone two calls later at the latest and
+            // is never counted in
+            unsigned int* ctr = p.seq_counter + (size_t)(p.epoch & 1u) * p.counter_stride + b;
+            const unsigned int want = atomicAdd(ctr, 1u) + 1u;
+            if ((long long)want == (long long)p.chunks * n_b) {
+                *ctr = 0u;                                   // a completed counter is left clean as well
+                const int slot = atomicAdd(&s_notes, 1);
+                if (slot < kArgmaxNoteMax) s_note[slot] = b;
+                else report(p.status, kErrBadTree);          // only inconsistent offsets can complete that many here
             }
         }
     }
-    if (bi != 0xffffffffu) key = argmax_key(bv, bi);
-    // ragged ends: at most 3 + 3 elements per chunk
-    if (threadIdx.x < 8) {
-        long long j = threadIdx.x < 4 ? c0 + threadIdx.x : a1 + (threadIdx.x - 4);
-        const long long lim = threadIdx.x < 4 ? a0 : c1;
-        if (j < lim) {
-            const unsigned long long k2 = argmax_key(base[j], (uint32_t)j);
-            key = k2 > key ? k2 : key;
-        }
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        const unsigned long long other = __shfl_xor_sync(0xffffffffu, key, o);
-        key = other > key ? other : key;
-    }
-    __shared__ unsigned long long s_key[kArgmaxThreads / 32];
-    if ((threadIdx.x & 31) == 0) s_key[threadIdx.x >> 5] = key;
+    __threadfence();
     __syncthreads();
-    __shared__ int s_walk_b;
-    if (threadIdx.x == 0) {
-#pragma unroll
-        for (int w = 1; w < kArgmaxThreads / 32; ++w) key = s_key[w] > key ? s_key[w] : key;
-        p.part_keys[(long long)row * p.chunks + blockIdx.x] = key;
-        // which sequence owns this row, and is this the last of its chunk keys?
-        int b, n_b;
-        if (p.node_offsets) {
-            int lo = 0, hi = p.batch;   // largest b with node_offsets[b] <= row
-            while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (p.node_offsets[mid] <= row) lo = mid; else hi = mid; }
-            b = lo;
-            n_b = p.node_offsets[b + 1] - p.node_offsets[b];
-        } else {
-            b = row / p.nodes_uniform;
-            n_b = p.nodes_uniform;
-        }
-        __threadfence();
-        // two sets of counters: this call counts in set (epoch & 1); the other one is cleared as a whole (above)
-        // for the next call, so a counter left dirty by malformed input is gone two calls later at the latest and
-        // is never counted in
-        unsigned int* ctr = p.seq_counter + (size_t)(p.epoch & 1u) * p.counter_stride + b;
-        const unsigned int want = atomicAdd(ctr, 1u) + 1u;
-        if ((long long)want == (long long)p.chunks * n_b) *ctr = 0u;   // a completed counter is left clean as well
-        s_walk_b = ((long long)want == (long long)p.chunks * n_b) ? b : -1;
-        __threadfence();
+    const int notes = min(s_notes, kArgmaxNoteMax);
+    for (int k = 0; k < notes; ++k) {
+        accept_walk_seq(p, s_note[k]);
+        __syncthreads();
     }
-    __syncthreads();
-    if (s_walk_b >= 0) accept_walk_seq(p, s_walk_b);
+}
+
+// Grid of the scan for `items` (row, chunk) items on a device with `sms` multiprocessors: as many warps as give
+// every warp the same number of items (4096 items on 2368 resident warps would leave a quarter of the warps idle
+// during the second half of the kernel; 2048 warps with two items each do not).
+__host__ inline unsigned argmax_grid(long long items, int sms) {
+    const long long max_warps = (long long)sms * kArgmaxCtasPerSm * kArgmaxWarps;
+    const long long rounds = (items + max_warps - 1) / max_warps;
+    const long long warps = rounds > 0 ? (items + rounds - 1) / rounds : 1;
+    const long long ctas = (warps + kArgmaxWarps - 1) / kArgmaxWarps;
+    return (unsigned)(ctas < 1 ? 1 : ctas);
 }
 
 }  // namespace owl

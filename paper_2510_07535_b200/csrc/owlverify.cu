@@ -432,7 +432,7 @@ static int tree_accept_impl(owl_ctx* ctx, const owl_dims* d, const float* logits
     p.counter_stride = ctx->max_dims.batch;
     p.epoch = ++ctx->accept_epoch;
     if (ctx->profiling) cudaEventRecord(ctx->ev[3], stream);
-    dim3 grid((unsigned)chunks, (unsigned)d->total_nodes);
+    dim3 grid(argmax_grid((long long)chunks * d->total_nodes, ctx->sm_count));
     launch_dependent(argmax_partial_kernel, grid, dim3(kArgmaxThreads), stream, p);   // the walk runs in the CTA that finishes a sequence
     ++ctx->launches;
     if (ctx->profiling) cudaEventRecord(ctx->ev[4], stream);
@@ -735,8 +735,9 @@ extern "C" int owl_tree_accept_static(const owl_dims* d, const float* logits, co
     p.seq_counter = reinterpret_cast<unsigned int*>(scratch + kStaticMaxKeys + kStaticStatusWords);   // 2 x kMaxBatch
     p.counter_stride = kMaxBatch;
     p.epoch = epoch;
-    dim3 grid((unsigned)chunks, (unsigned)d->total_nodes);
-    argmax_partial_kernel<<<grid, kArgmaxThreads, 0, stream>>>(p);
+    int sms = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) { cudaGetLastError(); return OWL_ERR_CUDA; }
+    argmax_partial_kernel<<<argmax_grid((long long)chunks * d->total_nodes, sms), kArgmaxThreads, 0, stream>>>(p);
     if (cudaGetLastError() != cudaSuccess) return OWL_ERR_CUDA;
     return OWL_OK;
 }

@@ -853,7 +853,7 @@ verify_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap 
         else if (kFused) {
             const long long items = (long long)ap.total_nodes * ap.chunks;
             for (long long it = 2ll * blockIdx.x + (warp - 2); it < items; it += 2ll * gridDim.x)
-                argmax_scan_chunk_warp(ap, (int)(it / ap.chunks), (int)(it % ap.chunks));
+                argmax_scan_chunk_warp<false>(ap, (int)(it / ap.chunks), (int)(it % ap.chunks));
         }
     } else {
         asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
