@@ -39,6 +39,15 @@ def _load():
         lib.owl_oracle_attn.restype = ctypes.c_int
         lib.owl_oracle_attn.argtypes = [ctypes.c_int] * 7 + [ctypes.c_double, u16p, u16p, u16p, i32p, i32p, i32p, i32p,
                                                               ctypes.c_int64, i32p, i32p, f64p, f64p]
+        lib.owl_oracle_attn_f16.restype = ctypes.c_int
+        lib.owl_oracle_attn_f16.argtypes = lib.owl_oracle_attn.argtypes
+        lib.owl_oracle_decode16.restype = None
+        lib.owl_oracle_decode16.argtypes = [u16p, ctypes.c_int64, ctypes.c_int, f64p]
+        lib.owl_oracle_howl_route.restype = None
+        lib.owl_oracle_howl_route.argtypes = [ctypes.c_int, ctypes.POINTER(ctypes.c_float), ctypes.c_float,
+                                              ctypes.POINTER(ctypes.c_uint8), i32p]
+        lib.owl_oracle_prepare_hybrid.restype = ctypes.c_int
+        lib.owl_oracle_prepare_hybrid.argtypes = [ctypes.c_int, i32p, i32p, i32p, i32p, i32p, ctypes.c_int32] + [i32p] * 5
         lib.owl_oracle_argmax.restype = None
         lib.owl_oracle_argmax.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.c_int64, ctypes.c_int64, i32p]
         lib.owl_oracle_accept.restype = ctypes.c_int
@@ -70,8 +79,8 @@ def _c(a, dtype) -> np.ndarray:
 
 
 def verify_attn(q, k_cache, v_cache, block_table, ctx_lens, node_offsets, tree_parent, sm_scale: float,
-                rows: Optional[Tuple[np.ndarray, np.ndarray]] = None) -> Tuple[np.ndarray, np.ndarray]:
-    """Tree-masked attention in fp64.
+                rows: Optional[Tuple[np.ndarray, np.ndarray]] = None, dtype: str = "bf16") -> Tuple[np.ndarray, np.ndarray]:
+    """Tree-masked attention in fp64.  ``dtype``: how the 16-bit patterns of q / k_cache / v_cache read, "bf16" or "f16".
 
     q uint16 [N,Hq,D] (bf16 bits); k_cache/v_cache uint16 [pages,Hkv,page,D]; block_table int32
     [B,max_pages]; ctx_lens int32 [B]; node_offsets int32 [B+1]; tree_parent int32 [N].
@@ -98,7 +107,8 @@ def verify_attn(q, k_cache, v_cache, block_table, ctx_lens, node_offsets, tree_p
         assert rh.shape[0] == n_rows
         out = np.empty((n_rows, D), dtype=np.float64)
         lse = np.empty((n_rows,), dtype=np.float64)
-    rc = lib.owl_oracle_attn(B, Hq, Hkv, D, page, block_table.shape[1], num_pages, float(sm_scale),
+    fn = {"bf16": lib.owl_oracle_attn, "f16": lib.owl_oracle_attn_f16}[dtype]
+    rc = fn(B, Hq, Hkv, D, page, block_table.shape[1], num_pages, float(sm_scale),
                              _p(q, ctypes.c_uint16), _p(k_cache, ctypes.c_uint16), _p(v_cache, ctypes.c_uint16),
                              _p(block_table, ctypes.c_int32), _p(ctx_lens, ctypes.c_int32),
                              _p(node_offsets, ctypes.c_int32), _p(tree_parent, ctypes.c_int32),
@@ -192,3 +202,44 @@ def kv_commit(k_cache, v_cache, block_table, ctx_lens, node_offsets, accept_len,
                                   _p(accept_path, i32), accept_path.shape[1])
     if rc != 0:
         raise ValueError(f"owl_oracle_kv_commit failed with code {rc}")
+
+
+def decode16(bits, dtype: str) -> np.ndarray:
+    """The oracle's own decoding of 16-bit patterns ("bf16" or "f16") to float64."""
+    lib = _load()
+    bits = _c(bits, np.uint16).ravel()
+    out = np.empty(bits.shape[0], np.float64)
+    lib.owl_oracle_decode16(_p(bits, ctypes.c_uint16), bits.shape[0], 1 if dtype == "f16" else 0, _p(out, ctypes.c_double))
+    return out
+
+
+def howl_route(score, c: float, lastwaslinear: np.ndarray) -> np.ndarray:
+    """Algorithm 1's routing for one step; ``lastwaslinear`` (uint8 [B]) is updated in place.
+    Returns route [B]: 0 = linear (non-tree) verification, 1 = tree from D_nospec, 2 = tree from D_spec."""
+    lib = _load()
+    score = _c(score, np.float32)
+    assert lastwaslinear.dtype == np.uint8 and lastwaslinear.flags["C_CONTIGUOUS"]
+    route = np.empty(score.shape[0], np.int32)
+    lib.owl_oracle_howl_route(score.shape[0], _p(score, ctypes.c_float), float(c), _p(lastwaslinear, ctypes.c_uint8),
+                              _p(route, ctypes.c_int32))
+    return route
+
+
+def prepare_hybrid(node_offsets, tree_parent, draft_tokens, ctx_lens, route, spec_token: int):
+    """Prepare(d) on a routed batch (route 0: chain as drafted; else [SPEC] leaves appended).  Returns
+    (node_offsets, tree_parent, draft_tokens, input_ids, position_ids) of the batch to verify."""
+    lib = _load()
+    node_offsets = _c(node_offsets, np.int32); tree_parent = _c(tree_parent, np.int32)
+    draft_tokens = _c(draft_tokens, np.int32); ctx_lens = _c(ctx_lens, np.int32); route = _c(route, np.int32)
+    B = node_offsets.shape[0] - 1
+    N = int(node_offsets[-1])
+    offs = np.empty(B + 1, np.int32)
+    par, drf, ids, pos = (np.empty(2 * N, np.int32) for _ in range(4))
+    i32 = ctypes.c_int32
+    rc = lib.owl_oracle_prepare_hybrid(B, _p(node_offsets, i32), _p(tree_parent, i32), _p(draft_tokens, i32), _p(ctx_lens, i32),
+                                       _p(route, i32), int(spec_token), _p(offs, i32), _p(par, i32), _p(drf, i32), _p(ids, i32),
+                                       _p(pos, i32))
+    if rc != 0:
+        raise ValueError(f"owl_oracle_prepare_hybrid failed with code {rc}")
+    M = int(offs[-1])
+    return offs, par[:M], drf[:M], ids[:M], pos[:M]

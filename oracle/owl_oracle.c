@@ -66,6 +66,21 @@ static double bf16_to_double(uint16_t h) {
     return (double)f;
 }
 
+/* IEEE binary16 to double, by the format's definition: sign, 5 exponent bits (bias 15), 10 fraction bits;
+ * exponent 0 = subnormal (fraction * 2^-24), exponent 31 = infinity or NaN. */
+static double f16_to_double(uint16_t h) {
+    const int sign = h >> 15, e = (h >> 10) & 31, f = h & 1023;
+    double v;
+    if (e == 0) v = ldexp((double)f, -24);
+    else if (e == 31) v = f ? NAN : INFINITY;
+    else v = ldexp((double)(1024 + f), e - 25);
+    return sign ? -v : v;
+}
+
+/* Element type of q / k_cache / v_cache: 0 = bf16 (the benchmark configurations), 1 = fp16 (the paper's own
+ * precision, Appendix "Inference Details"). */
+static double elem_to_double(uint16_t h, int is_f16) { return is_f16 ? f16_to_double(h) : bf16_to_double(h); }
+
 /* Sequence that owns packed node `n` (node_offsets has B+1 entries). */
 static int seq_of_node(const int32_t* node_offsets, int B, int n) {
     for (int b = 0; b < B; ++b)
@@ -105,7 +120,7 @@ static int tree_ok(const int32_t* parent, int n) {
  * n_rows must be N*Hq; otherwise rows r = (row_node[r], row_head[r]).
  * out is [n_rows, D] doubles, lse [n_rows] doubles.
  */
-int owl_oracle_attn(int B, int Hq, int Hkv, int D, int page_size, int max_pages_per_seq,
+static int attn_any(int is_f16, int B, int Hq, int Hkv, int D, int page_size, int max_pages_per_seq,
                     int num_pages, double sm_scale, const uint16_t* q, const uint16_t* k_cache,
                     const uint16_t* v_cache, const int32_t* block_table, const int32_t* ctx_lens,
                     const int32_t* node_offsets, const int32_t* tree_parent, int64_t n_rows,
@@ -157,7 +172,7 @@ int owl_oracle_attn(int B, int Hq, int Hkv, int D, int page_size, int max_pages_
                                           Hkv, page_size, D, h, vis[t]);
             if (!krow) { bad = 1; break; }
             double acc = 0.0;
-            for (int d = 0; d < D; ++d) acc += bf16_to_double(qrow[d]) * bf16_to_double(krow[d]);
+            for (int d = 0; d < D; ++d) acc += elem_to_double(qrow[d], is_f16) * elem_to_double(krow[d], is_f16);
             s[t] = sm_scale * acc;
             if (s[t] > m) m = s[t];
         }
@@ -175,13 +190,37 @@ int owl_oracle_attn(int B, int Hq, int Hkv, int D, int page_size, int max_pages_
             const uint16_t* vrow = kv_row(v_cache, block_table, b, max_pages_per_seq, num_pages,
                                           Hkv, page_size, D, h, vis[t]);
             const double p = exp(s[t] - m);
-            for (int d = 0; d < D; ++d) o[d] += p * bf16_to_double(vrow[d]);
+            for (int d = 0; d < D; ++d) o[d] += p * elem_to_double(vrow[d], is_f16);
         }
         for (int d = 0; d < D; ++d) o[d] /= Z;
         lse[r] = m + log(Z);
         free(vis); free(s);
     }
     return status;
+}
+
+int owl_oracle_attn(int B, int Hq, int Hkv, int D, int page_size, int max_pages_per_seq,
+                    int num_pages, double sm_scale, const uint16_t* q, const uint16_t* k_cache,
+                    const uint16_t* v_cache, const int32_t* block_table, const int32_t* ctx_lens,
+                    const int32_t* node_offsets, const int32_t* tree_parent, int64_t n_rows,
+                    const int32_t* row_node, const int32_t* row_head, double* out, double* lse) {
+    return attn_any(0, B, Hq, Hkv, D, page_size, max_pages_per_seq, num_pages, sm_scale, q, k_cache, v_cache, block_table,
+                    ctx_lens, node_offsets, tree_parent, n_rows, row_node, row_head, out, lse);
+}
+
+/* The same attention with q, k_cache and v_cache in fp16, the data type the paper ran in (Appendix "Inference Details"). */
+int owl_oracle_attn_f16(int B, int Hq, int Hkv, int D, int page_size, int max_pages_per_seq,
+                        int num_pages, double sm_scale, const uint16_t* q, const uint16_t* k_cache,
+                        const uint16_t* v_cache, const int32_t* block_table, const int32_t* ctx_lens,
+                        const int32_t* node_offsets, const int32_t* tree_parent, int64_t n_rows,
+                        const int32_t* row_node, const int32_t* row_head, double* out, double* lse) {
+    return attn_any(1, B, Hq, Hkv, D, page_size, max_pages_per_seq, num_pages, sm_scale, q, k_cache, v_cache, block_table,
+                    ctx_lens, node_offsets, tree_parent, n_rows, row_node, row_head, out, lse);
+}
+
+/* Decoders exposed for their own pin (every bit pattern against a library conversion). */
+void owl_oracle_decode16(const uint16_t* in, int64_t count, int is_f16, double* out) {
+    for (int64_t i = 0; i < count; ++i) out[i] = elem_to_double(in[i], is_f16);
 }
 
 /*
@@ -340,6 +379,65 @@ int owl_oracle_kv_commit(int B, int Hkv, int D, int page_size, int max_pages_per
             }
         free(tmp);
         ctx_lens[b] = (int32_t)(L + a);
+    }
+    return ORACLE_OK;
+}
+
+/*
+ * The routing of Algorithm 1 (Section 3.2.3), one decision per sequence and step.  `score` is the non-tree
+ * drafter's estimate of its acceptance length, c the threshold (the paper sets c = 9, the longest acceptance
+ * the tree drafter can reach, Appendix "Inference Details").
+ *   score > c            -> non-tree verification of the chain as drafted, no [SPEC]; lastwaslinear <- true
+ *   else, lastwaslinear  -> tree from the drafter trained WITHOUT [SPEC] (the last step produced no [SPEC]
+ *                           hidden state); lastwaslinear <- false
+ *   else                 -> tree from the drafter trained WITH [SPEC]
+ * Either tree is verified with [SPEC] leaves appended.  route: 0 = linear, 1 = tree / D_nospec, 2 = tree / D_spec.
+ */
+void owl_oracle_howl_route(int B, const float* score, float c, uint8_t* lastwaslinear, int32_t* route) {
+    for (int b = 0; b < B; ++b) {
+        if (score[b] > c) {
+            lastwaslinear[b] = 1;
+            route[b] = 0;
+        } else if (lastwaslinear[b]) {
+            route[b] = 1;
+            lastwaslinear[b] = 0;
+        } else {
+            route[b] = 2;
+        }
+    }
+}
+
+/*
+ * Prepare(d) on a routed batch: a sequence routed to non-tree verification (route 0) keeps its chain as drafted
+ * ("we do not append any [SPEC] to the input in this case", Section 3.2.3); every other sequence gets one [SPEC]
+ * leaf per node as in owl_oracle_prepare_spec.  Outputs are packed sequence after sequence (n or 2n nodes).
+ */
+int owl_oracle_prepare_hybrid(int B, const int32_t* node_offsets, const int32_t* tree_parent,
+                              const int32_t* draft_tokens, const int32_t* ctx_lens, const int32_t* route,
+                              int32_t spec_token, int32_t* out_offsets, int32_t* out_parent, int32_t* out_draft,
+                              int32_t* out_input_ids, int32_t* out_position) {
+    out_offsets[0] = 0;
+    for (int b = 0; b < B; ++b) {
+        const int base = node_offsets[b], n = node_offsets[b + 1] - base;
+        const int32_t* parent = tree_parent + base;
+        if (!tree_ok(parent, n)) return ORACLE_BAD_TREE;
+        const int ob = out_offsets[b];
+        const int with_spec = route[b] != 0;
+        out_offsets[b + 1] = ob + (with_spec ? 2 * n : n);
+        for (int j = 0; j < n; ++j) {
+            int depth = 0;
+            for (int c = j; parent[c] >= 0; c = parent[c]) ++depth;
+            out_parent[ob + j] = parent[j];
+            out_draft[ob + j] = draft_tokens[base + j];
+            out_input_ids[ob + j] = draft_tokens[base + j];
+            out_position[ob + j] = ctx_lens[b] + depth;
+            if (with_spec) {
+                out_parent[ob + n + j] = j;
+                out_draft[ob + n + j] = -1;
+                out_input_ids[ob + n + j] = spec_token;
+                out_position[ob + n + j] = ctx_lens[b] + depth + 1;
+            }
+        }
     }
     return ORACLE_OK;
 }
