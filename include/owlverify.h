@@ -120,6 +120,16 @@ int owl_verify_attn(owl_ctx* ctx, const owl_dims* dims, const void* q, const voi
                     void* stream);
 
 /*
+ * owl_verify_attn with q, k_cache, v_cache and out in fp16 (IEEE binary16) instead of bf16: the data type the
+ * paper ran in (Appendix "Inference Details": "use fp16 data type").  Same layouts, same semantics, same
+ * tolerances; the softmax weights are rounded to fp16 before the second product, lse stays fp32.
+ */
+int owl_verify_attn_f16(owl_ctx* ctx, const owl_dims* dims, const void* q, const void* k_cache,
+                        const void* v_cache, const int32_t* block_table, const int32_t* ctx_lens,
+                        const int32_t* node_offsets, const int32_t* tree_parent, void* out, float* lse,
+                        void* stream);
+
+/*
  * Greedy tree acceptance (Introduction: accepted tokens keep the target's output
  * distribution; Figure 1 caption: acceptance length; Section 3.2.2: paths start at the
  * root t_{N+1}, [SPEC] leaves are never candidate tokens).
@@ -176,6 +186,40 @@ int owl_prepare_spec_tree(owl_ctx* ctx, const owl_dims* dims, const int32_t* nod
                           int32_t spec_token, int32_t* out_node_offsets, int32_t* out_tree_parent,
                           int32_t* out_draft_tokens, int32_t* out_input_ids, int32_t* out_position_ids,
                           void* stream);
+
+/*
+ * The routing decision of Algorithm 1 (Section 3.2.3), once per sequence and decoding step.  HOST arrays: the
+ * score comes from the non-tree drafter, which runs on the CPU, and the decision steers host control flow
+ * (which drafter runs next).  score[b] = that drafter's estimate of its acceptance length; c = the threshold
+ * (the paper uses 9, the longest acceptance its depth-8 trees allow, Appendix "Inference Details");
+ * lastwaslinear[b] (in/out, 0 before the first step) = whether the sequence's previous step was verified as a
+ * chain.  route[b] (out):
+ *   OWL_ROUTE_LINEAR       score > c: verify the non-tree drafter's chain as drafted, no [SPEC] appended
+ *   OWL_ROUTE_TREE_NOSPEC  score <= c after a linear step: tree from the drafter trained without [SPEC]
+ *                          (the linear step produced no [SPEC] hidden state)
+ *   OWL_ROUTE_TREE_SPEC    score <= c otherwise: tree from the drafter trained with [SPEC]
+ * Both tree routes are verified with [SPEC] leaves (owl_prepare_hybrid).  A NaN score takes a tree route.
+ * Returns OWL_ERR_INVALID_ARG for batch < 1, a NULL pointer or a NaN threshold.
+ */
+#define OWL_ROUTE_LINEAR 0
+#define OWL_ROUTE_TREE_NOSPEC 1
+#define OWL_ROUTE_TREE_SPEC 2
+int owl_howl_route(int32_t batch, const float* score, float c, uint8_t* lastwaslinear, int32_t* route);
+
+/*
+ * Prepare(d) on a routed batch (Algorithm 1; Section 3.2.3: on the non-tree route "we do not append any [SPEC]").
+ * As owl_prepare_spec_tree, with route (device int32 [B], the values owl_howl_route gives): a sequence with
+ * route OWL_ROUTE_LINEAR keeps its n nodes as drafted (position ids ctx_len + depth, input ids = tokens), every
+ * other sequence becomes 2n nodes with [SPEC] leaves.  The sequences' outputs are packed one after the other:
+ * out_node_offsets [B+1] is the running sum of n or 2n; the other outputs need room for 2 * total_nodes entries.
+ * dims->max_nodes bounds the DRAFTED nodes of a sequence: up to 64 on the linear route, up to 32 on a tree route
+ * (a longer tree sets OWL_ERR_BAD_TREE on the device and leaves that sequence unwritten).
+ */
+int owl_prepare_hybrid(owl_ctx* ctx, const owl_dims* dims, const int32_t* node_offsets,
+                       const int32_t* tree_parent, const int32_t* draft_tokens, const int32_t* ctx_lens,
+                       const int32_t* route, int32_t spec_token, int32_t* out_node_offsets,
+                       int32_t* out_tree_parent, int32_t* out_draft_tokens, int32_t* out_input_ids,
+                       int32_t* out_position_ids, void* stream);
 
 /*
  * Commit of the accepted tokens to the cache (Algorithm 1: "l <- l; d", "N <- N + |d|").  During verification

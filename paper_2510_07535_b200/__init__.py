@@ -6,5 +6,5 @@ acceptance, as hand-written sm_100a CUDA kernels behind the C ABI of ``include/o
 ``build`` compiles the library.  Nothing here computes on the CPU.
 """
 from . import workloads  # noqa: F401
-from .binding import (OwlContext, OwlDims, OwlError, load_library, make_dims, owl_tree_accept_static,  # noqa: F401
-                      status_string)
+from .binding import (OwlContext, OwlDims, OwlError, load_library, make_dims, owl_howl_route,  # noqa: F401
+                      owl_tree_accept_static, status_string)

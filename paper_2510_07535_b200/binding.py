@@ -48,12 +48,18 @@ def load_library() -> ctypes.CDLL:
     lib.owl_destroy.argtypes = [vp]
     lib.owl_verify_attn.restype = i32
     lib.owl_verify_attn.argtypes = [vp, dp] + [vp] * 10
+    lib.owl_verify_attn_f16.restype = i32
+    lib.owl_verify_attn_f16.argtypes = [vp, dp] + [vp] * 10
     lib.owl_tree_accept.restype = i32
     lib.owl_tree_accept.argtypes = [vp, dp] + [vp] * 9
     lib.owl_tree_accept_spec.restype = i32
     lib.owl_tree_accept_spec.argtypes = [vp, dp] + [vp] * 10
     lib.owl_prepare_spec_tree.restype = i32
     lib.owl_prepare_spec_tree.argtypes = [vp, dp] + [vp] * 4 + [ctypes.c_int32] + [vp] * 6
+    lib.owl_prepare_hybrid.restype = i32
+    lib.owl_prepare_hybrid.argtypes = [vp, dp] + [vp] * 5 + [ctypes.c_int32] + [vp] * 6
+    lib.owl_howl_route.restype = i32
+    lib.owl_howl_route.argtypes = [ctypes.c_int32, vp, ctypes.c_float, vp, vp]
     lib.owl_kv_commit.restype = i32
     lib.owl_kv_commit.argtypes = [vp, dp] + [vp] * 8
     lib.owl_tree_accept_static.restype = i32
@@ -137,6 +143,19 @@ class OwlContext:
             raise OwlError(rc, "owl_verify_attn", self.last_error())
         return rc
 
+    def owl_verify_attn_f16(self, dims: OwlDims, q, k_cache, v_cache, block_table, ctx_lens, node_offsets, tree_parent,
+                            out, lse, check: bool = True) -> int:
+        dev = self.device
+        h = torch.float16
+        rc = self.lib.owl_verify_attn_f16(
+            self._h, ctypes.byref(dims), _ptr(q, h, dev, "q"), _ptr(k_cache, h, dev, "k_cache"), _ptr(v_cache, h, dev, "v_cache"),
+            _ptr(block_table, torch.int32, dev, "block_table"), _ptr(ctx_lens, torch.int32, dev, "ctx_lens"),
+            _ptr(node_offsets, torch.int32, dev, "node_offsets"), _ptr(tree_parent, torch.int32, dev, "tree_parent"),
+            _ptr(out, h, dev, "out"), _ptr(lse, torch.float32, dev, "lse"), _stream(dev))
+        if check and rc != OWL_OK:
+            raise OwlError(rc, "owl_verify_attn_f16", self.last_error())
+        return rc
+
     def owl_tree_accept(self, dims: OwlDims, logits, draft_tokens, node_offsets, tree_parent, accept_len, accept_path,
                         bonus_token, node_argmax=None, check: bool = True) -> int:
         dev = self.device
@@ -177,6 +196,21 @@ class OwlContext:
             _ptr(out_position_ids, i32, dev, "out_position_ids"), _stream(dev))
         if check and rc != OWL_OK:
             raise OwlError(rc, "owl_prepare_spec_tree", self.last_error())
+        return rc
+
+    def owl_prepare_hybrid(self, dims: OwlDims, node_offsets, tree_parent, draft_tokens, ctx_lens, route, spec_token: int,
+                           out_node_offsets, out_tree_parent, out_draft_tokens, out_input_ids, out_position_ids,
+                           check: bool = True) -> int:
+        dev = self.device
+        i32 = torch.int32
+        rc = self.lib.owl_prepare_hybrid(
+            self._h, ctypes.byref(dims), _ptr(node_offsets, i32, dev, "node_offsets"), _ptr(tree_parent, i32, dev, "tree_parent"),
+            _ptr(draft_tokens, i32, dev, "draft_tokens"), _ptr(ctx_lens, i32, dev, "ctx_lens"), _ptr(route, i32, dev, "route"),
+            int(spec_token), _ptr(out_node_offsets, i32, dev, "out_node_offsets"), _ptr(out_tree_parent, i32, dev, "out_tree_parent"),
+            _ptr(out_draft_tokens, i32, dev, "out_draft_tokens"), _ptr(out_input_ids, i32, dev, "out_input_ids"),
+            _ptr(out_position_ids, i32, dev, "out_position_ids"), _stream(dev))
+        if check and rc != OWL_OK:
+            raise OwlError(rc, "owl_prepare_hybrid", self.last_error())
         return rc
 
     def owl_kv_commit(self, dims: OwlDims, k_cache, v_cache, block_table, ctx_lens, node_offsets, accept_len, accept_path,
@@ -270,6 +304,22 @@ def owl_tree_accept_static(dims: OwlDims, logits, draft_tokens, node_offsets, tr
     if check and rc != OWL_OK:
         raise OwlError(rc, "owl_tree_accept_static")
     return rc
+
+
+def owl_howl_route(score, c: float, lastwaslinear):
+    """Algorithm 1's routing on HOST numpy arrays: score float32 [B]; lastwaslinear uint8 [B], updated in place.
+    Returns route int32 [B] (0 linear, 1 tree from D_nospec, 2 tree from D_spec)."""
+    import numpy as np
+    lib = load_library()
+    score = np.ascontiguousarray(score, dtype=np.float32)
+    if lastwaslinear.dtype != np.uint8 or not lastwaslinear.flags["C_CONTIGUOUS"]:
+        raise TypeError("lastwaslinear: contiguous uint8 array expected (it is updated in place)")
+    route = np.empty(score.shape[0], np.int32)
+    rc = lib.owl_howl_route(score.shape[0], score.ctypes.data_as(ctypes.c_void_p), float(c),
+                            lastwaslinear.ctypes.data_as(ctypes.c_void_p), route.ctypes.data_as(ctypes.c_void_p))
+    if rc != OWL_OK:
+        raise OwlError(rc, "owl_howl_route")
+    return route
 
 
 def status_string(code: int) -> str:

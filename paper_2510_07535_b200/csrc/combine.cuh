@@ -3,6 +3,8 @@
 // One warp per output row (packed node, query head); each lane owns 4 of the 128 output channels.
 #pragma once
 
+#include <cuda_fp16.h>
+
 #include "owl_common.cuh"
 #include "accept.cuh"
 
@@ -134,11 +136,16 @@ __global__ void __launch_bounds__(kCombineWarps * 32) combine_sched_kernel(const
     }
     if (bad_epoch == p.epoch) return;              // the pass found a bad tree or page in this sequence: no output
     const float inv = sum > 0.f ? 1.f / sum : 0.f;
-    __nv_bfloat162 lo2 = __floats2bfloat162_rn(acc.x * inv, acc.y * inv);
-    __nv_bfloat162 hi2 = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
     uint2 pk;
-    pk.x = *reinterpret_cast<uint32_t*>(&lo2);
-    pk.y = *reinterpret_cast<uint32_t*>(&hi2);
+    if (p.f16) {
+        __half2 lo2 = __floats2half2_rn(acc.x * inv, acc.y * inv), hi2 = __floats2half2_rn(acc.z * inv, acc.w * inv);
+        pk.x = *reinterpret_cast<uint32_t*>(&lo2);
+        pk.y = *reinterpret_cast<uint32_t*>(&hi2);
+    } else {
+        __nv_bfloat162 lo2 = __floats2bfloat162_rn(acc.x * inv, acc.y * inv), hi2 = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
+        pk.x = *reinterpret_cast<uint32_t*>(&lo2);
+        pk.y = *reinterpret_cast<uint32_t*>(&hi2);
+    }
     *reinterpret_cast<uint2*>(p.out + row_id * kHeadDim + lane * 4) = pk;
     if (p.lse && lane == 0) p.lse[row_id] = sum > 0.f ? mx + logf(sum) : -INFINITY;
 }

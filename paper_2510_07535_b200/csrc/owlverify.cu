@@ -45,6 +45,7 @@ struct owl_ctx {
         const void* k = nullptr;
         const void* v = nullptr;
         int pages = 0, heads = 0, page_size = 0;
+        bool fp16 = false;
         uint64_t used = 0;
     } maps[kMapCacheEntries];
     uint64_t map_clock = 0;
@@ -91,20 +92,28 @@ cudaError_t launch_dependent(void (*kernel)(Args...), dim3 grid, dim3 block, cud
     return cudaLaunchKernelEx(&cfg, kernel, args...);
 }
 
-// The attention kernel's instances: [more than 32 sequences][units above 128 rows][logits scan fused in]
+// The attention kernel's instances: [more than 32 sequences][units above 128 rows][logits scan fused in], bf16;
+// and the fp16 ones (attention only): [more than 32 sequences][units above 128 rows]
 using UmmaKernel = void (*)(AttnParams, CUtensorMap, CUtensorMap, AcceptParams);
-UmmaKernel umma_kernel(bool many, bool wide, bool fused) {
+UmmaKernel umma_kernel(bool many, bool wide, bool fused, bool fp16) {
+    using namespace umma_path;
     static const UmmaKernel table[2][2][2] = {
-        {{umma_path::verify_attn_umma_kernel<false, false, false>, umma_path::verify_attn_umma_kernel<false, false, true>},
-         {umma_path::verify_attn_umma_kernel<false, true, false>, umma_path::verify_attn_umma_kernel<false, true, true>}},
-        {{umma_path::verify_attn_umma_kernel<true, false, false>, umma_path::verify_attn_umma_kernel<true, false, true>},
-         {umma_path::verify_attn_umma_kernel<true, true, false>, umma_path::verify_attn_umma_kernel<true, true, true>}}};
-    return table[many][wide][fused];
+        {{verify_attn_umma_kernel<false, false, false, false>, verify_attn_umma_kernel<false, false, true, false>},
+         {verify_attn_umma_kernel<false, true, false, false>, verify_attn_umma_kernel<false, true, true, false>}},
+        {{verify_attn_umma_kernel<true, false, false, false>, verify_attn_umma_kernel<true, false, true, false>},
+         {verify_attn_umma_kernel<true, true, false, false>, verify_attn_umma_kernel<true, true, true, false>}}};
+    static const UmmaKernel table16[2][2] = {
+        {verify_attn_umma_kernel<false, false, false, true>, verify_attn_umma_kernel<false, true, false, true>},
+        {verify_attn_umma_kernel<true, false, false, true>, verify_attn_umma_kernel<true, true, false, true>}};
+    return fp16 ? table16[many][wide] : table[many][wide][fused];
 }
 bool set_umma_smem_attr() {
     bool ok = true;
     for (int i = 0; i < 8; ++i)
-        ok = ok && cudaFuncSetAttribute(umma_kernel(i & 4, i & 2, i & 1), cudaFuncAttributeMaxDynamicSharedMemorySize,
+        ok = ok && cudaFuncSetAttribute(umma_kernel(i & 4, i & 2, i & 1, false), cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        umma_path::kSmemBytes) == cudaSuccess;
+    for (int i = 0; i < 4; ++i)
+        ok = ok && cudaFuncSetAttribute(umma_kernel(i & 2, i & 1, false, true), cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         umma_path::kSmemBytes) == cudaSuccess;
     return ok;
 }
@@ -270,7 +279,8 @@ int owl_destroy(owl_ctx* ctx) {
 // spare warps and the acceptance walk in the merge kernel, two launches for the whole step.
 static int verify_attn_impl(owl_ctx* ctx, const owl_dims* d, const void* q, const void* k_cache, const void* v_cache,
                             const int32_t* block_table, const int32_t* ctx_lens, const int32_t* node_offsets,
-                            const int32_t* tree_parent, void* out, float* lse, void* stream_, const AcceptParams* ap) {
+                            const int32_t* tree_parent, void* out, float* lse, void* stream_, const AcceptParams* ap,
+                            bool fp16 = false) {
     if (!ctx) return OWL_ERR_INVALID_ARG;
     int rc = check_dims(d, true, false);
     if (rc != OWL_OK) return rc;
@@ -314,18 +324,19 @@ static int verify_attn_impl(owl_ctx* ctx, const owl_dims* d, const void* q, cons
     p.rows_per_slot = ctx->rows_per_slot;
     p.num_ctas = ctx->num_ctas;
     p.sm_scale = d->sm_scale;
+    p.f16 = fp16 ? 1 : 0;
 
     owl_ctx::MapEntry* maps = nullptr;
     {
         owl_ctx::MapEntry* lru = &ctx->maps[0];
         for (auto& m : ctx->maps) {
             if (m.k == k_cache && m.v == v_cache && m.pages == d->num_pages && m.heads == d->num_kv_heads &&
-                m.page_size == d->page_size) { maps = &m; break; }
+                m.page_size == d->page_size && m.fp16 == fp16) { maps = &m; break; }
             if (m.used < lru->used) lru = &m;
         }
         if (!maps) {
-            const int rk = make_kv_tensor_map(ctx->encode, &lru->kmap, k_cache, d->num_pages, d->num_kv_heads, d->page_size);
-            const int rv = make_kv_tensor_map(ctx->encode, &lru->vmap, v_cache, d->num_pages, d->num_kv_heads, d->page_size);
+            const int rk = make_kv_tensor_map(ctx->encode, &lru->kmap, k_cache, d->num_pages, d->num_kv_heads, d->page_size, fp16);
+            const int rv = make_kv_tensor_map(ctx->encode, &lru->vmap, v_cache, d->num_pages, d->num_kv_heads, d->page_size, fp16);
             if (rk != 0 || rv != 0) {
                 lru->k = lru->v = nullptr;
                 lru->used = 0;
@@ -333,7 +344,7 @@ static int verify_attn_impl(owl_ctx* ctx, const owl_dims* d, const void* q, cons
                 return OWL_ERR_CUDA;
             }
             lru->k = k_cache; lru->v = v_cache;
-            lru->pages = d->num_pages; lru->heads = d->num_kv_heads; lru->page_size = d->page_size;
+            lru->pages = d->num_pages; lru->heads = d->num_kv_heads; lru->page_size = d->page_size; lru->fp16 = fp16;
             maps = lru;
         }
         maps->used = ++ctx->map_clock;
@@ -356,7 +367,7 @@ static int verify_attn_impl(owl_ctx* ctx, const owl_dims* d, const void* q, cons
         // the instance that holds only this call's case: block-wide schedule above 32 sequences, the two-row-block
         // mode only if a unit (G * max_nodes rows at most) can exceed 128 rows, the logits scan only in a step
         const bool many = d->batch > 32, wide = G * d->max_nodes > 128;
-        cudaLaunchKernelEx(&cfg, umma_kernel(many, wide, ap != nullptr), p, maps->kmap, maps->vmap, ap ? *ap : AcceptParams{});
+        cudaLaunchKernelEx(&cfg, umma_kernel(many, wide, ap != nullptr, fp16), p, maps->kmap, maps->vmap, ap ? *ap : AcceptParams{});
     }
     ++ctx->launches;
     if (ctx->profiling) cudaEventRecord(ctx->ev[1], stream);
@@ -379,6 +390,13 @@ int owl_verify_attn(owl_ctx* ctx, const owl_dims* d, const void* q, const void* 
                     const int32_t* tree_parent, void* out, float* lse, void* stream_) {
     return verify_attn_impl(ctx, d, q, k_cache, v_cache, block_table, ctx_lens, node_offsets, tree_parent, out, lse, stream_,
                             nullptr);
+}
+
+int owl_verify_attn_f16(owl_ctx* ctx, const owl_dims* d, const void* q, const void* k_cache, const void* v_cache,
+                        const int32_t* block_table, const int32_t* ctx_lens, const int32_t* node_offsets,
+                        const int32_t* tree_parent, void* out, float* lse, void* stream_) {
+    return verify_attn_impl(ctx, d, q, k_cache, v_cache, block_table, ctx_lens, node_offsets, tree_parent, out, lse, stream_,
+                            nullptr, true);
 }
 
 // Argument checks of the acceptance and its kernel parameters (everything but the counters of the stand-alone kernel).
@@ -458,21 +476,24 @@ int owl_tree_accept_spec(owl_ctx* ctx, const owl_dims* d, const float* logits, c
                             spec_node, node_argmax, stream_);
 }
 
-int owl_prepare_spec_tree(owl_ctx* ctx, const owl_dims* d, const int32_t* node_offsets, const int32_t* tree_parent,
-                          const int32_t* draft_tokens, const int32_t* ctx_lens, int32_t spec_token,
-                          int32_t* out_node_offsets, int32_t* out_tree_parent, int32_t* out_draft_tokens,
-                          int32_t* out_input_ids, int32_t* out_position_ids, void* stream_) {
+static int prepare_impl(owl_ctx* ctx, const owl_dims* d, const int32_t* node_offsets, const int32_t* tree_parent,
+                        const int32_t* draft_tokens, const int32_t* ctx_lens, const int32_t* route, bool routed,
+                        int32_t spec_token, int32_t* out_node_offsets, int32_t* out_tree_parent,
+                        int32_t* out_draft_tokens, int32_t* out_input_ids, int32_t* out_position_ids, void* stream_) {
     if (!ctx) return OWL_ERR_INVALID_ARG;
     int rc = check_dims(d, false, false);
     if (rc != OWL_OK) return rc;
-    if (2 * d->max_nodes > kMaxNodes) return OWL_ERR_UNSUPPORTED;        // the prepared tree has twice the nodes
+    // the prepared tree of a sequence with [SPEC] leaves has twice the nodes; a routed batch may also hold chains
+    // of up to 64 nodes (kept as drafted), which the device sorts out per sequence
+    if (!routed && 2 * d->max_nodes > kMaxNodes) return OWL_ERR_UNSUPPORTED;
     if (!tree_parent || !draft_tokens || !ctx_lens || !out_node_offsets || !out_tree_parent || !out_draft_tokens ||
-        !out_input_ids || !out_position_ids)
+        !out_input_ids || !out_position_ids || (routed && !route))
         return OWL_ERR_INVALID_ARG;
     if (!node_offsets && d->total_nodes % d->batch != 0) return OWL_ERR_INVALID_ARG;
     DeviceGuard guard(ctx->device);
     PrepareParams p{};
     p.node_offsets = node_offsets; p.tree_parent = tree_parent; p.draft_tokens = draft_tokens; p.ctx_lens = ctx_lens;
+    p.route = route;
     p.out_offsets = out_node_offsets; p.out_parent = out_tree_parent; p.out_draft = out_draft_tokens;
     p.out_input_ids = out_input_ids; p.out_position = out_position_ids;
     p.status = ctx->status;
@@ -482,6 +503,32 @@ int owl_prepare_spec_tree(owl_ctx* ctx, const owl_dims* d, const int32_t* node_o
     ++ctx->launches;
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(ctx, e, "owl_prepare_spec_tree launch");
+    return OWL_OK;
+}
+
+int owl_prepare_spec_tree(owl_ctx* ctx, const owl_dims* d, const int32_t* node_offsets, const int32_t* tree_parent,
+                          const int32_t* draft_tokens, const int32_t* ctx_lens, int32_t spec_token,
+                          int32_t* out_node_offsets, int32_t* out_tree_parent, int32_t* out_draft_tokens,
+                          int32_t* out_input_ids, int32_t* out_position_ids, void* stream_) {
+    return prepare_impl(ctx, d, node_offsets, tree_parent, draft_tokens, ctx_lens, nullptr, false, spec_token, out_node_offsets,
+                        out_tree_parent, out_draft_tokens, out_input_ids, out_position_ids, stream_);
+}
+
+int owl_prepare_hybrid(owl_ctx* ctx, const owl_dims* d, const int32_t* node_offsets, const int32_t* tree_parent,
+                       const int32_t* draft_tokens, const int32_t* ctx_lens, const int32_t* route, int32_t spec_token,
+                       int32_t* out_node_offsets, int32_t* out_tree_parent, int32_t* out_draft_tokens,
+                       int32_t* out_input_ids, int32_t* out_position_ids, void* stream_) {
+    return prepare_impl(ctx, d, node_offsets, tree_parent, draft_tokens, ctx_lens, route, true, spec_token, out_node_offsets,
+                        out_tree_parent, out_draft_tokens, out_input_ids, out_position_ids, stream_);
+}
+
+int owl_howl_route(int32_t batch, const float* score, float c, uint8_t* lastwaslinear, int32_t* route) {
+    if (batch < 1 || !score || !lastwaslinear || !route || c != c) return OWL_ERR_INVALID_ARG;
+    for (int32_t b = 0; b < batch; ++b) {
+        const bool linear = score[b] > c;                      // a NaN score compares false: the tree drafter is used
+        route[b] = linear ? OWL_ROUTE_LINEAR : (lastwaslinear[b] ? OWL_ROUTE_TREE_NOSPEC : OWL_ROUTE_TREE_SPEC);
+        lastwaslinear[b] = linear ? 1 : 0;
+    }
     return OWL_OK;
 }
 

@@ -148,12 +148,13 @@ __device__ __forceinline__ uint64_t umma_smem_desc_sw128(uint32_t smem_addr, uin
     return d;
 }
 
-// Instruction descriptor of tcgen05.mma.kind::f16 with bf16 A and B, fp32 accumulator:
-// D format (1 = f32) in bits [4,6), A/B format (1 = bf16) in [7,10) / [10,13), A/B major-ness
-// (0 = K-major, 1 = MN-major) in bits 15 / 16, N >> 3 in [17,23), M >> 4 in [24,29).
-__host__ __device__ constexpr uint32_t umma_idesc_bf16(int m, int n, int a_mn_major, int b_mn_major) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn_major << 15) | ((uint32_t)b_mn_major << 16) |
-           ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+// Instruction descriptor of tcgen05.mma.kind::f16 with A and B both bf16 or both fp16 (the two operands of one
+// instruction always have the same type), fp32 accumulator: D format (1 = f32) in bits [4,6), A/B format
+// (0 = fp16, 1 = bf16) in [7,10) / [10,13), A/B major-ness (0 = K-major, 1 = MN-major) in bits 15 / 16,
+// N >> 3 in [17,23), M >> 4 in [24,29).
+__host__ __device__ constexpr uint32_t umma_idesc_16bit(int m, int n, int a_mn_major, int b_mn_major, bool fp16) {
+    return (1u << 4) | ((fp16 ? 0u : 1u) << 7) | ((fp16 ? 0u : 1u) << 10) | ((uint32_t)a_mn_major << 15) |
+           ((uint32_t)b_mn_major << 16) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
 // D[tmem] (+)= A[smem] * B[smem]; issued by one thread.

@@ -15,7 +15,8 @@ struct PrepareParams {
     const int32_t* tree_parent;
     const int32_t* draft_tokens;
     const int32_t* ctx_lens;
-    int32_t* out_offsets;          // [B + 1] = 2 x the drafted offsets
+    const int32_t* route;          // may be null (every sequence gets [SPEC] leaves); route[b] == 0: chain kept as drafted
+    int32_t* out_offsets;          // [B + 1]: running sum of the output node counts (n or 2 n per sequence)
     int32_t* out_parent;           // [2 N]
     int32_t* out_draft;            // [2 N], -1 for a [SPEC] leaf
     int32_t* out_input_ids;        // [2 N], spec_token for a [SPEC] leaf
@@ -25,19 +26,39 @@ struct PrepareParams {
 };
 
 constexpr int kPrepareThreads = 64;
-static_assert(kPrepareThreads >= kMaxNodes / 2, "one thread per drafted node");
+static_assert(kPrepareThreads >= kMaxNodes, "one thread per drafted node");
 
 // One CTA per sequence, one thread per drafted node j: node j keeps its place, its [SPEC] leaf is node n + j.
+// With a route array, a sequence routed to non-tree verification (route 0) keeps its chain without any [SPEC]
+// (Section 3.2.3); the sequences' outputs are packed one after the other, so every CTA first sums the output
+// node counts of the sequences before its own.
 __global__ void __launch_bounds__(kPrepareThreads) prepare_spec_kernel(const PrepareParams p) {
     const int b = blockIdx.x, j = threadIdx.x;
     const int base = p.node_offsets ? p.node_offsets[b] : b * p.nodes_uniform;
     const int n = p.node_offsets ? p.node_offsets[b + 1] - base : p.nodes_uniform;
-    __shared__ int s_parent[kMaxNodes / 2];
-    __shared__ int s_bad;
+    const bool with_spec = !p.route || p.route[b] != 0;
+    __shared__ int s_parent[kMaxNodes];
+    __shared__ int s_bad, s_before;
+    if (j == 0) { s_bad = 0; s_before = 0; }
+    __syncthreads();
+    long long before = 0;            // output nodes of sequences 0 .. b-1
+    if (p.route) {
+        for (int c = j; c < b; c += kPrepareThreads) {
+            const int nc = p.node_offsets ? p.node_offsets[c + 1] - p.node_offsets[c] : p.nodes_uniform;
+            before += p.route[c] != 0 ? 2 * nc : nc;
+        }
+        atomicAdd(&s_before, (int)before);
+    } else if (j == 0) {
+        s_before = 2 * base;
+    }
+    __syncthreads();
+    const int ob = s_before, count = with_spec ? 2 * n : n;
     if (j == 0) {
-        s_bad = (n < 1 || n > p.max_nodes || 2 * n > kMaxNodes || base < 0 || base + n > p.total_nodes) ? 1 : 0;
+        // the outputs hold 2 * total_nodes entries: whatever the offsets say, nothing is written outside them
+        s_bad = (n < 1 || n > p.max_nodes || count > kMaxNodes || base < 0 || base + n > p.total_nodes || ob < 0 ||
+                 (long long)ob + count > 2ll * p.total_nodes) ? 1 : 0;
         if (b == 0) p.out_offsets[0] = 0;
-        p.out_offsets[b + 1] = 2 * (base + n);
+        p.out_offsets[b + 1] = ob + count;
     }
     __syncthreads();
     if (s_bad) { if (j == 0) report(p.status, kErrBadTree); return; }
@@ -53,15 +74,17 @@ __global__ void __launch_bounds__(kPrepareThreads) prepare_spec_kernel(const Pre
         int depth = 0;
         for (int c = j; s_parent[c] >= 0 && depth < kMaxNodes; c = s_parent[c]) ++depth;
         const int L = p.ctx_lens[b], tok = p.draft_tokens[base + j];
-        const int o = 2 * base + j;
+        const int o = ob + j;
         p.out_parent[o] = parent;
         p.out_draft[o] = tok;
         p.out_input_ids[o] = tok;
         p.out_position[o] = L + depth;
-        p.out_parent[o + n] = j;
-        p.out_draft[o + n] = -1;
-        p.out_input_ids[o + n] = p.spec_token;
-        p.out_position[o + n] = L + depth + 1;
+        if (with_spec) {
+            p.out_parent[o + n] = j;
+            p.out_draft[o + n] = -1;
+            p.out_input_ids[o + n] = p.spec_token;
+            p.out_position[o + n] = L + depth + 1;
+        }
     }
 }
 

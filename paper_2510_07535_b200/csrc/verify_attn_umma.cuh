@@ -33,6 +33,8 @@
 // the status word reports OWL_ERR_TIMEOUT.
 #pragma once
 
+#include <cuda_fp16.h>
+
 #include <type_traits>
 
 #include "kv_tensor_map.cuh"
@@ -322,12 +324,12 @@ __device__ __forceinline__ void producer_loop(const AttnParams& p, const CUtenso
 //    wait for the tile itself);
 //  * the iterations in which both streams have both products to issue run in a loop of their own without
 //    per-product conditions; the first and the last ones of a segment take the general form.
-template <bool kWide>
+template <bool kWide, bool kF16>
 __device__ __forceinline__ void mma_loop(const AttnParams& p, Aux* aux, uint32_t smem_base, uint32_t tmem, Walker w) {
     constexpr unsigned kAll = 0xffffffffu;
     volatile int* abort_flag = &aux->abort_flag;
-    constexpr uint32_t idesc_qk = umma_idesc_bf16(128, kTileKeys, 0, 0);
-    constexpr uint32_t idesc_pv = umma_idesc_bf16(128, kHeadDim, 0, 1);
+    constexpr uint32_t idesc_qk = umma_idesc_16bit(128, kTileKeys, 0, 0, kF16);
+    constexpr uint32_t idesc_pv = umma_idesc_16bit(128, kHeadDim, 0, 1, kF16);
     const uint32_t ring = smem_base + kRingOff;
     const uint32_t elected = elect_one() ? 1u : 0u;
     // descriptors of Q block 0 and of ring slot 0; those of the other blocks and slots differ in the start-address
@@ -482,7 +484,15 @@ __device__ __forceinline__ float max3(float a, float b, float c) { return fmaxf(
 // whose rows are consecutive (part_row0 = row of lane 0).
 constexpr int kStageStride = 36;                     // floats per staged row: 16-byte aligned, conflict-free
 constexpr int kStageBytesPerWarp = 32 * kStageStride * 4;
-template <bool kFinal>
+// Two floats to two 16-bit values of the cache's element type (x in the low half), round to nearest even.
+template <bool kF16>
+__device__ __forceinline__ uint32_t pack2_16bit(float x, float y) {
+    if (kF16) { __half2 h = __floats2half2_rn(x, y); return *reinterpret_cast<uint32_t*>(&h); }
+    __nv_bfloat162 b = __floats2bfloat162_rn(x, y);
+    return *reinterpret_cast<uint32_t*>(&b);
+}
+
+template <bool kFinal, bool kF16>
 __device__ __forceinline__ void store_rows32(const AttnParams& p, float* stage, long long out_row, bool row_ok,
                                              long long part_row0, int col, const float (&v)[32]) {
     const int lane = threadIdx.x & 31;
@@ -500,11 +510,9 @@ __device__ __forceinline__ void store_rows32(const AttnParams& p, float* stage, 
             const bool ok = __shfl_sync(0xffffffffu, row_ok ? 1 : 0, row) != 0;
             const float4 a = *reinterpret_cast<const float4*>(stage + row * kStageStride + piece * 8);
             const float4 b2 = *reinterpret_cast<const float4*>(stage + row * kStageStride + piece * 8 + 4);
-            __nv_bfloat162 w0 = __floats2bfloat162_rn(a.x, a.y), w1 = __floats2bfloat162_rn(a.z, a.w);
-            __nv_bfloat162 w2 = __floats2bfloat162_rn(b2.x, b2.y), w3 = __floats2bfloat162_rn(b2.z, b2.w);
             uint4 u;
-            u.x = *reinterpret_cast<uint32_t*>(&w0); u.y = *reinterpret_cast<uint32_t*>(&w1);
-            u.z = *reinterpret_cast<uint32_t*>(&w2); u.w = *reinterpret_cast<uint32_t*>(&w3);
+            u.x = pack2_16bit<kF16>(a.x, a.y); u.y = pack2_16bit<kF16>(a.z, a.w);
+            u.z = pack2_16bit<kF16>(b2.x, b2.y); u.w = pack2_16bit<kF16>(b2.z, b2.w);
             if (ok) *reinterpret_cast<uint4*>(p.out + orow * kHeadDim + col + piece * 8) = u;
         }
     } else {
@@ -518,7 +526,7 @@ __device__ __forceinline__ void store_rows32(const AttnParams& p, float* stage, 
     }
 }
 
-template <bool kWide>
+template <bool kWide, bool kF16>
 __device__ __forceinline__ void softmax_loop(const AttnParams& p, Aux* aux, unsigned char* smem, uint32_t tmem, Walker w,
                                              const int s /*stream*/) {
     const int wtid = threadIdx.x - 128 - s * 128;          // 0..127 inside the warpgroup
@@ -692,11 +700,16 @@ __device__ __forceinline__ void softmax_loop(const AttnParams& p, Aux* aux, unsi
                     const uint64_t xx = fma_f32x2(pack_f32x2(sv[hf * 64 + 2 * j], sv[hf * 64 + 2 * j + 1]), scale2_x2, neg_m_x2);
                     unpack_f32x2(xx, x0, x1);
                     const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
-                    __nv_bfloat162 b2 = __floats2bfloat162_rn(p0, p1);
-                    const uint32_t u = *reinterpret_cast<uint32_t*>(&b2);
+                    const uint32_t u = pack2_16bit<kF16>(p0, p1);
                     pk[j] = u;
                     const uint64_t pe = pack_f32x2(p0, p1);
-                    const uint64_t pr = pack_f32x2(__uint_as_float(u << 16), __uint_as_float(u & 0xffff0000u));
+                    uint64_t pr;      // the two weights as the tensor core will read them
+                    if (kF16) {
+                        const float2 r = __half22float2(*reinterpret_cast<const __half2*>(&u));
+                        pr = pack_f32x2(r.x, r.y);
+                    } else {
+                        pr = pack_f32x2(__uint_as_float(u << 16), __uint_as_float(u & 0xffff0000u));
+                    }
                     if (j & 1) { ex_b = add_f32x2(ex_b, pe); rs_b = add_f32x2(rs_b, pr); }
                     else { ex_a = add_f32x2(ex_a, pe); rs_a = add_f32x2(rs_a, pr); }
                 }
@@ -780,8 +793,8 @@ __device__ __forceinline__ void softmax_loop(const AttnParams& p, Aux* aux, unsi
                 v[j] = __uint_as_float(oa[j]) * wa;           // rows that saw no key have O = 0 and weight 0
                 if (use_b) v[j] = fmaf(__uint_as_float(ob[j]), wb, v[j]);
             }
-            if (whole) store_rows32<true>(p, stage, out_row, row_ok, part_row0, c4 * 32, v);
-            else store_rows32<false>(p, stage, out_row, row_ok, part_row0, c4 * 32, v);
+            if (whole) store_rows32<true, kF16>(p, stage, out_row, row_ok, part_row0, c4 * 32, v);
+            else store_rows32<false, kF16>(p, stage, out_row, row_ok, part_row0, c4 * 32, v);
         }
         if (row_ok && write_lse) {
             if (whole) { if (p.lse) p.lse[out_row] = lse; }
@@ -800,7 +813,8 @@ __device__ __forceinline__ void softmax_loop(const AttnParams& p, Aux* aux, unsi
 // kFused: the verify step's logits scan rides along.  Warps 2 and 3 have no part in the attention; they take the
 // (row, vocabulary chunk) items of the arg-max scan in turn, 2 x gridDim.x warps in all, and leave one key per item
 // for the acceptance walk, which the merge kernel runs after this grid (`ap` is not looked at otherwise).
-template <bool kManySeqs, bool kWide, bool kFused>
+// kF16: q, the caches and out are fp16 instead of bf16 (the weights P are then rounded to fp16 as well).
+template <bool kManySeqs, bool kWide, bool kFused, bool kF16>
 __global__ void __launch_bounds__(kThreads, 1)
 verify_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap vmap,
                         const AcceptParams ap) {
@@ -849,7 +863,7 @@ verify_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap 
     if (warp < 4) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
         if (warp == 0) producer_loop<kWide>(p, &kmap, &vmap, aux, smem_base + kRingOff, w, items);
-        else if (warp == 1) mma_loop<kWide>(p, aux, smem_base, tmem, w);
+        else if (warp == 1) mma_loop<kWide, kF16>(p, aux, smem_base, tmem, w);
         else if (kFused) {
             const long long items = (long long)ap.total_nodes * ap.chunks;
             for (long long it = 2ll * blockIdx.x + (warp - 2); it < items; it += 2ll * gridDim.x)
@@ -857,7 +871,7 @@ verify_attn_umma_kernel(const AttnParams p, const __grid_constant__ CUtensorMap 
         }
     } else {
         asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
-        softmax_loop<kWide>(p, aux, smem, tmem, w, warp >= 8 ? 1 : 0);
+        softmax_loop<kWide, kF16>(p, aux, smem, tmem, w, warp >= 8 ? 1 : 0);
     }
 
     tc_fence_before();

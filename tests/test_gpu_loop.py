@@ -10,7 +10,7 @@ import pytest
 import torch
 
 import oracle
-from paper_2510_07535_b200 import OwlContext, make_dims, workloads as W
+from paper_2510_07535_b200 import OwlContext, make_dims, owl_howl_route, workloads as W
 
 pytestmark = pytest.mark.gpu
 
@@ -213,8 +213,8 @@ def test_kv_commit_hand_worked_and_errors(golden_dir):
 
 def test_decoding_loop_200_steps_on_the_device():
     """Algorithm 1 on the toy model.  The cache, the lengths, the prepared trees and the acceptance results live on
-    the device for all 200 verification steps (Prepare -> verify attention -> acceptance with [SPEC] pick ->
-    commit); the host only plays the drafter, which gets the next token as a drafter outside the GPU would.  The
+    the device for all 200 verification steps (routing -> Prepare on the routed batch -> verify attention ->
+    acceptance with [SPEC] pick -> commit); the host only plays the drafter, which gets the next token as a drafter outside the GPU would.  The
     same drafts go through the oracle's loop on the CPU.  Every step's acceptance and lengths must agree, the
     committed text must be the toy model's own (lossless), and at the end the two caches must be the same bits.
     Every 20th step the attention outputs of the step are compared as well."""
@@ -229,23 +229,29 @@ def test_decoding_loop_200_steps_on_the_device():
     noise_d = torch.from_numpy(toy_gpu.noise).to(DEV)
     roots = [int(toy_cpu.text(b, int(lens[b]) + 1)[-1]) for b in range(B)]
     emitted = [[] for _ in range(B)]
+    lastlinear_gpu, lastlinear_cpu = np.zeros(B, np.uint8), np.zeros(B, np.uint8)
     qrng = np.random.default_rng(5)
     for step in range(200):
         kinds, offs, par, tok = toy_gpu.draft(roots)
         kinds2, offs2, par2, tok2 = toy_cpu.draft(roots)
         assert kinds == kinds2 and np.array_equal(tok, tok2)
         N = int(offs[-1])
-        # ---- device: Prepare, then chains keep their drafted half (the hybrid of Section 3.2.3)
+        # ---- the router (Algorithm 1): the toy non-tree drafter "expects" 30 tokens of its chains, 4 otherwise
+        score = np.array([30.0 if kd == "chain" else 4.0 for kd in kinds], np.float32)
+        route = owl_howl_route(score, 9.0, lastlinear_gpu)
+        np.testing.assert_array_equal(route, oracle.howl_route(score, 9.0, lastlinear_cpu))
+        assert [r == 0 for r in route] == [kd == "chain" for kd in kinds]
+        # ---- device: Prepare on the routed batch (chains as drafted, trees with their [SPEC] leaves)
         pd = make_dims(batch=B, total_nodes=N, max_nodes=int(np.diff(offs).max()))
         o2 = torch.zeros(B + 1, dtype=torch.int32, device=DEV)
         p2, d2, i2, s2 = (torch.zeros(2 * N, dtype=torch.int32, device=DEV) for _ in range(4))
-        ctx.owl_prepare_spec_tree(pd, dev_i32(offs), dev_i32(par), dev_i32(tok), ld, toy_gpu.spec_token, o2, p2, d2, i2, s2)
-        keep = np.concatenate([2 * offs[b] + np.arange((1 if kinds[b] == "chain" else 2) * (offs[b + 1] - offs[b])) for b in range(B)])
-        keep_d = torch.from_numpy(keep).to(DEV)
-        v_par, v_tok, v_ids, v_pos = p2[keep_d].contiguous(), d2[keep_d].contiguous(), i2[keep_d].contiguous(), s2[keep_d].contiguous()
+        ctx.owl_prepare_hybrid(pd, dev_i32(offs), dev_i32(par), dev_i32(tok), ld, dev_i32(route), toy_gpu.spec_token, o2, p2, d2, i2, s2)
         counts = np.array([(1 if kinds[b] == "chain" else 2) * (offs[b + 1] - offs[b]) for b in range(B)])
         v_offs = np.concatenate([[0], np.cumsum(counts)]).astype(np.int32)
-        v_offs_d = dev_i32(v_offs)
+        np.testing.assert_array_equal(o2.cpu().numpy(), v_offs)
+        v_offs_d = o2
+        Mv = int(v_offs[-1])
+        v_par, v_tok, v_ids, v_pos = p2[:Mv].contiguous(), d2[:Mv].contiguous(), i2[:Mv].contiguous(), s2[:Mv].contiguous()
         M = int(v_offs[-1])
         seq_of = torch.from_numpy(np.repeat(np.arange(B), counts)).to(DEV)
         local = torch.from_numpy(np.concatenate([np.arange(c) for c in counts])).to(DEV)
@@ -273,8 +279,7 @@ def test_decoding_loop_200_steps_on_the_device():
         assert ctx.owl_get_status() == 0
 
         # ---- the oracle's step on the CPU with the same drafts
-        ro2, rp2, rd2, ri2, rs2 = oracle.prepare_spec_tree(offs, par, tok, lens, toy_cpu.spec_token)
-        r_par, r_tok, r_ids, r_pos = rp2[keep], rd2[keep], ri2[keep], rs2[keep]
+        ro2, r_par, r_tok, r_ids, r_pos = oracle.prepare_hybrid(offs, par, tok, lens, route, toy_cpu.spec_token)
         np.testing.assert_array_equal(v_par.cpu().numpy(), r_par)
         np.testing.assert_array_equal(v_pos.cpu().numpy(), r_pos)
         for b in range(B):
