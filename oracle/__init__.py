@@ -243,3 +243,58 @@ def prepare_hybrid(node_offsets, tree_parent, draft_tokens, ctx_lens, route, spe
         raise ValueError(f"owl_oracle_prepare_hybrid failed with code {rc}")
     M = int(offs[-1])
     return offs, par[:M], drf[:M], ids[:M], pos[:M]
+
+
+# ----------------------------------------------------------------------------- the steps either side of the path
+
+def lm_head_logits(hidden_bits, weight_bits) -> np.ndarray:
+    """Logits of the verifier's LM head in fp64: hidden (bf16 bits [N, K]) times weight^T (bf16 bits [V, K]).
+    A library matrix product of the exactly decoded operands; nothing else."""
+    h = decode16(hidden_bits, "bf16").reshape(np.shape(hidden_bits))
+    w = decode16(weight_bits, "bf16").reshape(np.shape(weight_bits))
+    return h @ w.T
+
+
+def lstm_alpha(n_depth: int, d: int) -> float:
+    """The embedding weight of Eq. 3-4: alpha_0 = 2^(-1/(2n)), alpha = 2 alpha_0 / ((1 - alpha_0^2) d)."""
+    a0 = 2.0 ** (-1.0 / (2.0 * n_depth))
+    return 2.0 * a0 / ((1.0 - a0 * a0) * d)
+
+
+def _layer_norm_gelu(x: np.ndarray, gamma, beta, eps: float) -> np.ndarray:
+    """f of Eq. 6 and 8: layer normalisation over the last axis (biased variance, eps inside the root), then GeLU
+    (the exact form, x Phi(x))."""
+    from math import erf
+    mu = x.mean(axis=-1, keepdims=True)
+    var = ((x - mu) ** 2).mean(axis=-1, keepdims=True)
+    y = (x - mu) / np.sqrt(var + eps)
+    if gamma is not None:
+        y = y * gamma
+    if beta is not None:
+        y = y + beta
+    phi = 0.5 * (1.0 + np.vectorize(erf)(y / np.sqrt(2.0)))
+    return y * phi
+
+
+def lstm_cell(h_bits, emb_bits, w_bits, z, alpha: float, ln_c=(None, None), ln_z=(None, None), eps: float = 1e-5):
+    """One step of the drafter cell, Eq. 1-8, in fp64.
+
+    h_bits bf16 bits [M, d_in]: hidden states; emb_bits bf16 bits [M, d]: E(t), the embeddings of the tokens (Eq. 1);
+    w_bits bf16 bits [4, d, d_in]: W^f, W^i, W^o, W^c stored output-major; z float [M, d]: the cell state (zeros at
+    the first step).  Returns (h_next [M, d], z_next [M, d]):
+        s^m = W^m h + alpha e                      (Eq. 2)
+        g^m = sigmoid(s^m), m in {f, i, o}         (Eq. 5)
+        s^c = f(s^c) g^i                           (Eq. 6)
+        z   = z g^f + s^c                          (Eq. 7)
+        h'  = f(z) g^o                             (Eq. 8)
+    with f = layer normalisation followed by GeLU."""
+    h = decode16(h_bits, "bf16").reshape(np.shape(h_bits))
+    e = decode16(emb_bits, "bf16").reshape(np.shape(emb_bits))
+    w = decode16(w_bits, "bf16").reshape(np.shape(w_bits))
+    s = [h @ w[m].T + alpha * e for m in range(4)]
+    sig = lambda x: 1.0 / (1.0 + np.exp(-x))
+    gf, gi, go = sig(s[0]), sig(s[1]), sig(s[2])
+    sc = _layer_norm_gelu(s[3], ln_c[0], ln_c[1], eps) * gi
+    z_next = np.asarray(z, dtype=np.float64) * gf + sc
+    h_next = _layer_norm_gelu(z_next, ln_z[0], ln_z[1], eps) * go
+    return h_next, z_next
