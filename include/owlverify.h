@@ -237,6 +237,44 @@ int owl_kv_commit(owl_ctx* ctx, const owl_dims* dims, void* k_cache, void* v_cac
                   const int32_t* accept_len, const int32_t* accept_path, void* stream);
 
 /*
+ * Acceptance straight from the verifier's last hidden states (Introduction: the target model's forward over the
+ * drafted tokens ends in logits, from which the accepted tokens follow): logits[n, :] = hidden[n, :] . weight^T is
+ * computed on the tensor cores (bf16 operands, fp32 accumulation) and reduced to its row arg-max inside the same
+ * kernel - the [N, V] logits are never written - then the acceptance walk of owl_tree_accept runs on those arg-max
+ * tokens.  hidden bf16 [N, hidden_dim] (row n = packed node n), weight bf16 [V, hidden_dim] (the LM head,
+ * output-major); hidden_dim a multiple of 64; N = dims->total_nodes <= 384; V = dims->vocab.  The other arguments
+ * and all outputs as owl_tree_accept.  Two logits of a row that differ by less than what fp32 accumulation order
+ * can move them (about 1e-5 for unit-scale operands) may be ranked either way; exact ties go to the lower index.
+ * Asynchronous on `stream`; device pointers, caller-owned.
+ */
+int owl_lm_head_accept(owl_ctx* ctx, const owl_dims* dims, int32_t hidden_dim, const void* hidden,
+                       const void* weight, const int32_t* draft_tokens, const int32_t* node_offsets,
+                       const int32_t* tree_parent, int32_t* accept_len, int32_t* accept_path,
+                       int32_t* bonus_token, int32_t* node_argmax, void* stream);
+
+/*
+ * One step of the drafter's LSTM cell (Section 3.2.1, Eq. 1-8), for `rows` drafter states at once:
+ *   e = E(t)  (Eq. 1, looked up by the caller);   s^m = W^m h + alpha e, m in {f, i, o, c}  (Eq. 2)
+ *   g^m = sigmoid(s^m), m in {f, i, o}  (Eq. 5);  s^c = f(s^c) g^i  (Eq. 6);  z = z g^f + s^c  (Eq. 7);
+ *   h' = f(z) g^o  (Eq. 8),   f = layer normalisation over the d outputs followed by GeLU.
+ * h bf16 [rows, d_in]; emb bf16 [rows, d]; w bf16 [4 d, d_in] = [W^f; W^i; W^o; W^c], each output-major;
+ * alpha from owl_lstm_alpha (Eq. 3-4) or the caller; ln_*_gamma / ln_*_beta fp32 [d], the affine parameters of f
+ * in Eq. 6 (c) and Eq. 8 (z), NULL for none; eps inside the root of the normalisation (1e-5 customarily);
+ * z fp32 [rows, d], read and overwritten (zeros before the first step); h_out_f32 fp32 [rows, d] and
+ * h_out_bf16 bf16 [rows, d] receive h' (either may be NULL, not both); workspace fp32 [rows, 4 d], scratch owned
+ * by the caller (the call allocates nothing).  The four projections run as one tensor-core product with fp32
+ * accumulation, the rest in fp32.  rows <= 384, d_in a multiple of 64, d a multiple of 4 up to 16384.
+ * Asynchronous on `stream`; device pointers.
+ */
+int owl_lstm_cell(owl_ctx* ctx, int32_t rows, int32_t d_in, int32_t d, const void* h, const void* emb,
+                  const void* w, float alpha, const float* ln_c_gamma, const float* ln_c_beta,
+                  const float* ln_z_gamma, const float* ln_z_beta, float eps, float* z, float* h_out_f32,
+                  void* h_out_bf16, float* workspace, void* stream);
+
+/* Eq. 3-4: alpha_0 = 2^(-1/(2 n)), alpha = 2 alpha_0 / ((1 - alpha_0^2) d), n = the tree depth drafted to. */
+double owl_lstm_alpha(int32_t n_depth, int32_t d);
+
+/*
  * One whole verify step on device buffers: owl_verify_attn and owl_tree_accept of the same batch
  * (Section 3.2.2 "Decode Stage" followed by the acceptance of the Introduction), arguments as in those
  * two calls, results bit for bit those of the two calls.  The two halves do not depend on each other (the

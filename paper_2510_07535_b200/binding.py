@@ -62,6 +62,13 @@ def load_library() -> ctypes.CDLL:
     lib.owl_howl_route.argtypes = [ctypes.c_int32, vp, ctypes.c_float, vp, vp]
     lib.owl_kv_commit.restype = i32
     lib.owl_kv_commit.argtypes = [vp, dp] + [vp] * 8
+    lib.owl_lm_head_accept.restype = i32
+    lib.owl_lm_head_accept.argtypes = [vp, dp, ctypes.c_int32] + [vp] * 10
+    lib.owl_lstm_cell.restype = i32
+    lib.owl_lstm_cell.argtypes = [vp, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, vp, vp, vp, ctypes.c_float, vp, vp, vp, vp,
+                                  ctypes.c_float, vp, vp, vp, vp, vp]
+    lib.owl_lstm_alpha.restype = ctypes.c_double
+    lib.owl_lstm_alpha.argtypes = [ctypes.c_int32, ctypes.c_int32]
     lib.owl_tree_accept_static.restype = i32
     lib.owl_tree_accept_static.argtypes = [dp] + [vp] * 10
     lib.owl_verify_step.restype = i32
@@ -226,6 +233,36 @@ class OwlContext:
             raise OwlError(rc, "owl_kv_commit", self.last_error())
         return rc
 
+    def owl_lm_head_accept(self, dims: OwlDims, hidden, weight, draft_tokens, node_offsets, tree_parent, accept_len, accept_path,
+                           bonus_token, node_argmax=None, check: bool = True) -> int:
+        dev = self.device
+        i32, bf = torch.int32, torch.bfloat16
+        rc = self.lib.owl_lm_head_accept(
+            self._h, ctypes.byref(dims), int((weight if hidden is None else hidden).shape[-1]), _ptr(hidden, bf, dev, "hidden"),
+            _ptr(weight, bf, dev, "weight"),
+            _ptr(draft_tokens, i32, dev, "draft_tokens"), _ptr(node_offsets, i32, dev, "node_offsets"),
+            _ptr(tree_parent, i32, dev, "tree_parent"), _ptr(accept_len, i32, dev, "accept_len"),
+            _ptr(accept_path, i32, dev, "accept_path"), _ptr(bonus_token, i32, dev, "bonus_token"),
+            _ptr(node_argmax, i32, dev, "node_argmax"), _stream(dev))
+        if check and rc != OWL_OK:
+            raise OwlError(rc, "owl_lm_head_accept", self.last_error())
+        return rc
+
+    def owl_lstm_cell(self, h, emb, w, alpha: float, z, h_out_f32, h_out_bf16, workspace, ln_c=(None, None), ln_z=(None, None),
+                      eps: float = 1e-5, check: bool = True) -> int:
+        dev = self.device
+        bf, f32 = torch.bfloat16, torch.float32
+        rows, d_in = h.shape
+        d = emb.shape[-1]
+        rc = self.lib.owl_lstm_cell(
+            self._h, rows, d_in, d, _ptr(h, bf, dev, "h"), _ptr(emb, bf, dev, "emb"), _ptr(w, bf, dev, "w"), float(alpha),
+            _ptr(ln_c[0], f32, dev, "ln_c_gamma"), _ptr(ln_c[1], f32, dev, "ln_c_beta"), _ptr(ln_z[0], f32, dev, "ln_z_gamma"),
+            _ptr(ln_z[1], f32, dev, "ln_z_beta"), float(eps), _ptr(z, f32, dev, "z"), _ptr(h_out_f32, f32, dev, "h_out_f32"),
+            _ptr(h_out_bf16, bf, dev, "h_out_bf16"), _ptr(workspace, f32, dev, "workspace"), _stream(dev))
+        if check and rc != OWL_OK:
+            raise OwlError(rc, "owl_lstm_cell", self.last_error())
+        return rc
+
     def owl_verify_step(self, dims: OwlDims, q, k_cache, v_cache, block_table, ctx_lens, node_offsets, tree_parent, out, lse,
                         logits, draft_tokens, accept_len, accept_path, bonus_token, node_argmax=None, check: bool = True) -> int:
         dev = self.device
@@ -320,6 +357,10 @@ def owl_howl_route(score, c: float, lastwaslinear):
     if rc != OWL_OK:
         raise OwlError(rc, "owl_howl_route")
     return route
+
+
+def owl_lstm_alpha(n_depth: int, d: int) -> float:
+    return float(load_library().owl_lstm_alpha(n_depth, d))
 
 
 def status_string(code: int) -> str:

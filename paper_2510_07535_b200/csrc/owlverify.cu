@@ -6,11 +6,13 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <cmath>
 #include <mutex>
 #include <new>
 
 #include "accept.cuh"
 #include "combine.cuh"
+#include "gemm_umma.cuh"
 #include "owl_common.cuh"
 #include "spec_loop.cuh"
 #include "verify_attn_umma.cuh"
@@ -34,6 +36,7 @@ struct owl_ctx {
     long long* sched_seq_begin = nullptr;
     SchedHeader* sched_header = nullptr;
     unsigned long long* part_keys = nullptr;
+    unsigned long long* lm_keys = nullptr;      // one arg-max key per row for the LM-head product's epilogue
     unsigned int* seq_counter = nullptr;
     uint32_t accept_epoch = 0;
     long long part_keys_len = 0;
@@ -170,6 +173,30 @@ __global__ void selftest_wait_kernel(int32_t* status, unsigned long long limit_n
     }
 }
 
+// C[M, N] = A[M, K] B[N, K]^T on the tensor cores with one of the two epilogues (gemm_umma.cuh).
+template <int kEpi>
+static int launch_gemm(owl_ctx* ctx, const void* a, const void* b, int M, int N, int K, unsigned long long* row_key, float* c,
+                       long long ldc, cudaStream_t stream) {
+    gemm_path::GemmParams g{};
+    g.M = M; g.N = N; g.K = K;
+    g.row_blocks = (M + gemm_path::kBM - 1) / gemm_path::kBM;
+    g.stages = gemm_path::ring_stages(g.row_blocks);
+    g.n_tiles = (N + gemm_path::kBN - 1) / gemm_path::kBN;
+    g.status = ctx->status;
+    g.row_key = row_key; g.c = c; g.ldc = ldc;
+    CUtensorMap amap, bmap;
+    const int ra = gemm_path::make_operand_map(ctx->encode, &amap, a, M, K);
+    const int rb = gemm_path::make_operand_map(ctx->encode, &bmap, b, N, K);
+    if (ra != 0 || rb != 0) {
+        snprintf(ctx->err, sizeof ctx->err, "cuTensorMapEncodeTiled failed (%d, %d): operands must be 16-byte aligned", ra, rb);
+        return OWL_ERR_CUDA;
+    }
+    const int grid = g.n_tiles < ctx->sm_count ? g.n_tiles : ctx->sm_count;
+    gemm_path::gemm_umma_kernel<kEpi><<<grid, gemm_path::kThreads, gemm_path::smem_bytes(g.row_blocks), stream>>>(g, amap, bmap);
+    ++ctx->launches;
+    return OWL_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -213,10 +240,8 @@ int owl_create(owl_ctx** out, int device, const owl_dims* max_dims) {
     ctx->sm_count = prop.multiProcessorCount;
     ctx->num_ctas = ctx->sm_count;
 
-    if (attn) {
-        ctx->encode = load_encode_tiled();
-        if (!ctx->encode) { delete ctx; return OWL_ERR_CUDA; }
-    }
+    ctx->encode = load_encode_tiled();
+    if (!ctx->encode) { delete ctx; return OWL_ERR_CUDA; }
 
     bool ok = true;
     auto alloc = [&](void** p, size_t bytes) {
@@ -236,6 +261,7 @@ int owl_create(owl_ctx** out, int device, const owl_dims* max_dims) {
     if (acc) {
         ctx->part_keys_len = (long long)max_dims->total_nodes * ((max_dims->vocab + kArgmaxChunk - 1) / kArgmaxChunk);
         alloc((void**)&ctx->part_keys, (size_t)ctx->part_keys_len * sizeof(unsigned long long));
+        alloc((void**)&ctx->lm_keys, (size_t)max_dims->total_nodes * sizeof(unsigned long long));
         alloc((void**)&ctx->seq_counter, 2 * (size_t)max_dims->batch * sizeof(unsigned int));
         if (ok) ok = cudaMemset(ctx->seq_counter, 0, 2 * (size_t)max_dims->batch * sizeof(unsigned int)) == cudaSuccess;
     }
@@ -246,6 +272,12 @@ int owl_create(owl_ctx** out, int device, const owl_dims* max_dims) {
     for (int i = 0; ok && i < 6; ++i) ok = cudaEventCreate(&ctx->ev[i]) == cudaSuccess;
     if (ok && attn) {
         ok = set_umma_smem_attr();
+    }
+    if (ok) {
+        ok = cudaFuncSetAttribute(gemm_path::gemm_umma_kernel<gemm_path::kEpiArgmax>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  gemm_path::kSmemLimit) == cudaSuccess &&
+             cudaFuncSetAttribute(gemm_path::gemm_umma_kernel<gemm_path::kEpiStore>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  gemm_path::kSmemLimit) == cudaSuccess;
     }
     if (!ok || cudaDeviceSynchronize() != cudaSuccess) {
         cudaGetLastError();
@@ -267,6 +299,7 @@ int owl_destroy(owl_ctx* ctx) {
     cudaFree(ctx->sched_seq_begin);
     cudaFree(ctx->sched_header);
     cudaFree(ctx->part_keys);
+    cudaFree(ctx->lm_keys);
     cudaFree(ctx->seq_counter);
     for (auto& s : ctx->stg) cudaFree(s.p);
     for (auto& ev : ctx->ev)
@@ -559,6 +592,69 @@ int owl_kv_commit(owl_ctx* ctx, const owl_dims* d, void* k_cache, void* v_cache,
     ctx->launches += 2;
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(ctx, e, "owl_kv_commit launch");
+    return OWL_OK;
+}
+
+int owl_lm_head_accept(owl_ctx* ctx, const owl_dims* d, int32_t hidden_dim, const void* hidden, const void* weight,
+                       const int32_t* draft_tokens, const int32_t* node_offsets, const int32_t* tree_parent,
+                       int32_t* accept_len, int32_t* accept_path, int32_t* bonus_token, int32_t* node_argmax, void* stream_) {
+    if (!ctx) return OWL_ERR_INVALID_ARG;
+    int rc = check_dims(d, false, true);
+    if (rc != OWL_OK) return rc;
+    if (!hidden || !weight || !draft_tokens || !tree_parent || !accept_len || !accept_path || !bonus_token) return OWL_ERR_INVALID_ARG;
+    if (!node_offsets && d->total_nodes % d->batch != 0) return OWL_ERR_INVALID_ARG;
+    if (hidden_dim < gemm_path::kBK) return OWL_ERR_INVALID_ARG;
+    if (hidden_dim % gemm_path::kBK != 0 || d->total_nodes > gemm_path::kMaxRowBlocks * gemm_path::kBM) return OWL_ERR_UNSUPPORTED;
+    if (!ctx->lm_keys || d->batch > ctx->max_dims.batch || d->total_nodes > ctx->max_dims.total_nodes) return OWL_ERR_TOO_LARGE;
+    DeviceGuard guard(ctx->device);
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    // the keys only ever grow (atomicMax): they start from 0, below every real key
+    cudaError_t e = cudaMemsetAsync(ctx->lm_keys, 0, (size_t)d->total_nodes * sizeof(unsigned long long), stream);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "owl_lm_head_accept");
+    rc = launch_gemm<gemm_path::kEpiArgmax>(ctx, hidden, weight, d->total_nodes, d->vocab, hidden_dim, ctx->lm_keys, nullptr, 0, stream);
+    if (rc != OWL_OK) return rc;
+    AcceptParams p{};
+    p.draft_tokens = draft_tokens; p.node_offsets = node_offsets; p.tree_parent = tree_parent;
+    p.accept_len = accept_len; p.accept_path = accept_path; p.bonus_token = bonus_token; p.node_argmax = node_argmax;
+    p.part_keys = ctx->lm_keys;
+    p.chunks = 1;
+    p.status = ctx->status;
+    p.batch = d->batch; p.total_nodes = d->total_nodes; p.nodes_uniform = d->total_nodes / d->batch;
+    p.max_nodes = d->max_nodes; p.vocab = d->vocab; p.path_stride = d->path_stride;
+    gemm_path::accept_walk_kernel<<<d->batch, kArgmaxThreads, 0, stream>>>(p);
+    ++ctx->launches;
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "owl_lm_head_accept launch");
+    return OWL_OK;
+}
+
+double owl_lstm_alpha(int32_t n_depth, int32_t d) {
+    if (n_depth < 1 || d < 1) return 0.0;
+    const double a0 = pow(2.0, -1.0 / (2.0 * n_depth));
+    return 2.0 * a0 / ((1.0 - a0 * a0) * d);
+}
+
+int owl_lstm_cell(owl_ctx* ctx, int32_t rows, int32_t d_in, int32_t d, const void* h, const void* emb, const void* w, float alpha,
+                  const float* ln_c_gamma, const float* ln_c_beta, const float* ln_z_gamma, const float* ln_z_beta, float eps,
+                  float* z, float* h_out_f32, void* h_out_bf16, float* workspace, void* stream_) {
+    if (!ctx || !h || !emb || !w || !z || !workspace || (!h_out_f32 && !h_out_bf16)) return OWL_ERR_INVALID_ARG;
+    if (rows < 1 || d < 1 || d_in < gemm_path::kBK || !(eps >= 0.f) || alpha != alpha) return OWL_ERR_INVALID_ARG;
+    if (d_in % gemm_path::kBK != 0 || rows > gemm_path::kMaxRowBlocks * gemm_path::kBM || d > kCellThreads * kCellPerThread ||
+        d % 4 != 0)
+        return OWL_ERR_UNSUPPORTED;
+    DeviceGuard guard(ctx->device);
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    int rc = launch_gemm<gemm_path::kEpiStore>(ctx, h, w, rows, 4 * d, d_in, nullptr, workspace, 4ll * d, stream);
+    if (rc != OWL_OK) return rc;
+    CellParams c{};
+    c.s = workspace; c.emb = static_cast<const __nv_bfloat16*>(emb);
+    c.gamma_c = ln_c_gamma; c.beta_c = ln_c_beta; c.gamma_z = ln_z_gamma; c.beta_z = ln_z_beta;
+    c.z = z; c.h_f32 = h_out_f32; c.h_bf16 = static_cast<__nv_bfloat16*>(h_out_bf16);
+    c.d = d; c.alpha = alpha; c.eps = eps;
+    lstm_cell_kernel<<<rows, kCellThreads, 0, stream>>>(c);
+    ++ctx->launches;
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "owl_lstm_cell launch");
     return OWL_OK;
 }
 
