@@ -341,6 +341,82 @@ def measure_workload(idx, args, ctx_factory, dev, world, rank, barrier, max_over
     return rec, extra
 
 
+def measure_next_rows(args, dev, barrier):
+    """The rows next to the hot path, each timed alone (CUDA events around back-to-back calls): acceptance straight from
+    hidden states (LM-head product with the arg-max in its epilogue), the drafter's LSTM cell at the paper's widths,
+    Prepare(d) and the KV commit on a 16-sequence batch."""
+    import torch
+    from paper_2510_07535_b200 import OwlContext, make_dims, workloads as W
+    from paper_2510_07535_b200.binding import owl_lstm_alpha
+
+    peak, peak_kind = measured_peaks()
+    bf = lambda bits: torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).to(dev).view(torch.bfloat16)
+    i32 = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(dev)
+    ss = np.random.SeedSequence(W.BASE_SEED + 100)
+    s_w, s_h, s_e, s_lw = ss.spawn(4)
+    K, V = 4096, W.VOCAB
+    out = {}
+    weight = bf(W.normal_bf16(s_w, V * K, scale=1.0 / np.sqrt(K)).reshape(V, K))
+    rng = np.random.default_rng(1)
+    for name, B, n in (("lm_head_accept_32_nodes", 1, 32), ("lm_head_accept_256_nodes", 4, 64)):
+        N = B * n
+        hidden = bf(W.normal_bf16(s_h, N * K).reshape(N, K))
+        par = i32(np.concatenate([W.random_tree_parents(rng, n, 8) for _ in range(B)]))
+        tok = i32(rng.integers(0, V, size=N))
+        d = make_dims(batch=B, total_nodes=N, max_nodes=n, vocab=V)
+        ctx = OwlContext(d, dev)
+        outs = [torch.zeros(B, dtype=torch.int32, device=dev), torch.zeros((B, 64), dtype=torch.int32, device=dev),
+                torch.zeros(B, dtype=torch.int32, device=dev), torch.zeros(N, dtype=torch.int32, device=dev)]
+        call = lambda _=0: ctx.owl_lm_head_accept(d, hidden, weight, tok, None, par, *outs)
+        for _ in range(3):
+            call()
+        us = float(np.median([_event_loop_us(call, 10, barrier) for _ in range(5)]))
+        assert ctx.owl_get_status() == 0
+        byts = 2 * V * K + 2 * N * K
+        out[name] = {"us": us, "hbm_gbs": byts / us / 1e3, "frac_of_hbm_peak": byts / us / 1e3 / peak, "tflops": 2.0 * N * K * V / us / 1e6,
+                     "bytes": byts, "note": "weight [128256, 4096] bf16 read once (1.05 GB > L2), logits never written"}
+        ctx.close()
+    del weight
+    torch.cuda.empty_cache()
+    M, d_in, dd = 10, 4096, 12288
+    ctx = OwlContext(make_dims(batch=16, total_nodes=16 * 32, max_nodes=32, num_kv_heads=8, max_pages_per_seq=8200, num_pages=16 * 8200), dev)
+    w = bf(W.normal_bf16(s_lw, 4 * dd * d_in, scale=1.0 / np.sqrt(d_in)).reshape(4 * dd, d_in))
+    h = bf(W.normal_bf16(s_h, M * d_in).reshape(M, d_in)); e = bf(W.normal_bf16(s_e, M * dd).reshape(M, dd))
+    z = torch.zeros((M, dd), dtype=torch.float32, device=dev); hf = torch.zeros_like(z)
+    hb = torch.zeros((M, dd), dtype=torch.bfloat16, device=dev); ws = torch.empty((M, 4 * dd), dtype=torch.float32, device=dev)
+    alpha = owl_lstm_alpha(8, dd)
+    call = lambda _=0: ctx.owl_lstm_cell(h, e, w, alpha, z, hf, hb, ws)
+    for _ in range(3):
+        call()
+    us = float(np.median([_event_loop_us(call, 10, barrier) for _ in range(5)]))
+    byts = 2 * 4 * dd * d_in
+    out["lstm_cell_10_states"] = {"us": us, "hbm_gbs": byts / us / 1e3, "frac_of_hbm_peak": byts / us / 1e3 / peak, "bytes": byts,
+                                  "note": "d_in 4096 -> d 12288, four projections [49152, 4096] bf16 read once (403 MB > L2)"}
+    del w
+    # Prepare(d) and the commit on 16 sequences of 30 drafted nodes (60 with [SPEC] leaves), 8 KV heads
+    B, n = 16, 30
+    par = i32(np.concatenate([W.random_tree_parents(rng, n, 8) for _ in range(B)]))
+    tok = i32(rng.integers(0, 1000, size=B * n)); lens = i32(np.full(B, 131072 - 64))
+    o = [torch.zeros(B + 1, dtype=torch.int32, device=dev)] + [torch.zeros(2 * B * n, dtype=torch.int32, device=dev) for _ in range(4)]
+    pd = make_dims(batch=B, total_nodes=B * n, max_nodes=n)
+    call = lambda _=0: ctx.owl_prepare_spec_tree(pd, None, par, tok, lens, 7, *o)
+    call()
+    out["prepare_spec_tree_16x30"] = {"us": float(np.median([_event_loop_us(call, 20, barrier) for _ in range(5)]))}
+    cd = make_dims(batch=B, total_nodes=2 * B * n, max_nodes=2 * n, num_kv_heads=8, max_pages_per_seq=8200, num_pages=B * 8200)
+    kc = torch.zeros((B * 8200, 8, 16, 128), dtype=torch.bfloat16, device=dev); vc = torch.zeros_like(kc)
+    table = i32(np.arange(B * 8200).reshape(B, 8200))
+    alen = i32(np.full(B, 5)); path = i32(np.tile(np.array([0, 3, 9, 20, 41] + [-1] * 59), (B, 1)))
+    def commit(_=0):
+        lens.fill_(131072 - 64)
+        ctx.owl_kv_commit(cd, kc, vc, table, lens, None, alen, path)
+    commit()
+    out["kv_commit_16_seqs_5_accepted"] = {"us": float(np.median([_event_loop_us(commit, 20, barrier) for _ in range(5)])),
+                                           "note": "includes the torch fill that resets the lengths between calls"}
+    assert ctx.owl_get_status() == 0
+    ctx.close()
+    return out
+
+
 def run_gpu(args, rank, world, local_rank):
     import torch
     import torch.distributed as dist
@@ -370,6 +446,9 @@ def run_gpu(args, rank, world, local_rank):
         records[rec["workload"]] = rec
         if idx == head_idx:
             head, extra = rec, ex
+    next_rows = None
+    if args.workload is None and world == 1 and not args.no_next_rows:
+        next_rows = measure_next_rows(args, dev, barrier)
     sampler.stop()
 
     if rank == 0:
@@ -388,6 +467,8 @@ def run_gpu(args, rank, world, local_rank):
         big = next((r for n, r in records.items() if n.startswith("cfg2")), None)
         if big:
             line["headline_128k"] = {k: big[k] for k in ("workload", "verify_step_us", "hbm_gbs", "frac_of_hbm_peak", "roofline", "clocks")}
+        if next_rows:
+            line["next_rows"] = next_rows
         if "cpu_baseline" in extra:
             line["cpu_baseline"] = extra["cpu_baseline"]
         print(json.dumps(line), flush=True)
@@ -407,6 +488,7 @@ def main():
     ap.add_argument("--impl", default="owl", choices=["owl", "reference"])
     ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of CPU oracle work per sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-next-rows", action="store_true", help="skip the timings of the rows next to the hot path")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "owl" else args.warmup
     rank = int(os.environ.get("RANK", "0"))

@@ -724,6 +724,9 @@ __device__ __forceinline__ void softmax_loop(const AttnParams& p, Aux* aux, unsi
             }
             tmem_wait_st();
             tc_fence_before();
+            // Hand-off of P: hardware barrier 4 + s, 160 threads (this warpgroup + the MMA warp).  Executed once per
+            // key tile of this stream - n_it times per segment, the count of the MMA warp's bar.sync on it - on every
+            // path: nothing above leaves the loop body early, and a wait that gave up only changed what was computed.
             asm volatile("bar.arrive %0, 160;" ::"r"(4 + s) : "memory");
             // In a unit of more than 128 rows the MMA warp polls no mbarrier between O += P V of this tile and
             // S = Q K^T of the next one: the first warp of the warpgroup looks at that tile's arrival barrier for it
@@ -733,6 +736,8 @@ __device__ __forceinline__ void softmax_loop(const AttnParams& p, Aux* aux, unsi
             if (g.shared && s == 0 && wtid < 32 && i + 1 < n_it) {
                 const uint32_t seq = tile_base + (uint32_t)(i + 1);
                 mbar_wait(smem_u32(&aux->full[seq % kTilesInFlight]), (seq / kTilesInFlight) & 1u, abort_flag);
+                // hardware barrier 6, 64 threads (this warp + the MMA warp): once per tile but the segment's last,
+                // T - 1 times, matching the MMA warp's bar.sync 6 before S of tiles 1 .. T - 1; unconditional
                 asm volatile("bar.arrive 6, 64;" ::: "memory");
             }
             ++it;
