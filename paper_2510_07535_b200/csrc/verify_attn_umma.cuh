@@ -443,27 +443,29 @@ __device__ __forceinline__ void mma_loop(const AttnParams& p, Aux* aux, uint32_t
 #pragma unroll 1
         for (int i = -1; i < n_it[0]; ++i) {
             if (i < 0 || i >= n_it[1] - 1) { general(i); continue; }
-            const uint32_t issue = ok ? elected : 0u;
-            // one body per mode, so that what a mode does not need (stream 0's slot releases and stream 1's tile
-            // barrier when both streams read every tile) is not even a predicated-off instruction
-            auto steady = [&](auto mode) {
-                constexpr bool kBoth = decltype(mode)::value;
+            // Steady state: both streams have both products.  (Releasing the ring slots from a softmax thread instead -
+            // a score tile's arrival covers every product issued before it - would spare this warp two commits of 60 to
+            // 100 clocks per tile, but the slots then come back late and the ring runs dry: 15 to 35 % slower.)
+            auto steady = [&]() {
+                const uint32_t issue = ok ? elected : 0u;
 #pragma unroll
                 for (int s = 0; s < 2; ++s) {
-                    constexpr bool kRelease = !kBoth;   // (for s == 1 see below)
                     asm volatile("bar.sync %0, 160;" ::"r"(4 + s) : "memory");
                     tc_fence_after();
                     issue_pv(s, issue, i > 0 ? 1u : 0u);
-                    if (kRelease || s == 1) umma_commit_if(issue, smem_u32(&aux->empty[v_slot[s]]));
+                    if (!shared || s == 1) umma_commit_if(issue, smem_u32(&aux->empty[v_slot[s]]));
                     advance(v_slot[s]);
                     wait_next_k(s, i);                                      // the next K tile has landed
                     issue_qk(s, ok ? issue : 0u);
                     umma_commit_if(issue, smem_u32(&aux->s_full[s]));
-                    if (kRelease || s == 1) umma_commit_if(issue, smem_u32(&aux->empty[k_slot[s]]));
+                    if (!shared || s == 1) umma_commit_if(issue, smem_u32(&aux->empty[k_slot[s]]));
                     advance(k_slot[s]);
                 }
             };
-            if (kWide && shared) steady(std::true_type{}); else steady(std::false_type{});
+            // (The backward branch over this long unrolled body stalls the warp for some 400 clocks - the loop head has
+            // left the instruction caches by the time it is taken.  Two tiles per trip halve the count of branches but
+            // double the text; measured, neither form wins.)
+            steady();
         }
         item_base += 2u * (uint32_t)T;
         ++seg_no;
@@ -645,82 +647,144 @@ __device__ __forceinline__ void softmax_loop(const AttnParams& p, Aux* aux, unsi
                     fence_proxy_async_smem();
                 }
             }
-            float sv[128];
-            {
-                uint32_t (&raw)[128] = reinterpret_cast<uint32_t(&)[128]>(sv);
-                tmem_ld64(tS, reinterpret_cast<uint32_t(&)[64]>(raw[0]));
-                tmem_ld64(tS + 64, reinterpret_cast<uint32_t(&)[64]>(raw[64]));
-                tmem_wait_ld();
-            }
-            // four independent chains: a single one would be 64 dependent instructions long
-            float mx4[4];
+            // Fast path (every tile but a segment's first, as long as the running maximum holds): the weights are
+            // computed against the running maximum m straight away, 32 columns at a time while the next 32 are on
+            // their way from tensor memory, with no pass for the tile's own maximum.  A softmax job is what the products
+            // of its stream wait for, and every instruction of it also competes with the MMA warp for the issue slots
+            // of their SM sub-partition.  If some row's weights add up to more than 2^8 (some score may then exceed m
+            // by more than the lazy threshold; rare after the first tiles), nothing has been stored yet and the tile
+            // is redone the long way.
+            bool done = false, force = false;
+            if (i > 0 && !__any_sync(0xffffffffu, m == -INFINITY)) {
+                const uint64_t scale2_x2 = pack_f32x2(scale2, scale2), neg_m_x2 = pack_f32x2(-m, -m);
+                uint64_t ex_a = 0ull, ex_b = 0ull, rs_a = 0ull, rs_b = 0ull;
+                uint32_t pk[64];
+                uint32_t buf_a[32], buf_b[32];
+                tmem_ld32(tS, buf_a);
 #pragma unroll
-            for (int q = 0; q < 4; ++q) mx4[q] = max3(sv[32 * q], sv[32 * q + 1], sv[32 * q + 2]);
+                for (int c4 = 0; c4 < 4; ++c4) {
+                    uint32_t (&cur)[32] = (c4 & 1) ? buf_b : buf_a;
+                    uint32_t (&nxt)[32] = (c4 & 1) ? buf_a : buf_b;
+                    tmem_wait_ld();
+                    if (c4 < 3) tmem_ld32(tS + (c4 + 1) * 32, nxt);
 #pragma unroll
-            for (int c = 3; c + 1 < 32; c += 2)
-#pragma unroll
-                for (int q = 0; q < 4; ++q) mx4[q] = max3(mx4[q], sv[32 * q + c], sv[32 * q + c + 1]);
-            const float mx = fmaxf(fmaxf(max3(mx4[0], sv[31], sv[63]), max3(mx4[1], sv[95], sv[127])), fmaxf(mx4[2], mx4[3]));
-            const float m_new = fmaxf(m, mx * scale2);
-            const bool need = (m_new - m) > kLazyRescale;      // false when both are -inf (NaN compares false)
-            if (__any_sync(0xffffffffu, need)) {
-                const float alpha = (m_new == -INFINITY) ? 1.f : fast_exp2(m - m_new);
-                if (i > 0) {
-                    // S of this tile is here, and its product was issued after O += P V of the tile before: the
-                    // commit that announced S covers that product too, so O may be touched now
-                    tc_fence_after();
-                    const uint32_t tO = tmem + lane_sel + 256 + s * 128;
-#pragma unroll 1
-                    for (int c4 = 0; c4 < 4; ++c4) {
-                        uint32_t o[32];
-                        tmem_ld32(tO + c4 * 32, o);
-                        tmem_wait_ld();
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * alpha);
-                        tmem_st32(tO + c4 * 32, o);
+                    for (int j = 0; j < 16; ++j) {
+                        float x0, x1;
+                        const uint64_t xx = fma_f32x2(pack_f32x2(__uint_as_float(cur[2 * j]), __uint_as_float(cur[2 * j + 1])),
+                                                      scale2_x2, neg_m_x2);
+                        unpack_f32x2(xx, x0, x1);
+                        const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
+                        const uint32_t u = pack2_16bit<kF16>(p0, p1);
+                        pk[c4 * 16 + j] = u;
+                        const uint64_t pe = pack_f32x2(p0, p1);
+                        uint64_t pr;      // the two weights as the tensor core will read them
+                        if (kF16) {
+                            const float2 r = __half22float2(*reinterpret_cast<const __half2*>(&u));
+                            pr = pack_f32x2(r.x, r.y);
+                        } else {
+                            pr = pack_f32x2(__uint_as_float(u << 16), __uint_as_float(u & 0xffff0000u));
+                        }
+                        if (j & 1) { ex_b = add_f32x2(ex_b, pe); rs_b = add_f32x2(rs_b, pr); }
+                        else { ex_a = add_f32x2(ex_a, pe); rs_a = add_f32x2(rs_a, pr); }
                     }
-                    tmem_wait_st();
-                    l *= alpha;
-                    lx *= alpha;
                 }
-                m = m_new;
-            }
-            const float neg_m = (m == -INFINITY) ? 0.f : -m;
-            const uint64_t scale2_x2 = pack_f32x2(scale2, scale2), neg_m_x2 = pack_f32x2(neg_m, neg_m);
-            // two packed accumulators each for the exact sum (LSE) and for the sum of the bf16-rounded weights:
-            // the normaliser takes the very numbers P V multiplies by, so that out = sum(p v) / sum(p) stays a
-            // true weighted mean (exact when one key dominates)
-            uint64_t ex_a = 0ull, ex_b = 0ull, rs_a = 0ull, rs_b = 0ull;
-#pragma unroll
-            for (int hf = 0; hf < 2; ++hf) {
-                uint32_t pk[32];
-#pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    float x0, x1;
-                    const uint64_t xx = fma_f32x2(pack_f32x2(sv[hf * 64 + 2 * j], sv[hf * 64 + 2 * j + 1]), scale2_x2, neg_m_x2);
-                    unpack_f32x2(xx, x0, x1);
-                    const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
-                    const uint32_t u = pack2_16bit<kF16>(p0, p1);
-                    pk[j] = u;
-                    const uint64_t pe = pack_f32x2(p0, p1);
-                    uint64_t pr;      // the two weights as the tensor core will read them
-                    if (kF16) {
-                        const float2 r = __half22float2(*reinterpret_cast<const __half2*>(&u));
-                        pr = pack_f32x2(r.x, r.y);
-                    } else {
-                        pr = pack_f32x2(__uint_as_float(u << 16), __uint_as_float(u & 0xffff0000u));
-                    }
-                    if (j & 1) { ex_b = add_f32x2(ex_b, pe); rs_b = add_f32x2(rs_b, pr); }
-                    else { ex_a = add_f32x2(ex_a, pe); rs_a = add_f32x2(rs_a, pr); }
-                }
-                tmem_st32(tS + hf * 32, pk);
-            }
-            {
                 float a0, a1, b0, b1;
                 unpack_f32x2(add_f32x2(rs_a, rs_b), a0, a1);
                 unpack_f32x2(add_f32x2(ex_a, ex_b), b0, b1);
-                l += a0 + a1;
-                lx += b0 + b1;
+                // no weight can exceed the tile's sum: a sum of at most 2^8 means that no score is more than the lazy
+                // threshold above m (a larger sum sends the tile the long way, which then moves m up)
+                force = (b0 + b1) > 256.f;
+                if (!__any_sync(0xffffffffu, force)) {
+                    tmem_st32(tS, reinterpret_cast<uint32_t(&)[32]>(pk[0]));
+                    tmem_st32(tS + 32, reinterpret_cast<uint32_t(&)[32]>(pk[32]));
+                    l += a0 + a1;
+                    lx += b0 + b1;
+                    done = true;
+                }
+            }
+            if (!done) {
+                // The long way: the tile's maximum first, then the weights; twice over tensor memory and rolled, because
+                // it runs on a segment's first tile and after a jump of the maximum only - its length in the kernel's
+                // text costs every launch more than its speed gains.
+                float mx = -INFINITY;
+#pragma unroll 1
+                for (int c4 = 0; c4 < 4; ++c4) {
+                    uint32_t r[32];
+                    tmem_ld32(tS + c4 * 32, r);
+                    tmem_wait_ld();
+                    float a = max3(__uint_as_float(r[0]), __uint_as_float(r[1]), __uint_as_float(r[2])), b = __uint_as_float(r[3]);
+#pragma unroll
+                    for (int j = 4; j + 3 < 32; j += 4) {
+                        a = max3(a, __uint_as_float(r[j]), __uint_as_float(r[j + 1]));
+                        b = max3(b, __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
+                    }
+                    mx = max3(mx, a, b);
+                }
+                const float m_new = fmaxf(m, mx * scale2);
+                // (false when both are -inf: NaN compares false)  A tile sent here by the fast path's sum moves m up at once.
+                const bool need = force ? m_new > m : (m_new - m) > kLazyRescale;
+                if (__any_sync(0xffffffffu, need)) {
+                    const float alpha = (m_new == -INFINITY) ? 1.f : fast_exp2(m - m_new);
+                    if (i > 0) {
+                        // S of this tile is here, and its product was issued after O += P V of the tile before: the
+                        // commit that announced S covers that product too, so O may be touched now
+                        tc_fence_after();
+                        const uint32_t tO = tmem + lane_sel + 256 + s * 128;
+#pragma unroll 1
+                        for (int c4 = 0; c4 < 4; ++c4) {
+                            uint32_t o[32];
+                            tmem_ld32(tO + c4 * 32, o);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * alpha);
+                            tmem_st32(tO + c4 * 32, o);
+                        }
+                        tmem_wait_st();
+                        l *= alpha;
+                        lx *= alpha;
+                    }
+                    m = m_new;
+                }
+                const float neg_m = (m == -INFINITY) ? 0.f : -m;
+                const uint64_t scale2_x2 = pack_f32x2(scale2, scale2), neg_m_x2 = pack_f32x2(neg_m, neg_m);
+                // two packed accumulators each for the exact sum (LSE) and for the sum of the rounded weights: the
+                // normaliser takes the very numbers P V multiplies by, so that out = sum(p v) / sum(p) stays a true
+                // weighted mean (exact when one key dominates)
+                uint64_t ex_a = 0ull, ex_b = 0ull, rs_a = 0ull, rs_b = 0ull;
+#pragma unroll 1
+                for (int hf = 0; hf < 2; ++hf) {
+                    // keys [64 hf, 64 hf + 64) lie in columns the weights written so far (columns below 32 hf) do not reach
+                    uint32_t sv[64], pk[32];
+                    tmem_ld64(tS + hf * 64, sv);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        float x0, x1;
+                        const uint64_t xx = fma_f32x2(pack_f32x2(__uint_as_float(sv[2 * j]), __uint_as_float(sv[2 * j + 1])), scale2_x2, neg_m_x2);
+                        unpack_f32x2(xx, x0, x1);
+                        const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
+                        const uint32_t u = pack2_16bit<kF16>(p0, p1);
+                        pk[j] = u;
+                        const uint64_t pe = pack_f32x2(p0, p1);
+                        uint64_t pr;      // the two weights as the tensor core will read them
+                        if (kF16) {
+                            const float2 r = __half22float2(*reinterpret_cast<const __half2*>(&u));
+                            pr = pack_f32x2(r.x, r.y);
+                        } else {
+                            pr = pack_f32x2(__uint_as_float(u << 16), __uint_as_float(u & 0xffff0000u));
+                        }
+                        if (j & 1) { ex_b = add_f32x2(ex_b, pe); rs_b = add_f32x2(rs_b, pr); }
+                        else { ex_a = add_f32x2(ex_a, pe); rs_a = add_f32x2(rs_a, pr); }
+                    }
+                    tmem_st32(tS + hf * 32, pk);
+                }
+                {
+                    float a0, a1, b0, b1;
+                    unpack_f32x2(add_f32x2(rs_a, rs_b), a0, a1);
+                    unpack_f32x2(add_f32x2(ex_a, ex_b), b0, b1);
+                    l += a0 + a1;
+                    lx += b0 + b1;
+                }
             }
             tmem_wait_st();
             tc_fence_before();
