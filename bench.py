@@ -435,6 +435,10 @@ def run_gpu(args, rank, world, local_rank):
     def max_over_ranks(x: float) -> float:
         return replicas.aggregate(0.0, float(x), dev)[1]
 
+    if args.only_next_rows:
+        if rank == 0:
+            print(json.dumps({"next_rows": measure_next_rows(args, dev, barrier)}), flush=True)
+        return
     sampler = ClockSampler(physical_gpu_index(local_rank))
     sampler.start()
     workloads = [args.workload] if args.workload is not None else [1, 0, 2, 3, 4]
@@ -489,6 +493,7 @@ def main():
     ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of CPU oracle work per sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-next-rows", action="store_true", help="skip the timings of the rows next to the hot path")
+    ap.add_argument("--only-next-rows", action="store_true", help="time the rows next to the hot path alone (for profiling them)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "owl" else args.warmup
     rank = int(os.environ.get("RANK", "0"))

@@ -4,12 +4,17 @@
 //               keeps of every row only its arg-max over the vocabulary - the logits are never written;
 //   drafter     A = h [rows, d_in], B = [W^f; W^i; W^o; W^c] ([4d, d_in]), Eq. 2; the epilogue stores fp32.
 // M is small (up to 384 rows: 1 to 3 blocks of 128), N is huge: B is read from HBM exactly once, A comes again and
-// again out of L2.  One persistent CTA per SM takes the 128-column tiles of C round-robin:
-//   warp 0     TMA producer: per 64-wide k-block one box per row block of A and one box of B into a ring of stages
-//   warp 1     issues the tcgen05.mma (one thread): per k-block 4 k-steps x row blocks, accumulating 128 x 128 tiles
-//   warps 4-7  epilogue, thread = row: reads its 128 accumulators of every row block and reduces or stores them
-// With at most two row blocks the accumulators are double-buffered (2 x 256 columns), so the epilogue of a tile runs
-// under the products of the next one.  Every wait is bounded as in the attention kernel.
+// again out of L2.  One persistent CTA per SM takes column tiles of C round-robin:
+//   warp 0     TMA producer: per 64-wide k-block one box per row block of A and one or two boxes of B into a ring
+//   warp 1     issues the tcgen05.mma (one thread): per k-block 4 k-steps x row blocks, 128 x width x 16 each
+//   warps 4-7  epilogue, thread = row: reads its accumulators of every row block and reduces or stores them
+// Tile width.  A 128 x 128 x 16 instruction reads 4 KB of A and 4 KB of B from shared memory in its 64 clocks, which
+// together with the TMA writes is more than the 128 B / clock shared memory delivers: two row blocks ran at 875
+// clocks per k-block for 512 of tensor-pipe time.  A 128 x 256 x 16 instruction reads 12 KB in 128 clocks, so up to
+// two row blocks take 256-column tiles (all 512 columns of tensor memory as one accumulator buffer for two row
+// blocks, two buffers for one) - as many full rounds of them as the grid has CTAs, the rest of the columns in
+// 128-wide tiles, so that the last round is not a quarter empty.  Three row blocks take 128-wide tiles throughout.
+// Every wait is bounded as in the attention kernel.
 #pragma once
 
 #include <cuda.h>
@@ -39,7 +44,8 @@ struct GemmParams {
     int M, N, K;
     int row_blocks;                 // ceil(M / 128)
     int stages;                     // ring depth: what fits beside the aux area
-    int n_tiles;                    // ceil(N / 128)
+    int wide_tiles;                 // tiles [0, wide_tiles) are 256 columns wide, the others 128
+    int n_tiles;                    // wide_tiles + ceil((N - 256 wide_tiles) / 128)
     int32_t* status;
     unsigned long long* row_key;    // kEpiArgmax: [M] keys (value, ~column), raised by atomicMax; cleared by the caller
     float* c;                       // kEpiStore: fp32 [M, ldc]
@@ -54,7 +60,9 @@ struct Aux {
 };
 static_assert(sizeof(Aux) <= kAuxBytes, "aux area too small");
 
-__host__ __device__ inline int stage_bytes(int row_blocks) { return (row_blocks + 1) * kTileBytes; }
+// a stage holds the row blocks of A and 256 (128 with three row blocks) rows of B for one k-block
+__host__ __device__ inline int b_boxes(int row_blocks) { return row_blocks <= 2 ? 2 : 1; }
+__host__ __device__ inline int stage_bytes(int row_blocks) { return (row_blocks + b_boxes(row_blocks)) * kTileBytes; }
 __host__ inline int ring_stages(int row_blocks) {
     const int s = (kSmemLimit - kAuxBytes) / stage_bytes(row_blocks);
     return s < kMaxStages ? s : kMaxStages;
@@ -104,7 +112,10 @@ gemm_umma_kernel(const GemmParams p, const __grid_constant__ CUtensorMap amap, c
     tc_fence_after();
     const uint32_t tmem = aux->tmem_base;
     const int kblocks = p.K / kBK;
-    const int nbuf = rb <= 2 ? 2 : 1;              // accumulator buffers of rb x 128 columns each
+    const int wmax = b_boxes(rb) * kBN;            // widest tile: 256 columns, 128 with three row blocks
+    const int nbuf = rb * wmax * 2 <= 512 ? 2 : 1; // accumulator buffers of rb x wmax columns each
+    auto tile_col0 = [&](int tile) { return tile < p.wide_tiles ? tile * 2 * kBN : p.wide_tiles * 2 * kBN + (tile - p.wide_tiles) * kBN; };
+    auto tile_width = [&](int tile) { return tile < p.wide_tiles ? 2 * kBN : kBN; };
     uint32_t issued = 0;
 
     if (warp == 0) {
@@ -118,19 +129,22 @@ gemm_umma_kernel(const GemmParams p, const __grid_constant__ CUtensorMap amap, c
                     if (!mbar_wait(smem_u32(&aux->empty[stage]), ph ^ 1u, abort_flag)) continue;
                     const uint32_t full = smem_u32(&aux->full[stage]);
                     const uint32_t dst = smem_base + stage * sbytes;
-                    mbar_arrive_expect_tx(full, (uint32_t)sbytes);
+                    const int boxes = tile_width(tile) / kBN, col0 = tile_col0(tile);
+                    mbar_arrive_expect_tx(full, (uint32_t)((rb + boxes) * kTileBytes));
                     for (int r = 0; r < rb; ++r) tma_load_2d_hint(dst + r * kTileBytes, &amap, full, kb * kBK, r * kBM, keep_policy);
-                    tma_load_2d_hint(dst + rb * kTileBytes, &bmap, full, kb * kBK, tile * kBN, stream_policy);
+                    for (int bx = 0; bx < boxes; ++bx)      // 128 rows of B each, back to back: one K-major operand of 256 rows
+                        tma_load_2d_hint(dst + (rb + bx) * kTileBytes, &bmap, full, kb * kBK, col0 + bx * kBN, stream_policy);
                     issued = it + 1;
                 }
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            constexpr uint32_t idesc = umma_idesc_16bit(kBM, kBN, 0, 0, false);
+            constexpr uint32_t idesc_128 = umma_idesc_16bit(kBM, kBN, 0, 0, false), idesc_256 = umma_idesc_16bit(kBM, 2 * kBN, 0, 0, false);
             uint32_t it = 0, tcount = 0;
             for (int tile = blockIdx.x; tile < p.n_tiles; tile += gridDim.x, ++tcount) {
                 const uint32_t buf = tcount % nbuf, acc_ph = (tcount / nbuf) & 1u;
+                const uint32_t idesc = tile_width(tile) == kBN ? idesc_128 : idesc_256;
                 bool ok = mbar_wait(smem_u32(&aux->acc_empty[buf]), acc_ph ^ 1u, abort_flag);   // the epilogue has read this buffer
                 tc_fence_after();
                 for (int kb = 0; kb < kblocks; ++kb, ++it) {
@@ -142,7 +156,7 @@ gemm_umma_kernel(const GemmParams p, const __grid_constant__ CUtensorMap amap, c
                         const uint64_t bdesc = umma_smem_desc_sw128(a0 + rb * kTileBytes, 16, 1024);
                         for (int r = 0; r < rb; ++r) {
                             const uint64_t adesc = umma_smem_desc_sw128(a0 + r * kTileBytes, 16, 1024);
-                            const uint32_t d = tmem + buf * (uint32_t)(rb * kBN) + r * kBN;
+                            const uint32_t d = tmem + buf * (uint32_t)(rb * wmax) + r * wmax;
 #pragma unroll
                             for (int ks = 0; ks < kBK / 16; ++ks)    // 32 bytes along K inside the 128-byte swizzle row
                                 umma_ss(d, adesc + (uint64_t)(ks * 2), bdesc + (uint64_t)(ks * 2), idesc, (kb | ks) ? 1u : 0u);
@@ -161,14 +175,14 @@ gemm_umma_kernel(const GemmParams p, const __grid_constant__ CUtensorMap amap, c
             const uint32_t buf = tcount % nbuf, acc_ph = (tcount / nbuf) & 1u;
             const bool ok = mbar_wait(smem_u32(&aux->acc_full[buf]), acc_ph, abort_flag);
             tc_fence_after();
-            const int n0 = tile * kBN;
+            const int n0 = tile_col0(tile), chunks = tile_width(tile) / 32;
             for (int r = 0; r < rb; ++r) {
                 const int row = r * kBM + lane_row;
-                const uint32_t taddr = tmem + lane_sel + buf * (uint32_t)(rb * kBN) + r * kBN;
+                const uint32_t taddr = tmem + lane_sel + buf * (uint32_t)(rb * wmax) + r * wmax;
                 float bv = -INFINITY;
                 uint32_t bi = 0xffffffffu;
 #pragma unroll 1
-                for (int c4 = 0; c4 < kBN / 32; ++c4) {
+                for (int c4 = 0; c4 < chunks; ++c4) {
                     uint32_t v[32];
                     tmem_ld32(taddr + c4 * 32, v);
                     tmem_wait_ld();

@@ -181,7 +181,10 @@ static int launch_gemm(owl_ctx* ctx, const void* a, const void* b, int M, int N,
     g.M = M; g.N = N; g.K = K;
     g.row_blocks = (M + gemm_path::kBM - 1) / gemm_path::kBM;
     g.stages = gemm_path::ring_stages(g.row_blocks);
-    g.n_tiles = (N + gemm_path::kBN - 1) / gemm_path::kBN;
+    // as many full rounds of 256-column tiles as there are CTAs, the remaining columns in 128-wide tiles
+    const int wide_cap = gemm_path::b_boxes(g.row_blocks) == 2 ? N / (2 * gemm_path::kBN) : 0;
+    g.wide_tiles = wide_cap >= ctx->sm_count ? (wide_cap / ctx->sm_count) * ctx->sm_count : 0;
+    g.n_tiles = g.wide_tiles + (N - g.wide_tiles * 2 * gemm_path::kBN + gemm_path::kBN - 1) / gemm_path::kBN;
     g.status = ctx->status;
     g.row_key = row_key; g.c = c; g.ldc = ldc;
     CUtensorMap amap, bmap;
