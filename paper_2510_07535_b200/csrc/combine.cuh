@@ -31,9 +31,9 @@ constexpr int kCombineWarps = 8;
 // fill the machine.  The host takes 32 up to 4096 output rows.
 template <bool kFused, int kGroup>
 __global__ void __launch_bounds__(kCombineWarps * 32) combine_sched_kernel(const AttnParams p, const AcceptParams ap) {
+    const long long rows = (long long)p.total_nodes * p.num_q_heads;
+    const unsigned row_ctas = (unsigned)p.combine_row_ctas;
     if (kFused) {
-        const long long rows = (long long)p.total_nodes * p.num_q_heads;
-        const unsigned row_ctas = (unsigned)((rows + kCombineWarps - 1) / kCombineWarps);
         if (blockIdx.x >= row_ctas) {
             static_assert(kCombineWarps * 32 >= kMaxNodes, "the walk needs one thread per node");
             asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -42,26 +42,21 @@ __global__ void __launch_bounds__(kCombineWarps * 32) combine_sched_kernel(const
             return;
         }
     }
+    // The row CTAs are persistent: a warp derives the schedule once and then takes rows first, first + stride, ...
+    // (one CTA per eight rows cost a launch of 8192 rows 19 us, most of it the schedule derived 8192 times).
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const long long row_id = (long long)blockIdx.x * kCombineWarps + warp;
-    const bool row_valid = row_id < (long long)p.total_nodes * p.num_q_heads;
-    const int n = row_valid ? (int)(row_id / p.num_q_heads) : 0, hq = row_valid ? (int)(row_id % p.num_q_heads) : 0;
+    const long long first = (long long)blockIdx.x * kCombineWarps + warp, stride = (long long)row_ctas * kCombineWarps;
     const bool small = p.batch <= 32;
-    int b = 0, node_base = 0, tiles = 0;
-    long long seq_begin = 0;
+    WarpSchedule ws{};
     Partition part;
     if (small) {
-        const WarpSchedule ws = warp_schedule(p);
-        const unsigned hit = __ballot_sync(0xffffffffu, lane < p.batch && ws.tiles > 0 && n >= ws.node_base && n < ws.node_base + ws.n);
-        b = hit ? __ffs(hit) - 1 : 0;
-        node_base = __shfl_sync(0xffffffffu, ws.node_base, b);
-        tiles = hit ? __shfl_sync(0xffffffffu, ws.tiles, b) : 0;
-        seq_begin = __shfl_sync(0xffffffffu, ws.excl_t, b);
+        ws = warp_schedule(p);
         part.init(ws.total, p.num_ctas, ws.units, ws.uniform_tiles);
     }
-    // the CTAs c0..c1 whose pieces cut the row's unit, and the slot row of the partial this lane fetches first
-    int lrow = 0, c0 = 0, c1 = 0;
-    long long t0 = 0, prow_first = 0;
+    // per row: its sequence, the CTAs c0..c1 whose pieces cut the row's unit, and the slot row of the partial this
+    // lane fetches first
+    int n = 0, hq = 0, b = 0, node_base = 0, tiles = 0, lrow = 0, c0 = 0, c1 = 0;
+    long long seq_begin = 0, t0 = 0, prow_first = 0;
     auto row_of = [&](int c) -> long long { return (2ll * c + (part.begin(c) < t0 ? 1 : 0)) * p.rows_per_slot + lrow; };
     auto plan = [&]() {
         if (tiles == 0) return;
@@ -72,82 +67,97 @@ __global__ void __launch_bounds__(kCombineWarps * 32) combine_sched_kernel(const
         c1 = part.owner(t0 + tiles - 1);
         prow_first = row_of(c0 + min(lane & (kGroup - 1), c1 - c0));
     };
-    if (small) plan();
+    auto locate = [&](long long row_id) {       // every lane of the warp, same row
+        n = (int)(row_id / p.num_q_heads);
+        hq = (int)(row_id - (long long)n * p.num_q_heads);
+        if (small) {
+            const unsigned hit = __ballot_sync(0xffffffffu, lane < p.batch && ws.tiles > 0 && n >= ws.node_base && n < ws.node_base + ws.n);
+            b = hit ? __ffs(hit) - 1 : 0;
+            node_base = __shfl_sync(0xffffffffu, ws.node_base, b);
+            tiles = hit ? __shfl_sync(0xffffffffu, ws.tiles, b) : 0;
+            seq_begin = __shfl_sync(0xffffffffu, ws.excl_t, b);
+        } else {
+            int lo = 0, hi = p.batch;  // largest b with node_offsets[b] <= n
+            if (p.node_offsets) {
+                while (hi - lo > 1) { int mid = (lo + hi) >> 1; if (p.node_offsets[mid] <= n) lo = mid; else hi = mid; }
+                b = lo;
+            } else {
+                b = n / p.nodes_uniform;
+            }
+            const long long sb = p.sched_seq_begin[b], se = p.sched_seq_begin[b + 1];
+            node_base = seq_node_base(p, b);
+            seq_begin = sb;
+            tiles = (int)((se - sb) / p.num_kv_heads);
+        }
+        plan();
+    };
+    // latency after the pass has ended is what this kernel costs: whatever needs no output of the pass comes before
+    // the wait - for batches of at most 32 sequences the whole plan of the warp's first row
+    if (small && first < rows) locate(first);
     // from here on the split-KV pass has completed and its writes are visible (a no-op in an ordinary launch)
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next kernel in the stream may queue up
-    if (!row_valid) return;
     if (!small) {
-        int lo = 0, hi = p.batch;  // largest b with node_offsets[b] <= n
-        if (p.node_offsets) {
-            while (hi - lo > 1) { int mid = (lo + hi) >> 1; if (p.node_offsets[mid] <= n) lo = mid; else hi = mid; }
-            b = lo;
-        } else {
-            b = n / p.nodes_uniform;
-        }
-        // independent loads first, tests afterwards: one round trip instead of four
-        const long long sb = p.sched_seq_begin[b], se = p.sched_seq_begin[b + 1];
-        const SchedHeader hdr = *p.sched_header;
-        node_base = seq_node_base(p, b);
-        seq_begin = sb;
-        tiles = (int)((se - sb) / p.num_kv_heads);
+        const SchedHeader hdr = *p.sched_header;      // larger batches read the schedule the pass left
         part.init(hdr.total_tiles, p.num_ctas, hdr.units, hdr.uniform_tiles);
-        plan();
     }
-    if (tiles == 0) return;
-    if (c0 == c1) return;  // a single CTA saw every key of this unit and wrote the result itself
-    const int bad_epoch = __ldcg(p.seq_bad + b);   // (its round trip overlaps the partial loads below)
-    const int count = c1 - c0 + 1;
+    for (long long row_id = first; row_id < rows; row_id += stride) {
+        if (!small || row_id != first) locate(row_id);
+        if (tiles == 0) continue;
+        if (c0 == c1) continue;  // a single CTA saw every key of this unit and wrote the result itself
+        const int bad_epoch = __ldcg(p.seq_bad + b);   // (its round trip overlaps the partial loads below)
+        const int count = c1 - c0 + 1;
 
-    // Partials are taken kGroup at a time: lane j (< kGroup) of a group owns partial base + j.  The row loads do
-    // not depend on the LSE values, so both go out together: one memory round trip per group.  Groups are folded
-    // online (running maximum).
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    float sum = 0.f, mx = -INFINITY;
-    for (int base = 0; base < count; base += kGroup) {
-        const int mine = base + (lane & (kGroup - 1));
-        const bool have = mine < count;
-        const long long prow = base == 0 ? prow_first : row_of(c0 + (have ? mine : 0));
-        const float my_lse = have ? __ldcg(p.part_lse + prow) : -INFINITY;
-        float4 v[kGroup];
-#pragma unroll
-        for (int j = 0; j < kGroup; ++j) {
-            const long long pj = __shfl_sync(0xffffffffu, prow, j);
-            v[j] = base + j < count ? __ldcg(reinterpret_cast<const float4*>(p.part_o + pj * kHeadDim + lane * 4))
-                                    : make_float4(0.f, 0.f, 0.f, 0.f);
-        }
-        float gmx = my_lse;
-#pragma unroll
-        for (int o = kGroup / 2; o > 0; o >>= 1) gmx = fmaxf(gmx, __shfl_xor_sync(0xffffffffu, gmx, o));
-        const float mx_new = fmaxf(mx, gmx);
-        if (mx_new > -INFINITY) {
-            const float rescale = mx > -INFINITY ? __expf(mx - mx_new) : 0.f;
-            acc.x *= rescale; acc.y *= rescale; acc.z *= rescale; acc.w *= rescale;
-            sum *= rescale;
-            const float w = have ? __expf(my_lse - mx_new) : 0.f;     // -inf partial: weight 0
+        // Partials are taken kGroup at a time: lane j (< kGroup) of a group owns partial base + j.  The row loads do
+        // not depend on the LSE values, so both go out together: one memory round trip per group.  Groups are folded
+        // online (running maximum).
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        float sum = 0.f, mx = -INFINITY;
+        for (int base = 0; base < count; base += kGroup) {
+            const int mine = base + (lane & (kGroup - 1));
+            const bool have = mine < count;
+            const long long prow = base == 0 ? prow_first : row_of(c0 + (have ? mine : 0));
+            const float my_lse = have ? __ldcg(p.part_lse + prow) : -INFINITY;
+            float4 v[kGroup];
 #pragma unroll
             for (int j = 0; j < kGroup; ++j) {
-                const float wj = __shfl_sync(0xffffffffu, w, j);
-                acc.x += wj * v[j].x; acc.y += wj * v[j].y; acc.z += wj * v[j].z; acc.w += wj * v[j].w;
-                sum += wj;
+                const long long pj = __shfl_sync(0xffffffffu, prow, j);
+                v[j] = base + j < count ? __ldcg(reinterpret_cast<const float4*>(p.part_o + pj * kHeadDim + lane * 4))
+                                        : make_float4(0.f, 0.f, 0.f, 0.f);
             }
-            mx = mx_new;
+            float gmx = my_lse;
+#pragma unroll
+            for (int o = kGroup / 2; o > 0; o >>= 1) gmx = fmaxf(gmx, __shfl_xor_sync(0xffffffffu, gmx, o));
+            const float mx_new = fmaxf(mx, gmx);
+            if (mx_new > -INFINITY) {
+                const float rescale = mx > -INFINITY ? __expf(mx - mx_new) : 0.f;
+                acc.x *= rescale; acc.y *= rescale; acc.z *= rescale; acc.w *= rescale;
+                sum *= rescale;
+                const float w = have ? __expf(my_lse - mx_new) : 0.f;     // -inf partial: weight 0
+#pragma unroll
+                for (int j = 0; j < kGroup; ++j) {
+                    const float wj = __shfl_sync(0xffffffffu, w, j);
+                    acc.x += wj * v[j].x; acc.y += wj * v[j].y; acc.z += wj * v[j].z; acc.w += wj * v[j].w;
+                    sum += wj;
+                }
+                mx = mx_new;
+            }
         }
+        if (bad_epoch == p.epoch) continue;            // the pass found a bad tree or page in this sequence: no output
+        const float inv = sum > 0.f ? 1.f / sum : 0.f;
+        uint2 pk;
+        if (p.f16) {
+            __half2 lo2 = __floats2half2_rn(acc.x * inv, acc.y * inv), hi2 = __floats2half2_rn(acc.z * inv, acc.w * inv);
+            pk.x = *reinterpret_cast<uint32_t*>(&lo2);
+            pk.y = *reinterpret_cast<uint32_t*>(&hi2);
+        } else {
+            __nv_bfloat162 lo2 = __floats2bfloat162_rn(acc.x * inv, acc.y * inv), hi2 = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
+            pk.x = *reinterpret_cast<uint32_t*>(&lo2);
+            pk.y = *reinterpret_cast<uint32_t*>(&hi2);
+        }
+        *reinterpret_cast<uint2*>(p.out + row_id * kHeadDim + lane * 4) = pk;
+        if (p.lse && lane == 0) p.lse[row_id] = sum > 0.f ? mx + logf(sum) : -INFINITY;
     }
-    if (bad_epoch == p.epoch) return;              // the pass found a bad tree or page in this sequence: no output
-    const float inv = sum > 0.f ? 1.f / sum : 0.f;
-    uint2 pk;
-    if (p.f16) {
-        __half2 lo2 = __floats2half2_rn(acc.x * inv, acc.y * inv), hi2 = __floats2half2_rn(acc.z * inv, acc.w * inv);
-        pk.x = *reinterpret_cast<uint32_t*>(&lo2);
-        pk.y = *reinterpret_cast<uint32_t*>(&hi2);
-    } else {
-        __nv_bfloat162 lo2 = __floats2bfloat162_rn(acc.x * inv, acc.y * inv), hi2 = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
-        pk.x = *reinterpret_cast<uint32_t*>(&lo2);
-        pk.y = *reinterpret_cast<uint32_t*>(&hi2);
-    }
-    *reinterpret_cast<uint2*>(p.out + row_id * kHeadDim + lane * 4) = pk;
-    if (p.lse && lane == 0) p.lse[row_id] = sum > 0.f ? mx + logf(sum) : -INFINITY;
 }
 
 }  // namespace owl

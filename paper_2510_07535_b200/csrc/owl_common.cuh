@@ -43,6 +43,7 @@ struct AttnParams {
     int32_t page_size, page_shift, max_pages_per_seq, num_pages;
     int32_t rows_per_slot;        // row stride of one partial slot
     int32_t num_ctas;             // CTAs of the split-KV pass (the flat tile range is cut into this many pieces)
+    int32_t combine_row_ctas;     // CTAs of the merge kernel that take output rows (persistent, eight warps each)
     int32_t f16;                  // q / caches / out are fp16 instead of bf16 (same size; typed as bf16 pointers here)
     float sm_scale;
 };

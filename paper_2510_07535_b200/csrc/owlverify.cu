@@ -388,7 +388,10 @@ static int verify_attn_impl(owl_ctx* ctx, const owl_dims* d, const void* q, cons
 
     if (ctx->profiling) cudaEventRecord(ctx->ev[0], stream);
     const long long rows = (long long)d->total_nodes * d->num_q_heads;
-    const unsigned grid = (unsigned)((rows + kCombineWarps - 1) / kCombineWarps);
+    // one warp per row up to two CTAs per SM; beyond that the merge kernel's warps stride over the rows
+    const long long want_ctas = (rows + kCombineWarps - 1) / kCombineWarps;
+    const unsigned grid = (unsigned)(want_ctas < 2ll * ctx->sm_count ? want_ctas : 2ll * ctx->sm_count);
+    p.combine_row_ctas = (int32_t)grid;
     {
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(ctx->num_ctas);
