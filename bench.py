@@ -215,7 +215,9 @@ def run_reference(args, rank, world):
         "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": est * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic", "impl": "reference",
-        "config": {"workload": spec.name, "note": "CPU oracle (plain fp64 C, OpenMP) on sampled rows of the same workload"},
+        "config": {"batch": spec.batch, "ctx_lens": [int(min(spec.ctx_lens)), int(max(spec.ctx_lens))], "nodes": int(wl.total_nodes),
+                   "q_heads": spec.num_q_heads, "kv_heads": spec.num_kv_heads, "vocab": spec.vocab, "workload": spec.name},
+        "note": "CPU oracle (plain fp64 C, OpenMP) on sampled rows of the same workload",
         "cpu_baseline": {"value": value, "unit": "GB/s", "cores": threads, "kind": "oracle", "sample": desc},
         "e2e": {"value": value, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "verify_step_us": est * 1e6, "gpu_launches": 0,
@@ -461,8 +463,9 @@ def run_gpu(args, rank, world, local_rank):
             "metric": METRIC, "value": world * step_bytes / head["verify_step_us"] / 1e3, "unit": "GB/s", "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": head["verify_step_us"] * 1e-3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": dict(head["config"], workload=head["workload"], parallelism="replicas only" if world > 1 else "single GPU",
-                           l2=head["l2"], timing=f"median of {args.regions} timed regions of {args.steps} steps each"),
+            "config": dict(head["config"], workload=head["workload"]),
+            "parallelism": "replicas only" if world > 1 else "single GPU", "l2": head["l2"],
+            "timing": f"median of {args.regions} timed regions of {args.steps} steps each",
             "verify_step_us": head["verify_step_us"], "frac_of_hbm_peak": head["frac_of_hbm_peak"],
             "kernel_us": head["kernel_us"], "bytes_per_step": head["bytes_per_step"], "roofline": head["roofline"],
             "accept_gbs": head["accept_gbs"], "e2e": extra.get("e2e"), "gpu_launches": extra.get("launches_region"),
