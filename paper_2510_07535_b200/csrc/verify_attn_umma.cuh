@@ -360,22 +360,22 @@ __device__ __forceinline__ void mma_loop(const AttnParams& p, Aux* aux, uint32_t
         auto advance = [&](uint32_t& slot) { slot += step_items; if (slot >= (uint32_t)kSlots) slot -= kSlots; };
         // O_s (+)= P_s V: A from tensor memory, B = the V tile as it lies in the ring (MN-major)
         auto issue_pv = [&](int s, uint32_t issue, uint32_t acc0) {
-            const uint64_t vdesc = v_desc0 + (uint64_t)(v_slot[s] * (uint32_t)(kSlotBytes >> 4));
+            const uint32_t v_lo = (uint32_t)v_desc0 + v_slot[s] * (uint32_t)(kSlotBytes >> 4), v_hi = (uint32_t)(v_desc0 >> 32);
             const uint32_t tO = tmem + 256 + s * 128, tP = tmem + s * 128;
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks)
-                umma_ts_if(issue, tO, tP + ks * 8, vdesc + (uint64_t)(ks * 4096 >> 4), idesc_pv, ks ? 1u : acc0);
+                umma_ts_lh_if(issue, tO, tP + ks * 8, v_lo + (uint32_t)(ks * 4096 >> 4), v_hi, idesc_pv, ks ? 1u : acc0);
         };
         // S_s = Q K^T: both operands K-major in shared memory
         auto issue_qk = [&](int s, uint32_t issue) {
-            const uint64_t qdesc = q_desc0 + (uint64_t)((shared && s) ? (kQBytes >> 4) : 0);
-            const uint64_t kdesc = k_desc0 + (uint64_t)(k_slot[s] * (uint32_t)(kSlotBytes >> 4));
+            const uint32_t q_lo = (uint32_t)q_desc0 + (uint32_t)((shared && s) ? (kQBytes >> 4) : 0), q_hi = (uint32_t)(q_desc0 >> 32);
+            const uint32_t k_lo = (uint32_t)k_desc0 + k_slot[s] * (uint32_t)(kSlotBytes >> 4), k_hi = (uint32_t)(k_desc0 >> 32);
 #pragma unroll
             for (int hf = 0; hf < 2; ++hf)
 #pragma unroll
                 for (int ks = 0; ks < 4; ++ks)
-                    umma_ss_if(issue, tmem + s * 128, qdesc + (uint64_t)((hf * 16384 + ks * 32) >> 4),
-                               kdesc + (uint64_t)((hf * 1024 + ks * 32) >> 4), idesc_qk, (hf | ks) ? 1u : 0u);
+                    umma_ss_lh_if(issue, tmem + s * 128, q_lo + (uint32_t)((hf * 16384 + ks * 32) >> 4), q_hi,
+                                  k_lo + (uint32_t)((hf * 1024 + ks * 32) >> 4), k_hi, idesc_qk, (hf | ks) ? 1u : 0u);
         };
         // Before S = Q K^T of the stream's tile i + 1.  M > 128: the issue loop is what bounds the unit, and the
         // softmax warpgroup, which has time to spare, looks at the tile's arrival barrier and passes the news on
