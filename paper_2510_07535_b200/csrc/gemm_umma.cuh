@@ -11,13 +11,24 @@
 // Tile width.  A 128 x 128 x 16 instruction reads 4 KB of A and 4 KB of B from shared memory in its 64 clocks, which
 // together with the TMA writes is more than the 128 B / clock shared memory delivers: two row blocks ran at 875
 // clocks per k-block for 512 of tensor-pipe time.  A 128 x 256 x 16 instruction reads 12 KB in 128 clocks, so up to
-// two row blocks take 256-column tiles (all 512 columns of tensor memory as one accumulator buffer for two row
-// blocks, two buffers for one) - as many full rounds of them as the grid has CTAs, the rest of the columns in
-// 128-wide tiles, so that the last round is not a quarter empty.  Three row blocks take 128-wide tiles throughout.
+// two row blocks take tiles of up to 256 columns (all 512 columns of tensor memory as one accumulator buffer for two
+// row blocks, two buffers for one); three row blocks take up to 128.
+// Balance.  B is read once and every CTA streams at the same rate, so the columns are dealt out evenly: each CTA
+// gets ceil(N / 16 / CTAs) units of 16 columns, cut into as few tiles as the width limit allows, the tiles of one
+// round equally wide on every CTA (widths differ by at most 16 between rounds).  The instruction's N is the tile
+// width (any multiple of 16), one TMA box brings the tile's rows of B.  N = 49152 on 148 CTAs: rounds of 176 and
+// 160 columns, 98.8 % of the last round filled, against 65 % with 256-wide tiles only.
+// Ring.  At 6.5 TB/s over 148 SMs and 2.5-3 us of loaded memory latency a CTA needs 110-130 KB of B in flight, so a
+// stage holds what is loaded and nothing else: the tile's rows of B and the valid rows of A rounded up to 8 (one
+// swizzle atom).  The instruction still reads 128 rows of A: past the loaded ones it finds whatever follows in
+// shared memory (the stage's B, the next stage, the pad behind the ring), which only feeds accumulator rows >= M that
+// nobody reads - an output row depends on its own row of A alone.  10 rows against 176 of B: 24 KB per stage, 8
+// stages, 176 KB in flight (with 48 KB stages there were 88 KB in flight and the product ran at 4.2 TB/s).
 // Every wait is bounded as in the attention kernel.
 #pragma once
 
 #include <cuda.h>
+#include <cooperative_groups.h>
 #include <cuda_bf16.h>
 
 #include "accept.cuh"
@@ -34,7 +45,7 @@ constexpr int kBM = 128, kBN = 128, kBK = 64;
 constexpr int kThreads = 256;
 constexpr int kTileBytes = kBM * kBK * 2;        // 16 KB: 128 rows of one 128-byte swizzle row each
 constexpr int kMaxRowBlocks = 3;
-constexpr int kMaxStages = 8;
+constexpr int kMaxStages = 12;
 constexpr int kAuxBytes = 1024;
 constexpr int kSmemLimit = 232448;               // 227 KB
 
@@ -43,9 +54,12 @@ enum Epilogue { kEpiArgmax = 0, kEpiStore = 1 };
 struct GemmParams {
     int M, N, K;
     int row_blocks;                 // ceil(M / 128)
-    int stages;                     // ring depth: what fits beside the aux area
-    int wide_tiles;                 // tiles [0, wide_tiles) are 256 columns wide, the others 128
-    int n_tiles;                    // wide_tiles + ceil((N - 256 wide_tiles) / 128)
+    int stages;                     // ring depth: what fits beside the aux area and the pad
+    int a_bytes;                    // per stage: full row blocks of 16 KB, then the last block's rows rounded up to 8
+    int stage_bytes;                // a_bytes + the widest tile's rows of B, 128 bytes each
+    int rounds;                     // tiles per CTA; round t holds one tile per CTA, all of the same width
+    int wide_rounds;                // rounds [0, wide_rounds) are w_lo + 16 columns wide, the others w_lo
+    int w_lo;                       // multiple of 16, <= 256 (128 with three row blocks)
     int32_t* status;
     unsigned long long* row_key;    // kEpiArgmax: [M] keys (value, ~column), raised by atomicMax; cleared by the caller
     float* c;                       // kEpiStore: fp32 [M, ldc]
@@ -60,14 +74,14 @@ struct Aux {
 };
 static_assert(sizeof(Aux) <= kAuxBytes, "aux area too small");
 
-// a stage holds the row blocks of A and 256 (128 with three row blocks) rows of B for one k-block
+// up to two row blocks take tiles of 256 columns, three of 128 (tensor memory: row blocks x width <= 512 columns)
 __host__ __device__ inline int b_boxes(int row_blocks) { return row_blocks <= 2 ? 2 : 1; }
-__host__ __device__ inline int stage_bytes(int row_blocks) { return (row_blocks + b_boxes(row_blocks)) * kTileBytes; }
-__host__ inline int ring_stages(int row_blocks) {
-    const int s = (kSmemLimit - kAuxBytes) / stage_bytes(row_blocks);
+// shared memory: [aux][stages x stage_bytes][pad: the A operand window of the last stage may reach one tile past it]
+__host__ inline int ring_stages(int stage_bytes) {
+    const int s = (kSmemLimit - kAuxBytes - kTileBytes) / stage_bytes;
     return s < kMaxStages ? s : kMaxStages;
 }
-__host__ inline int smem_bytes(int row_blocks) { return ring_stages(row_blocks) * stage_bytes(row_blocks) + kAuxBytes; }
+__host__ inline int smem_bytes(int stages, int stage_bytes) { return kAuxBytes + stages * stage_bytes + kTileBytes; }
 
 // 2-D tile load global -> shared with an L2 cache policy, completion counted in bytes on an mbarrier of this CTA.
 __device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const void* tmap, uint32_t bar, int c0, int c1, uint64_t policy) {
@@ -83,13 +97,14 @@ __device__ __forceinline__ uint64_t l2_policy_evict_last() {
 
 template <int kEpi>
 __global__ void __launch_bounds__(kThreads, 1)
-gemm_umma_kernel(const GemmParams p, const __grid_constant__ CUtensorMap amap, const __grid_constant__ CUtensorMap bmap) {
+gemm_umma_kernel(const GemmParams p, const __grid_constant__ CUtensorMap amap, const __grid_constant__ CUtensorMap amap_last,
+                 const __grid_constant__ CUtensorMap bmap_hi, const __grid_constant__ CUtensorMap bmap_lo) {
     extern __shared__ __align__(1024) unsigned char smem[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const uint32_t smem_base = smem_u32(smem);
+    const uint32_t smem_base = smem_u32(smem) + kAuxBytes;       // the ring
     const int rb = p.row_blocks, stages = p.stages;
-    const int sbytes = stage_bytes(rb);
-    Aux* aux = reinterpret_cast<Aux*>(smem + stages * sbytes);
+    const int sbytes = p.stage_bytes;
+    Aux* aux = reinterpret_cast<Aux*>(smem);
     volatile int* abort_flag = &aux->abort_flag;
     // may be launched as a programmatic dependent of the kernel before it in the stream
     asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -104,7 +119,9 @@ gemm_umma_kernel(const GemmParams p, const __grid_constant__ CUtensorMap amap, c
         aux->abort_flag = 0;
         fence_barrier_init();
         tma_prefetch_desc(&amap);
-        tma_prefetch_desc(&bmap);
+        tma_prefetch_desc(&amap_last);
+        tma_prefetch_desc(&bmap_hi);
+        tma_prefetch_desc(&bmap_lo);
     }
     if (warp == 0) { tmem_alloc(smem_u32(&aux->tmem_base), 512); tmem_relinquish(); }
     tc_fence_before();
@@ -114,8 +131,12 @@ gemm_umma_kernel(const GemmParams p, const __grid_constant__ CUtensorMap amap, c
     const int kblocks = p.K / kBK;
     const int wmax = b_boxes(rb) * kBN;            // widest tile: 256 columns, 128 with three row blocks
     const int nbuf = rb * wmax * 2 <= 512 ? 2 : 1; // accumulator buffers of rb x wmax columns each
-    auto tile_col0 = [&](int tile) { return tile < p.wide_tiles ? tile * 2 * kBN : p.wide_tiles * 2 * kBN + (tile - p.wide_tiles) * kBN; };
-    auto tile_width = [&](int tile) { return tile < p.wide_tiles ? 2 * kBN : kBN; };
+    // round t: one tile per CTA, the rounds' column bands one after the other; a tile that starts past N is empty
+    auto tile_width = [&](int t) { return t < p.wide_rounds ? p.w_lo + 16 : p.w_lo; };
+    auto tile_col0 = [&](int t) {
+        const int hi = t < p.wide_rounds ? t : p.wide_rounds;
+        return (int)gridDim.x * (hi * (p.w_lo + 16) + (t - hi) * p.w_lo) + (int)blockIdx.x * tile_width(t);
+    };
     uint32_t issued = 0;
 
     if (warp == 0) {
@@ -123,28 +144,30 @@ gemm_umma_kernel(const GemmParams p, const __grid_constant__ CUtensorMap amap, c
             const uint64_t stream_policy = l2_policy_evict_first();   // B is read once
             const uint64_t keep_policy = l2_policy_evict_last();      // A is read by every CTA for every tile
             uint32_t it = 0;
-            for (int tile = blockIdx.x; tile < p.n_tiles; tile += gridDim.x) {
+            for (int t = 0; t < p.rounds; ++t) {
+                const int col0 = tile_col0(t), w = tile_width(t);
+                if (col0 >= p.N) break;
+                const CUtensorMap* bmap = t < p.wide_rounds ? &bmap_hi : &bmap_lo;   // box = the tile's w rows of B
                 for (int kb = 0; kb < kblocks; ++kb, ++it) {
                     const uint32_t stage = it % stages, ph = (it / stages) & 1u;
                     if (!mbar_wait(smem_u32(&aux->empty[stage]), ph ^ 1u, abort_flag)) continue;
                     const uint32_t full = smem_u32(&aux->full[stage]);
                     const uint32_t dst = smem_base + stage * sbytes;
-                    const int boxes = tile_width(tile) / kBN, col0 = tile_col0(tile);
-                    mbar_arrive_expect_tx(full, (uint32_t)((rb + boxes) * kTileBytes));
-                    for (int r = 0; r < rb; ++r) tma_load_2d_hint(dst + r * kTileBytes, &amap, full, kb * kBK, r * kBM, keep_policy);
-                    for (int bx = 0; bx < boxes; ++bx)      // 128 rows of B each, back to back: one K-major operand of 256 rows
-                        tma_load_2d_hint(dst + (rb + bx) * kTileBytes, &bmap, full, kb * kBK, col0 + bx * kBN, stream_policy);
+                    mbar_arrive_expect_tx(full, (uint32_t)(p.a_bytes + w * kBK * 2));
+                    for (int r = 0; r < rb; ++r)       // the last row block's box is as high as its valid rows (rounded up to 8)
+                        tma_load_2d_hint(dst + r * kTileBytes, r + 1 < rb ? &amap : &amap_last, full, kb * kBK, r * kBM, keep_policy);
+                    tma_load_2d_hint(dst + p.a_bytes, bmap, full, kb * kBK, col0, stream_policy);
                     issued = it + 1;
                 }
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            constexpr uint32_t idesc_128 = umma_idesc_16bit(kBM, kBN, 0, 0, false), idesc_256 = umma_idesc_16bit(kBM, 2 * kBN, 0, 0, false);
             uint32_t it = 0, tcount = 0;
-            for (int tile = blockIdx.x; tile < p.n_tiles; tile += gridDim.x, ++tcount) {
+            for (int t = 0; t < p.rounds; ++t, ++tcount) {
+                if (tile_col0(t) >= p.N) break;
                 const uint32_t buf = tcount % nbuf, acc_ph = (tcount / nbuf) & 1u;
-                const uint32_t idesc = tile_width(tile) == kBN ? idesc_128 : idesc_256;
+                const uint32_t idesc = umma_idesc_16bit(kBM, tile_width(t), 0, 0, false);
                 bool ok = mbar_wait(smem_u32(&aux->acc_empty[buf]), acc_ph ^ 1u, abort_flag);   // the epilogue has read this buffer
                 tc_fence_after();
                 for (int kb = 0; kb < kblocks; ++kb, ++it) {
@@ -153,7 +176,7 @@ gemm_umma_kernel(const GemmParams p, const __grid_constant__ CUtensorMap amap, c
                     tc_fence_after();
                     if (ok) {
                         const uint32_t a0 = smem_base + stage * sbytes;
-                        const uint64_t bdesc = umma_smem_desc_sw128(a0 + rb * kTileBytes, 16, 1024);
+                        const uint64_t bdesc = umma_smem_desc_sw128(a0 + p.a_bytes, 16, 1024);
                         for (int r = 0; r < rb; ++r) {
                             const uint64_t adesc = umma_smem_desc_sw128(a0 + r * kTileBytes, 16, 1024);
                             const uint32_t d = tmem + buf * (uint32_t)(rb * wmax) + r * wmax;
@@ -171,11 +194,16 @@ gemm_umma_kernel(const GemmParams p, const __grid_constant__ CUtensorMap amap, c
         const int lane_row = (warp & 3) * 32 + lane;                    // TMEM lane = row inside a row block
         const uint32_t lane_sel = (uint32_t)((warp & 3) * 32) << 16;
         uint32_t tcount = 0;
-        for (int tile = blockIdx.x; tile < p.n_tiles; tile += gridDim.x, ++tcount) {
+        for (int t = 0; t < p.rounds; ++t, ++tcount) {
+            const int n0 = tile_col0(t);
+            if (n0 >= p.N) break;
             const uint32_t buf = tcount % nbuf, acc_ph = (tcount / nbuf) & 1u;
             const bool ok = mbar_wait(smem_u32(&aux->acc_full[buf]), acc_ph, abort_flag);
             tc_fence_after();
-            const int n0 = tile_col0(tile), chunks = tile_width(tile) / 32;
+            // columns [n0, n_end) are this tile's; a width that is an odd multiple of 16 leaves half of the last chunk
+            // of 32 unused (those columns of tensor memory hold another tile's or no data)
+            const int n_end = n0 + tile_width(t) < p.N ? n0 + tile_width(t) : p.N;
+            const int chunks = (tile_width(t) + 31) / 32;
             for (int r = 0; r < rb; ++r) {
                 const int row = r * kBM + lane_row;
                 const uint32_t taddr = tmem + lane_sel + buf * (uint32_t)(rb * wmax) + r * wmax;
@@ -194,16 +222,16 @@ gemm_umma_kernel(const GemmParams p, const __grid_constant__ CUtensorMap amap, c
                             // NaN reads as -inf; strict '>' keeps the lowest column among equal values
                             const float x = __uint_as_float(v[j]);
                             const float e = x != x ? -INFINITY : x;
-                            if (col0 + j < p.N && (bi == 0xffffffffu || e > bv)) { bv = e; bi = (uint32_t)(col0 + j); }
+                            if (col0 + j < n_end && (bi == 0xffffffffu || e > bv)) { bv = e; bi = (uint32_t)(col0 + j); }
                         }
                     } else {
                         float* dst = p.c + (long long)row * p.ldc + col0;
-                        if (col0 + 32 <= p.N && ((reinterpret_cast<uintptr_t>(dst) & 15) == 0)) {
+                        if (col0 + 32 <= n_end && ((reinterpret_cast<uintptr_t>(dst) & 15) == 0)) {
 #pragma unroll
                             for (int j = 0; j < 8; ++j)
                                 reinterpret_cast<uint4*>(dst)[j] = make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
                         } else {
-                            for (int j = 0; j < 32 && col0 + j < p.N; ++j) dst[j] = __uint_as_float(v[j]);
+                            for (int j = 0; j < 32 && col0 + j < n_end; ++j) dst[j] = __uint_as_float(v[j]);
                         }
                     }
                 }
@@ -234,13 +262,14 @@ gemm_umma_kernel(const GemmParams p, const __grid_constant__ CUtensorMap amap, c
     }
 }
 
-// Row-major bf16 matrix [rows, K] as a 2-D tensor map with boxes of 64 columns x 128 rows (128-byte swizzle): one box
-// is one operand tile in the canonical K-major layout.  Rows past the end read as zeros.
-inline int make_operand_map(EncodeTiledFn encode, CUtensorMap* map, const void* ptr, long long rows, long long K) {
+// Row-major bf16 matrix [rows, K] as a 2-D tensor map with boxes of 64 columns x box_rows rows (128-byte swizzle; a
+// multiple of 8 rows up to 256): one box is one operand tile in the canonical K-major layout.  Rows past the end read
+// as zeros.
+inline int make_operand_map(EncodeTiledFn encode, CUtensorMap* map, const void* ptr, long long rows, long long K, int box_rows) {
     if (!encode) return -1;
     const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
     const cuuint64_t strides[1] = {(cuuint64_t)K * 2};
-    const cuuint32_t box[2] = {kBK, kBM};
+    const cuuint32_t box[2] = {kBK, (cuuint32_t)box_rows};
     const cuuint32_t elem_strides[2] = {1, 1};
     return (int)encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, elem_strides,
                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -255,15 +284,21 @@ __global__ void __launch_bounds__(kArgmaxThreads) accept_walk_kernel(const Accep
 }  // namespace gemm_path
 
 // ------------------------------------------------------------------------------------------------------------
-// The drafter cell's element-wise half (Eq. 2, 5-8): one CTA per row over the fp32 pre-activations
+// The drafter cell's element-wise half (Eq. 2, 5-8) over the fp32 pre-activations
 // S = h [W^f; W^i; W^o; W^c]^T ([rows, 4d]).  f = layer normalisation (biased variance, eps inside the root,
 // optional affine) followed by exact GeLU.
+// A row is spread over a cluster of 8 CTAs (a handful of rows would otherwise sit on a handful of SMs: 10 rows of
+// 12288 took 30 us on one CTA each).  The four row statistics (mean and variance of s^c and of z') are sums over the
+// whole row: every CTA leaves its partial in its own shared memory, the cluster synchronises, and every CTA adds the
+// eight partials in rank order out of distributed shared memory, so all of them hold the same value.
 // ------------------------------------------------------------------------------------------------------------
-constexpr int kCellThreads = 1024;
-constexpr int kCellPerThread = 16;               // d <= 16384
+constexpr int kCellCluster = 8;
+constexpr int kCellThreads = 512;
+constexpr int kCellPerThread = 4;                // d <= 8 * 512 * 4 = 16384
+constexpr int kCellMaxD = kCellCluster * kCellThreads * kCellPerThread;
 
 struct CellParams {
-    const float* s;                  // [rows, 4d]
+    const float* s;                  // [rows, 4d]: W^f h, W^i h, W^o h, W^c h
     const __nv_bfloat16* emb;        // [rows, d]  E(t), Eq. 1
     const float* gamma_c; const float* beta_c;   // affine of f in Eq. 6 (may be null)
     const float* gamma_z; const float* beta_z;   // affine of f in Eq. 8 (may be null)
@@ -274,84 +309,98 @@ struct CellParams {
     float alpha, eps;
 };
 
-__device__ __forceinline__ float block_sum(float v, float* s_red) {
+// Sum of v over all threads of the cluster.  `slot` (0..3) names this reduction's cell in s_cta, so that no cell is
+// written twice while a peer may still read it; s_warp is free again once the cluster barrier has been passed.
+__device__ __forceinline__ float cluster_sum(float v, float* s_warp, float* s_cta, int slot) {
+    namespace cg = cooperative_groups;
+    cg::cluster_group cluster = cg::this_cluster();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-    __syncthreads();                 // s_red may still be read from the call before
-    if (lane == 0) s_red[warp] = v;
+    if (lane == 0) s_warp[warp] = v;
     __syncthreads();
-    float t = lane < kCellThreads / 32 ? s_red[lane] : 0.f;
+    if (warp == 0) {
+        float t = lane < kCellThreads / 32 ? s_warp[lane] : 0.f;
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
-    return t;
+        for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+        if (lane == 0) s_cta[slot] = t;
+    }
+    cluster.sync();
+    float total = 0.f;
+#pragma unroll
+    for (int r = 0; r < kCellCluster; ++r) total += cluster.map_shared_rank(s_cta, r)[slot];
+    return total;
 }
 
 __device__ __forceinline__ float gelu_exact(float x) { return 0.5f * x * (1.f + erff(x * 0.70710678118654752f)); }
 __device__ __forceinline__ float sigmoid_f(float x) { return 1.f / (1.f + __expf(-x)); }
 
-__global__ void __launch_bounds__(kCellThreads) lstm_cell_kernel(const CellParams p) {
-    __shared__ float s_red[kCellThreads / 32];
-    const long long row = blockIdx.x;
+__global__ void __cluster_dims__(kCellCluster, 1, 1) __launch_bounds__(kCellThreads) lstm_cell_kernel(const CellParams p) {
+    namespace cg = cooperative_groups;
+    __shared__ float s_warp[kCellThreads / 32];
+    __shared__ float s_cta[4];
+    cg::cluster_group cluster = cg::this_cluster();
+    // may be launched as a programmatic dependent of the product that writes S
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const long long row = blockIdx.x / kCellCluster;
     const int d = p.d;
+    const int slice = (d + kCellCluster - 1) / kCellCluster;
+    const int j0 = (int)cluster.block_rank() * slice;             // this CTA's columns: [j0, min(j0 + slice, d))
     const float* s = p.s + row * 4ll * d;
-    float xc[kCellPerThread], gi[kCellPerThread], zn[kCellPerThread];
+    float xc[kCellPerThread], ae[kCellPerThread], zn[kCellPerThread];
+    bool on[kCellPerThread];
     // s^c = W^c h + alpha e; its mean and variance over the d outputs (two passes over registers)
     float sum = 0.f;
 #pragma unroll
     for (int k = 0; k < kCellPerThread; ++k) {
-        const int j = k * kCellThreads + threadIdx.x;
-        xc[k] = 0.f;
-        if (j < d) { xc[k] = s[3ll * d + j] + p.alpha * __bfloat162float(p.emb[row * d + j]); sum += xc[k]; }
+        const int i = k * kCellThreads + threadIdx.x, j = j0 + i;
+        on[k] = i < slice && j < d;
+        xc[k] = 0.f; ae[k] = 0.f;
+        if (on[k]) { ae[k] = p.alpha * __bfloat162float(p.emb[row * d + j]); xc[k] = s[3ll * d + j] + ae[k]; sum += xc[k]; }
     }
-    const float mean_c = block_sum(sum, s_red) / d;
+    const float mean_c = cluster_sum(sum, s_warp, s_cta, 0) / d;
     float sq = 0.f;
 #pragma unroll
-    for (int k = 0; k < kCellPerThread; ++k) {
-        const int j = k * kCellThreads + threadIdx.x;
-        if (j < d) { const float t = xc[k] - mean_c; sq += t * t; }
-    }
-    const float rstd_c = rsqrtf(block_sum(sq, s_red) / d + p.eps);
+    for (int k = 0; k < kCellPerThread; ++k)
+        if (on[k]) { const float t = xc[k] - mean_c; sq += t * t; }
+    const float rstd_c = rsqrtf(cluster_sum(sq, s_warp, s_cta, 1) / d + p.eps);
     // z' = z g^f + f(s^c) g^i  (Eq. 5-7)
     sum = 0.f;
 #pragma unroll
     for (int k = 0; k < kCellPerThread; ++k) {
-        const int j = k * kCellThreads + threadIdx.x;
+        const int j = j0 + k * kCellThreads + threadIdx.x;
         zn[k] = 0.f;
-        if (j < d) {
-            const float ae = p.alpha * __bfloat162float(p.emb[row * d + j]);
+        if (on[k]) {
             float y = (xc[k] - mean_c) * rstd_c;
             if (p.gamma_c) y *= p.gamma_c[j];
             if (p.beta_c) y += p.beta_c[j];
-            gi[k] = sigmoid_f(s[1ll * d + j] + ae);
-            const float gf = sigmoid_f(s[j] + ae);
-            zn[k] = p.z[row * d + j] * gf + gelu_exact(y) * gi[k];
+            const float gi = sigmoid_f(s[1ll * d + j] + ae[k]);
+            const float gf = sigmoid_f(s[j] + ae[k]);
+            zn[k] = p.z[row * d + j] * gf + gelu_exact(y) * gi;
             p.z[row * d + j] = zn[k];
             sum += zn[k];
         }
     }
-    const float mean_z = block_sum(sum, s_red) / d;
+    const float mean_z = cluster_sum(sum, s_warp, s_cta, 2) / d;
     sq = 0.f;
 #pragma unroll
-    for (int k = 0; k < kCellPerThread; ++k) {
-        const int j = k * kCellThreads + threadIdx.x;
-        if (j < d) { const float t = zn[k] - mean_z; sq += t * t; }
-    }
-    const float rstd_z = rsqrtf(block_sum(sq, s_red) / d + p.eps);
+    for (int k = 0; k < kCellPerThread; ++k)
+        if (on[k]) { const float t = zn[k] - mean_z; sq += t * t; }
+    const float rstd_z = rsqrtf(cluster_sum(sq, s_warp, s_cta, 3) / d + p.eps);
     // h' = f(z') g^o  (Eq. 8)
 #pragma unroll
     for (int k = 0; k < kCellPerThread; ++k) {
-        const int j = k * kCellThreads + threadIdx.x;
-        if (j < d) {
+        const int j = j0 + k * kCellThreads + threadIdx.x;
+        if (on[k]) {
             float y = (zn[k] - mean_z) * rstd_z;
             if (p.gamma_z) y *= p.gamma_z[j];
             if (p.beta_z) y += p.beta_z[j];
-            const float go = sigmoid_f(s[2ll * d + j] + p.alpha * __bfloat162float(p.emb[row * d + j]));
-            const float h = gelu_exact(y) * go;
+            const float h = gelu_exact(y) * sigmoid_f(s[2ll * d + j] + ae[k]);
             if (p.h_f32) p.h_f32[row * d + j] = h;
             if (p.h_bf16) p.h_bf16[row * d + j] = __float2bfloat16_rn(h);
         }
     }
+    cluster.sync();      // no CTA leaves while a peer may still read its partials
 }
 
 }  // namespace owl

@@ -180,22 +180,32 @@ static int launch_gemm(owl_ctx* ctx, const void* a, const void* b, int M, int N,
     gemm_path::GemmParams g{};
     g.M = M; g.N = N; g.K = K;
     g.row_blocks = (M + gemm_path::kBM - 1) / gemm_path::kBM;
-    g.stages = gemm_path::ring_stages(g.row_blocks);
-    // as many full rounds of 256-column tiles as there are CTAs, the remaining columns in 128-wide tiles
-    const int wide_cap = gemm_path::b_boxes(g.row_blocks) == 2 ? N / (2 * gemm_path::kBN) : 0;
-    g.wide_tiles = wide_cap >= ctx->sm_count ? (wide_cap / ctx->sm_count) * ctx->sm_count : 0;
-    g.n_tiles = g.wide_tiles + (N - g.wide_tiles * 2 * gemm_path::kBN + gemm_path::kBN - 1) / gemm_path::kBN;
+    // every CTA gets the same number of 16-column units, cut into as few tiles as the width limit allows
+    const int units = (N + 15) / 16;
+    const int grid = units < ctx->sm_count ? units : ctx->sm_count;
+    const int per_cta = (units + grid - 1) / grid;
+    const int wmax_units = gemm_path::b_boxes(g.row_blocks) * gemm_path::kBN / 16;
+    g.rounds = (per_cta + wmax_units - 1) / wmax_units;
+    g.w_lo = per_cta / g.rounds * 16;
+    g.wide_rounds = per_cta % g.rounds;
+    // a stage: the rows of A that exist (the last row block rounded up to 8 rows) and the widest tile's rows of B
+    const int last_rows = (M - (g.row_blocks - 1) * gemm_path::kBM + 7) / 8 * 8;
+    g.a_bytes = (g.row_blocks - 1) * gemm_path::kTileBytes + last_rows * gemm_path::kBK * 2;
+    g.stage_bytes = g.a_bytes + (g.w_lo + (g.wide_rounds ? 16 : 0)) * gemm_path::kBK * 2;
+    g.stages = gemm_path::ring_stages(g.stage_bytes);
     g.status = ctx->status;
     g.row_key = row_key; g.c = c; g.ldc = ldc;
-    CUtensorMap amap, bmap;
-    const int ra = gemm_path::make_operand_map(ctx->encode, &amap, a, M, K);
-    const int rb = gemm_path::make_operand_map(ctx->encode, &bmap, b, N, K);
+    CUtensorMap amap, amap_last, bmap_hi, bmap_lo;
+    int ra = gemm_path::make_operand_map(ctx->encode, &amap, a, M, K, gemm_path::kBM);
+    if (ra == 0) ra = gemm_path::make_operand_map(ctx->encode, &amap_last, a, M, K, last_rows);
+    int rb = gemm_path::make_operand_map(ctx->encode, &bmap_lo, b, N, K, g.w_lo);
+    if (rb == 0) rb = g.wide_rounds ? gemm_path::make_operand_map(ctx->encode, &bmap_hi, b, N, K, g.w_lo + 16) : (bmap_hi = bmap_lo, 0);
     if (ra != 0 || rb != 0) {
         snprintf(ctx->err, sizeof ctx->err, "cuTensorMapEncodeTiled failed (%d, %d): operands must be 16-byte aligned", ra, rb);
         return OWL_ERR_CUDA;
     }
-    const int grid = g.n_tiles < ctx->sm_count ? g.n_tiles : ctx->sm_count;
-    gemm_path::gemm_umma_kernel<kEpi><<<grid, gemm_path::kThreads, gemm_path::smem_bytes(g.row_blocks), stream>>>(g, amap, bmap);
+    gemm_path::gemm_umma_kernel<kEpi><<<grid, gemm_path::kThreads, gemm_path::smem_bytes(g.stages, g.stage_bytes), stream>>>(g, amap, amap_last, bmap_hi,
+                                                                                                      bmap_lo);
     ++ctx->launches;
     return OWL_OK;
 }
@@ -645,7 +655,7 @@ int owl_lstm_cell(owl_ctx* ctx, int32_t rows, int32_t d_in, int32_t d, const voi
                   float* z, float* h_out_f32, void* h_out_bf16, float* workspace, void* stream_) {
     if (!ctx || !h || !emb || !w || !z || !workspace || (!h_out_f32 && !h_out_bf16)) return OWL_ERR_INVALID_ARG;
     if (rows < 1 || d < 1 || d_in < gemm_path::kBK || !(eps >= 0.f) || alpha != alpha) return OWL_ERR_INVALID_ARG;
-    if (d_in % gemm_path::kBK != 0 || rows > gemm_path::kMaxRowBlocks * gemm_path::kBM || d > kCellThreads * kCellPerThread ||
+    if (d_in % gemm_path::kBK != 0 || rows > gemm_path::kMaxRowBlocks * gemm_path::kBM || d > kCellMaxD ||
         d % 4 != 0)
         return OWL_ERR_UNSUPPORTED;
     DeviceGuard guard(ctx->device);
@@ -657,7 +667,7 @@ int owl_lstm_cell(owl_ctx* ctx, int32_t rows, int32_t d_in, int32_t d, const voi
     c.gamma_c = ln_c_gamma; c.beta_c = ln_c_beta; c.gamma_z = ln_z_gamma; c.beta_z = ln_z_beta;
     c.z = z; c.h_f32 = h_out_f32; c.h_bf16 = static_cast<__nv_bfloat16*>(h_out_bf16);
     c.d = d; c.alpha = alpha; c.eps = eps;
-    lstm_cell_kernel<<<rows, kCellThreads, 0, stream>>>(c);
+    launch_dependent(lstm_cell_kernel, dim3((unsigned)rows * kCellCluster), dim3(kCellThreads), stream, c);
     ++ctx->launches;
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(ctx, e, "owl_lstm_cell launch");
