@@ -88,6 +88,9 @@ def _lm_head_case(ctx, seed, trees, K, V, plant=0.7):
     ([("tree", 64, 8)] * 3 + [("chain", 8)], 256, 5000),            # 200 rows: two row blocks, double-buffered accumulators
     ([("tree", 64, 8)] * 5, 512, 3000),                             # 320 rows: three row blocks, one accumulator buffer
     ([("tree", 32, 6)], 4096, 20000),                               # the real hidden width: 64 k-blocks per tile
+    ([("tree", 64, 8)] * 3, 64, 40000),                             # two row blocks, two rounds of tiles (144 + 128 columns)
+    ([("tree", 64, 8)] * 5, 64, 20000),                             # three row blocks, two rounds (80 + 64 columns)
+    ([("chain", 5)], 64, 16),                                       # the whole vocabulary is one 16-column tile on one CTA
 ])
 def test_lm_head_accept_small(trees, K, V):
     ctx = OwlContext(make_dims(batch=8, total_nodes=384, max_nodes=64, vocab=V))
@@ -160,6 +163,8 @@ def _cell_case(ctx, seed, M, d_in, d, affine, steps=1):
     (5, 128, 260, True),            # d no multiple of the column tile: ragged last tile of the product
     (130, 256, 512, True),          # two row blocks
     (300, 64, 128, False),          # three row blocks
+    (2, 64, 4, True),               # fewer columns than CTAs in a row's cluster: half of them hold none
+    (1, 64, 16384, True),           # the widest cell: four columns per thread, two rounds of product tiles
 ])
 def test_lstm_cell_small(M, d_in, d, affine):
     ctx = OwlContext(make_dims(batch=1, total_nodes=1, max_nodes=1))
