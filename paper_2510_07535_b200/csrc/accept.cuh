@@ -227,6 +227,7 @@ __device__ __forceinline__ void argmax_scan_chunk_warp(const AcceptParams& p, co
 constexpr int kArgmaxWarps = kArgmaxThreads / 32;
 constexpr int kArgmaxCtasPerSm = 2;     // what fits at the kernel's register count
 constexpr int kArgmaxNoteMax = 64;
+constexpr int kArgmaxOffsMax = 1024;            // sequences whose packed offsets a CTA keeps in shared memory
 
 __global__ void __launch_bounds__(kArgmaxThreads) argmax_partial_kernel(const AcceptParams p) {
     // may be launched as a programmatic dependent of the kernel before it in the stream: nothing is read
@@ -235,7 +236,13 @@ __global__ void __launch_bounds__(kArgmaxThreads) argmax_partial_kernel(const Ac
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next kernel may queue up; it waits likewise
     __shared__ int s_note[kArgmaxNoteMax];
     __shared__ int s_notes;
+    // packed offsets of up to kArgmaxOffsMax sequences: every item looks its sequence up by binary search, and from
+    // global memory that is log2(B) dependent round trips per item with the warp's loads drained
+    __shared__ int s_offs[kArgmaxOffsMax + 1];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const bool offs_staged = p.node_offsets && p.batch <= kArgmaxOffsMax;
+    if (offs_staged)
+        for (int b = threadIdx.x; b <= p.batch; b += kArgmaxThreads) s_offs[b] = p.node_offsets[b];
     if (threadIdx.x == 0) s_notes = 0;
     if (blockIdx.x == 0) {
         // Once per call: clear every counter of the idle set (the next call counts there, whatever its batch), and
@@ -263,10 +270,11 @@ __global__ void __launch_bounds__(kArgmaxThreads) argmax_partial_kernel(const Ac
             // which sequence owns this row, and is this the last of its chunk keys?
             int b, n_b;
             if (p.node_offsets) {
+                const int* offs = offs_staged ? s_offs : p.node_offsets;
                 int lo = 0, hi = p.batch;   // largest b with node_offsets[b] <= row
-                while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (p.node_offsets[mid] <= row) lo = mid; else hi = mid; }
+                while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (offs[mid] <= row) lo = mid; else hi = mid; }
                 b = lo;
-                n_b = p.node_offsets[b + 1] - p.node_offsets[b];
+                n_b = offs[b + 1] - offs[b];
             } else {
                 b = row / p.nodes_uniform;
                 n_b = p.nodes_uniform;
