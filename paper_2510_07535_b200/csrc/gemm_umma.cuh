@@ -288,9 +288,8 @@ __global__ void __launch_bounds__(kArgmaxThreads) accept_walk_kernel(const Accep
 // S = h [W^f; W^i; W^o; W^c]^T ([rows, 4d]).  f = layer normalisation (biased variance, eps inside the root,
 // optional affine) followed by exact GeLU.
 // A row is spread over a cluster of 8 CTAs (a handful of rows would otherwise sit on a handful of SMs: 10 rows of
-// 12288 took 30 us on one CTA each).  The four row statistics (mean and variance of s^c and of z') are sums over the
-// whole row: every CTA leaves its partial in its own shared memory, the cluster synchronises, and every CTA adds the
-// eight partials in rank order out of distributed shared memory, so all of them hold the same value.
+// 12288 took 30 us on one CTA each).  The statistics of the two layer normalisations are over the whole row: one
+// exchange through distributed shared memory and one cluster barrier each (cluster_mean_rstd).
 // ------------------------------------------------------------------------------------------------------------
 constexpr int kCellCluster = 8;
 constexpr int kCellThreads = 512;
@@ -309,27 +308,61 @@ struct CellParams {
     float alpha, eps;
 };
 
-// Sum of v over all threads of the cluster.  `slot` (0..3) names this reduction's cell in s_cta, so that no cell is
-// written twice while a peer may still read it; s_warp is free again once the cluster barrier has been passed.
-__device__ __forceinline__ float cluster_sum(float v, float* s_warp, float* s_cta, int slot) {
-    namespace cg = cooperative_groups;
-    cg::cluster_group cluster = cg::this_cluster();
+// Sum of v over the CTA's threads; s_warp is free again after the second barrier.
+__device__ __forceinline__ float cell_block_sum(float v, float* s_warp) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
     if (lane == 0) s_warp[warp] = v;
     __syncthreads();
-    if (warp == 0) {
-        float t = lane < kCellThreads / 32 ? s_warp[lane] : 0.f;
+    float t = lane < kCellThreads / 32 ? s_warp[lane] : 0.f;
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
-        if (lane == 0) s_cta[slot] = t;
+    for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+    __syncthreads();
+    return t;
+}
+
+// Mean and 1 / sqrt(variance + eps) over a whole row from the values x[] this thread holds (on[] says which exist).
+// Each CTA takes the mean and the sum of squared deviations of its own `count` columns (two block reductions), pushes
+// the pair into slot `which` of every CTA of the cluster, and after one cluster barrier all of them combine the eight
+// pairs in rank order by the pairwise-variance identity  M2 = sum_i M2_i + sum_i n_i (mean_i - mean)^2 : the same
+// numbers everywhere, no cancellation, and nobody reads a peer's shared memory after the barrier.
+__device__ __forceinline__ void cluster_mean_rstd(const float (&x)[kCellPerThread], const bool (&on)[kCellPerThread], int count,
+                                                  int slice, int d, float eps, float* s_warp, float (*s_stat)[kCellCluster][2],
+                                                  int which, float& mean, float& rstd) {
+    namespace cg = cooperative_groups;
+    cg::cluster_group cluster = cg::this_cluster();
+    float sum = 0.f;
+#pragma unroll
+    for (int k = 0; k < kCellPerThread; ++k) sum += on[k] ? x[k] : 0.f;
+    const float mean_cta = count > 0 ? cell_block_sum(sum, s_warp) / count : (cell_block_sum(sum, s_warp), 0.f);
+    float sq = 0.f;
+#pragma unroll
+    for (int k = 0; k < kCellPerThread; ++k)
+        if (on[k]) { const float t = x[k] - mean_cta; sq += t * t; }
+    const float m2_cta = cell_block_sum(sq, s_warp);
+    const int rank = (int)cluster.block_rank();
+    if (threadIdx.x < kCellCluster) {
+        float* dst = &cluster.map_shared_rank(s_stat, threadIdx.x)[which][rank][0];
+        dst[0] = mean_cta;
+        dst[1] = m2_cta;
     }
     cluster.sync();
     float total = 0.f;
 #pragma unroll
-    for (int r = 0; r < kCellCluster; ++r) total += cluster.map_shared_rank(s_cta, r)[slot];
-    return total;
+    for (int r = 0; r < kCellCluster; ++r) {
+        const int n_r = min(slice, max(d - r * slice, 0));
+        total += (float)n_r * s_stat[which][r][0];
+    }
+    mean = total / d;
+    float m2 = 0.f;
+#pragma unroll
+    for (int r = 0; r < kCellCluster; ++r) {
+        const int n_r = min(slice, max(d - r * slice, 0));
+        const float dm = s_stat[which][r][0] - mean;
+        m2 += s_stat[which][r][1] + (float)n_r * dm * dm;
+    }
+    rstd = rsqrtf(m2 / d + eps);
 }
 
 __device__ __forceinline__ float gelu_exact(float x) { return 0.5f * x * (1.f + erff(x * 0.70710678118654752f)); }
@@ -338,7 +371,7 @@ __device__ __forceinline__ float sigmoid_f(float x) { return 1.f / (1.f + __expf
 __global__ void __cluster_dims__(kCellCluster, 1, 1) __launch_bounds__(kCellThreads) lstm_cell_kernel(const CellParams p) {
     namespace cg = cooperative_groups;
     __shared__ float s_warp[kCellThreads / 32];
-    __shared__ float s_cta[4];
+    __shared__ float s_stat[2][kCellCluster][2];     // [which normalisation][CTA of the cluster][mean, M2]
     cg::cluster_group cluster = cg::this_cluster();
     // may be launched as a programmatic dependent of the product that writes S
     asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -346,47 +379,39 @@ __global__ void __cluster_dims__(kCellCluster, 1, 1) __launch_bounds__(kCellThre
     const int d = p.d;
     const int slice = (d + kCellCluster - 1) / kCellCluster;
     const int j0 = (int)cluster.block_rank() * slice;             // this CTA's columns: [j0, min(j0 + slice, d))
+    const int count = min(slice, max(d - j0, 0));
     const float* s = p.s + row * 4ll * d;
-    float xc[kCellPerThread], ae[kCellPerThread], zn[kCellPerThread];
+    // everything a column needs is asked for at once: the four pre-activations, E(t) and z
+    float xc[kCellPerThread], sf[kCellPerThread], si[kCellPerThread], so[kCellPerThread], zo[kCellPerThread], zn[kCellPerThread];
     bool on[kCellPerThread];
-    // s^c = W^c h + alpha e; its mean and variance over the d outputs (two passes over registers)
-    float sum = 0.f;
 #pragma unroll
     for (int k = 0; k < kCellPerThread; ++k) {
         const int i = k * kCellThreads + threadIdx.x, j = j0 + i;
         on[k] = i < slice && j < d;
-        xc[k] = 0.f; ae[k] = 0.f;
-        if (on[k]) { ae[k] = p.alpha * __bfloat162float(p.emb[row * d + j]); xc[k] = s[3ll * d + j] + ae[k]; sum += xc[k]; }
+        xc[k] = sf[k] = si[k] = so[k] = zo[k] = zn[k] = 0.f;
+        if (on[k]) {
+            const float ae = p.alpha * __bfloat162float(p.emb[row * d + j]);     // s^m = W^m h + alpha e  (Eq. 2)
+            sf[k] = s[j] + ae; si[k] = s[1ll * d + j] + ae; so[k] = s[2ll * d + j] + ae; xc[k] = s[3ll * d + j] + ae;
+            zo[k] = p.z[row * d + j];
+        }
     }
-    const float mean_c = cluster_sum(sum, s_warp, s_cta, 0) / d;
-    float sq = 0.f;
-#pragma unroll
-    for (int k = 0; k < kCellPerThread; ++k)
-        if (on[k]) { const float t = xc[k] - mean_c; sq += t * t; }
-    const float rstd_c = rsqrtf(cluster_sum(sq, s_warp, s_cta, 1) / d + p.eps);
+    cluster.sync();      // every CTA of the cluster is running before anyone writes into its shared memory (the loads fly)
+    float mean_c, rstd_c;
+    cluster_mean_rstd(xc, on, count, slice, d, p.eps, s_warp, s_stat, 0, mean_c, rstd_c);
     // z' = z g^f + f(s^c) g^i  (Eq. 5-7)
-    sum = 0.f;
 #pragma unroll
     for (int k = 0; k < kCellPerThread; ++k) {
         const int j = j0 + k * kCellThreads + threadIdx.x;
-        zn[k] = 0.f;
         if (on[k]) {
             float y = (xc[k] - mean_c) * rstd_c;
             if (p.gamma_c) y *= p.gamma_c[j];
             if (p.beta_c) y += p.beta_c[j];
-            const float gi = sigmoid_f(s[1ll * d + j] + ae[k]);
-            const float gf = sigmoid_f(s[j] + ae[k]);
-            zn[k] = p.z[row * d + j] * gf + gelu_exact(y) * gi;
+            zn[k] = zo[k] * sigmoid_f(sf[k]) + gelu_exact(y) * sigmoid_f(si[k]);
             p.z[row * d + j] = zn[k];
-            sum += zn[k];
         }
     }
-    const float mean_z = cluster_sum(sum, s_warp, s_cta, 2) / d;
-    sq = 0.f;
-#pragma unroll
-    for (int k = 0; k < kCellPerThread; ++k)
-        if (on[k]) { const float t = zn[k] - mean_z; sq += t * t; }
-    const float rstd_z = rsqrtf(cluster_sum(sq, s_warp, s_cta, 3) / d + p.eps);
+    float mean_z, rstd_z;
+    cluster_mean_rstd(zn, on, count, slice, d, p.eps, s_warp, s_stat, 1, mean_z, rstd_z);
     // h' = f(z') g^o  (Eq. 8)
 #pragma unroll
     for (int k = 0; k < kCellPerThread; ++k) {
@@ -395,12 +420,11 @@ __global__ void __cluster_dims__(kCellCluster, 1, 1) __launch_bounds__(kCellThre
             float y = (zn[k] - mean_z) * rstd_z;
             if (p.gamma_z) y *= p.gamma_z[j];
             if (p.beta_z) y += p.beta_z[j];
-            const float h = gelu_exact(y) * sigmoid_f(s[2ll * d + j] + ae[k]);
+            const float h = gelu_exact(y) * sigmoid_f(so[k]);
             if (p.h_f32) p.h_f32[row * d + j] = h;
             if (p.h_bf16) p.h_bf16[row * d + j] = __float2bfloat16_rn(h);
         }
     }
-    cluster.sync();      // no CTA leaves while a peer may still read its partials
 }
 
 }  // namespace owl
