@@ -106,9 +106,6 @@ gemm_umma_kernel(const GemmParams p, const __grid_constant__ CUtensorMap amap, c
     const int sbytes = p.stage_bytes;
     Aux* aux = reinterpret_cast<Aux*>(smem);
     volatile int* abort_flag = &aux->abort_flag;
-    // may be launched as a programmatic dependent of the kernel before it in the stream
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (smem_base & 1023u) {                       // operand tiles must sit on swizzle-atom boundaries
         if (tid == 0) report(p.status, kErrTimeout);
         return;
@@ -124,6 +121,11 @@ gemm_umma_kernel(const GemmParams p, const __grid_constant__ CUtensorMap amap, c
         tma_prefetch_desc(&bmap_lo);
     }
     if (warp == 0) { tmem_alloc(smem_u32(&aux->tmem_base), 512); tmem_relinquish(); }
+    // may be launched as a programmatic dependent of the kernel before it in the stream: the set-up above touched no
+    // input and ran beside that kernel's tail; from here on it has completed (a no-op in an ordinary launch).  The
+    // kernel after this one may queue up in turn; it waits likewise before it reads anything.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -373,8 +375,9 @@ __global__ void __cluster_dims__(kCellCluster, 1, 1) __launch_bounds__(kCellThre
     __shared__ float s_warp[kCellThreads / 32];
     __shared__ float s_stat[2][kCellCluster][2];     // [which normalisation][CTA of the cluster][mean, M2]
     cg::cluster_group cluster = cg::this_cluster();
-    // may be launched as a programmatic dependent of the product that writes S
+    // may be launched as a programmatic dependent of the product that writes S; the kernel after this one may queue up
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const long long row = blockIdx.x / kCellCluster;
     const int d = p.d;
     const int slice = (d + kCellCluster - 1) / kCellCluster;

@@ -81,11 +81,11 @@ int cuda_fail(owl_ctx* ctx, cudaError_t e, const char* what) {
 // Launch `kernel(arg)` so that it may be scheduled while the kernel before it in the stream is still running
 // (programmatic dependent launch); the kernel itself waits (griddepcontrol.wait) before it reads anything.
 template <typename... Args>
-cudaError_t launch_dependent(void (*kernel)(Args...), dim3 grid, dim3 block, cudaStream_t stream, const Args&... args) {
+cudaError_t launch_dependent_smem(void (*kernel)(Args...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, const Args&... args) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
     cfg.blockDim = block;
-    cfg.dynamicSmemBytes = 0;
+    cfg.dynamicSmemBytes = smem;
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -93,6 +93,10 @@ cudaError_t launch_dependent(void (*kernel)(Args...), dim3 grid, dim3 block, cud
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+template <typename... Args>
+cudaError_t launch_dependent(void (*kernel)(Args...), dim3 grid, dim3 block, cudaStream_t stream, const Args&... args) {
+    return launch_dependent_smem(kernel, grid, block, 0, stream, args...);
 }
 
 // The attention kernel's instances: [more than 32 sequences][units above 128 rows][logits scan fused in], bf16;
@@ -204,8 +208,8 @@ static int launch_gemm(owl_ctx* ctx, const void* a, const void* b, int M, int N,
         snprintf(ctx->err, sizeof ctx->err, "cuTensorMapEncodeTiled failed (%d, %d): operands must be 16-byte aligned", ra, rb);
         return OWL_ERR_CUDA;
     }
-    gemm_path::gemm_umma_kernel<kEpi><<<grid, gemm_path::kThreads, gemm_path::smem_bytes(g.stages, g.stage_bytes), stream>>>(g, amap, amap_last, bmap_hi,
-                                                                                                      bmap_lo);
+    launch_dependent_smem(gemm_path::gemm_umma_kernel<kEpi>, dim3(grid), dim3(gemm_path::kThreads),
+                          (size_t)gemm_path::smem_bytes(g.stages, g.stage_bytes), stream, g, amap, amap_last, bmap_hi, bmap_lo);
     ++ctx->launches;
     return OWL_OK;
 }
