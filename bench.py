@@ -90,6 +90,10 @@ class ClockSampler(threading.Thread):
             self.nv = pynvml
             self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
             self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+            # the first query of each kind can take tens of milliseconds: pay that here, not inside a timed region
+            pynvml.nvmlDeviceGetClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            pynvml.nvmlDeviceGetPowerUsage(self.h)
+            pynvml.nvmlDeviceGetCurrentClocksEventReasons(self.h)
         except Exception:
             self.nv = None
 
@@ -117,6 +121,9 @@ class ClockSampler(threading.Thread):
     def begin(self, _label=""):
         self.samples, self.power, self.reasons = [], [], set()
         self.active.set()
+
+    def count(self):
+        return len(self.samples)
 
     def end(self):
         self.active.clear()
@@ -269,9 +276,22 @@ def measure_workload(idx, args, ctx_factory, dev, world, rank, barrier, max_over
     # ---- the two halves on their own, same inputs, same rotation: attention (split-KV kernel + merge) and acceptance
     attn_us = max_over_ranks(np.median([_event_loop_us(lambda i: reps[(r * K + i) % copies].attn(ctx), K, barrier) for r in range(5)]))
     accept_us = max_over_ranks(np.median([_event_loop_us(lambda i: reps[(r * K + i) % copies].accept(ctx), K, barrier) for r in range(5)]))
-    clocks = sampler.end()
-    assert ctx.owl_get_status() == 0
     step_us = float(np.median(region_us))
+    topped_up = False
+    if sampler.nv is not None and sampler.count() < 8:
+        # a step of tens of microseconds: the regions can be over before the sampler has had a handful of looks.  The
+        # same steps go on, untimed, until it has (a quarter of a second at most); the record says so.
+        topped_up = True
+        t_end = time.time() + 0.25
+        i = 0
+        while sampler.count() < 8 and time.time() < t_end:
+            for _ in range(64):
+                reps[i % copies].step(ctx)
+                i += 1
+            torch.cuda.synchronize()
+    clocks = sampler.end()
+    clocks["sampled_beyond_timed_regions"] = topped_up
+    assert ctx.owl_get_status() == 0
 
     fused = launches // K == 2 and logit_b > 0     # small scan: no arg-max kernel, the attention launch reads the logits too
     rec = {
