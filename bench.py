@@ -434,6 +434,24 @@ def measure_next_rows(args, dev, barrier):
     commit()
     out["kv_commit_16_seqs_5_accepted"] = {"us": float(np.median([_event_loop_us(commit, 20, barrier) for _ in range(5)])),
                                            "note": "includes the torch fill that resets the lengths between calls"}
+    # The two rows above are bound by the Python binding's call overhead (three launches in 25-30 us of host time).
+    # Device time of the three kernels: the same calls enqueued while the GPU sits in a 20 ms sleep kernel, so that
+    # every launch is already queued when its turn comes.
+    def queued(_=0):
+        lens.fill_(1000)
+        torch.cuda.synchronize()
+        torch.cuda._sleep(40_000_000)
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev0.record()
+        for _i in range(100):
+            ctx.owl_prepare_spec_tree(pd, None, par, tok, lens, 7, *o)
+            ctx.owl_kv_commit(cd, kc, vc, table, lens, None, alen, path)
+        ev1.record()
+        torch.cuda.synchronize()
+        return ev0.elapsed_time(ev1) * 1e3 / 100
+    queued()
+    out["prepare_plus_commit_device"] = {"us": float(np.median([queued() for _ in range(5)])),
+                                         "note": "three kernels per iteration, launches pre-queued behind a sleep kernel (no host time)"}
     assert ctx.owl_get_status() == 0
     ctx.close()
     return out

@@ -552,7 +552,7 @@ static int prepare_impl(owl_ctx* ctx, const owl_dims* d, const int32_t* node_off
     p.status = ctx->status;
     p.batch = d->batch; p.total_nodes = d->total_nodes; p.nodes_uniform = d->total_nodes / d->batch;
     p.max_nodes = d->max_nodes; p.spec_token = spec_token;
-    prepare_spec_kernel<<<d->batch, kPrepareThreads, 0, static_cast<cudaStream_t>(stream_)>>>(p);
+    launch_dependent(prepare_spec_kernel, dim3((unsigned)d->batch), dim3(kPrepareThreads), static_cast<cudaStream_t>(stream_), p);
     ++ctx->launches;
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(ctx, e, "owl_prepare_spec_tree launch");
@@ -607,8 +607,9 @@ int owl_kv_commit(owl_ctx* ctx, const owl_dims* d, void* k_cache, void* v_cache,
     p.max_nodes = d->max_nodes; p.num_kv_heads = d->num_kv_heads;
     p.page_size = d->page_size; p.page_shift = log2_exact(d->page_size);
     p.max_pages_per_seq = d->max_pages_per_seq; p.num_pages = d->num_pages; p.path_stride = d->path_stride;
-    kv_commit_move_kernel<<<dim3(2u * (unsigned)d->num_kv_heads, (unsigned)d->batch), kCommitThreads, 0, stream>>>(p);
-    kv_commit_lens_kernel<<<d->batch, kCommitThreads, 0, stream>>>(p);
+    // the second kernel's wait is what keeps a length from being bumped while a CTA of the first still reads it
+    launch_dependent(kv_commit_move_kernel, dim3(2u * (unsigned)d->num_kv_heads, (unsigned)d->batch), dim3(kCommitThreads), stream, p);
+    launch_dependent(kv_commit_lens_kernel, dim3((unsigned)d->batch), dim3(kCommitThreads), stream, p);
     ctx->launches += 2;
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(ctx, e, "owl_kv_commit launch");

@@ -33,6 +33,10 @@ static_assert(kPrepareThreads >= kMaxNodes, "one thread per drafted node");
 // (Section 3.2.3); the sequences' outputs are packed one after the other, so every CTA first sums the output
 // node counts of the sequences before its own.
 __global__ void __launch_bounds__(kPrepareThreads) prepare_spec_kernel(const PrepareParams p) {
+    // may be launched as a programmatic dependent: nothing is read before the kernel before it in the stream has
+    // completed (a no-op in an ordinary launch); the kernel after this one may queue up and waits likewise
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int b = blockIdx.x, j = threadIdx.x;
     const int base = p.node_offsets ? p.node_offsets[b] : b * p.nodes_uniform;
     const int n = p.node_offsets ? p.node_offsets[b + 1] - base : p.nodes_uniform;
@@ -136,6 +140,10 @@ __device__ __forceinline__ int commit_verdict(const CommitParams& p, int b, int&
 // grid (2 * Hkv, B): blockIdx.x = 2 * head + (0: K, 1: V).  Every source row is read into shared memory before any
 // destination is written, because a position can be the source of one move and the destination of a later one.
 __global__ void __launch_bounds__(kCommitThreads) kv_commit_move_kernel(const CommitParams p) {
+    // may be launched as a programmatic dependent: nothing is read before the kernel before it in the stream has
+    // completed (a no-op in an ordinary launch); the kernel after this one may queue up and waits likewise
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     __shared__ uint4 s_rows[kMaxNodes * 16];       // up to 64 rows of 128 bf16
     __shared__ int s_path[kMaxNodes];
     __shared__ int s_flag;
@@ -162,6 +170,10 @@ __global__ void __launch_bounds__(kCommitThreads) kv_commit_move_kernel(const Co
 
 // One CTA per sequence, after the move kernel in stream order: the committed length grows by accept_len.
 __global__ void __launch_bounds__(kCommitThreads) kv_commit_lens_kernel(const CommitParams p) {
+    // may be launched as a programmatic dependent: nothing is read before the kernel before it in the stream has
+    // completed (a no-op in an ordinary launch); the kernel after this one may queue up and waits likewise
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     __shared__ int s_path[kMaxNodes];
     __shared__ int s_flag;
     int L, n, a;
