@@ -278,8 +278,13 @@ inline int make_operand_map(EncodeTiledFn encode, CUtensorMap* map, const void* 
                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
 }
 
-// One sequence's acceptance walk per CTA over one key per row (the arg-max the product's epilogue left).
-__global__ void __launch_bounds__(kArgmaxThreads) accept_walk_kernel(const AcceptParams p) {
+// One sequence's acceptance walk per CTA over one key per row (the arg-max the product's epilogue left).  The grid
+// also clears `idle_keys[0, idle_len)`, the key set the next call's product will raise (nothing of this call uses it).
+// Launched as a programmatic dependent of the product: it reads nothing before the product has completed.
+__global__ void __launch_bounds__(kArgmaxThreads) accept_walk_kernel(const AcceptParams p, unsigned long long* idle_keys, int idle_len) {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    for (int i = blockIdx.x * kArgmaxThreads + threadIdx.x; i < idle_len; i += gridDim.x * kArgmaxThreads) idle_keys[i] = 0ull;
     accept_walk_seq(p, (int)blockIdx.x);
 }
 

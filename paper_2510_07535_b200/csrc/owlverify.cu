@@ -36,7 +36,8 @@ struct owl_ctx {
     long long* sched_seq_begin = nullptr;
     SchedHeader* sched_header = nullptr;
     unsigned long long* part_keys = nullptr;
-    unsigned long long* lm_keys = nullptr;      // one arg-max key per row for the LM-head product's epilogue
+    unsigned long long* lm_keys = nullptr;      // two sets of one arg-max key per row for the LM-head product's epilogue
+    uint32_t lm_epoch = 0;                      // calls launched so far: set (lm_epoch & 1) is in use, the other one clean
     unsigned int* seq_counter = nullptr;
     uint32_t accept_epoch = 0;
     long long part_keys_len = 0;
@@ -278,7 +279,8 @@ int owl_create(owl_ctx** out, int device, const owl_dims* max_dims) {
     if (acc) {
         ctx->part_keys_len = (long long)max_dims->total_nodes * ((max_dims->vocab + kArgmaxChunk - 1) / kArgmaxChunk);
         alloc((void**)&ctx->part_keys, (size_t)ctx->part_keys_len * sizeof(unsigned long long));
-        alloc((void**)&ctx->lm_keys, (size_t)max_dims->total_nodes * sizeof(unsigned long long));
+        alloc((void**)&ctx->lm_keys, 2 * (size_t)max_dims->total_nodes * sizeof(unsigned long long));
+        if (ok) ok = cudaMemset(ctx->lm_keys, 0, 2 * (size_t)max_dims->total_nodes * sizeof(unsigned long long)) == cudaSuccess;
         alloc((void**)&ctx->seq_counter, 2 * (size_t)max_dims->batch * sizeof(unsigned int));
         if (ok) ok = cudaMemset(ctx->seq_counter, 0, 2 * (size_t)max_dims->batch * sizeof(unsigned int)) == cudaSuccess;
     }
@@ -629,23 +631,28 @@ int owl_lm_head_accept(owl_ctx* ctx, const owl_dims* d, int32_t hidden_dim, cons
     if (!ctx->lm_keys || d->batch > ctx->max_dims.batch || d->total_nodes > ctx->max_dims.total_nodes) return OWL_ERR_TOO_LARGE;
     DeviceGuard guard(ctx->device);
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-    // the keys only ever grow (atomicMax): they start from 0, below every real key
-    cudaError_t e = cudaMemsetAsync(ctx->lm_keys, 0, (size_t)d->total_nodes * sizeof(unsigned long long), stream);
-    if (e != cudaSuccess) return cuda_fail(ctx, e, "owl_lm_head_accept");
-    rc = launch_gemm<gemm_path::kEpiArgmax>(ctx, hidden, weight, d->total_nodes, d->vocab, hidden_dim, ctx->lm_keys, nullptr, 0, stream);
+    // The keys only ever grow (atomicMax) and must start from 0, below every real key.  Two sets alternate between
+    // calls: this call's set was cleared, as a whole, by the walk kernel of the call before it (by owl_create for the
+    // first two), and this call's walk kernel clears the other one - no memset in front of the product, which can
+    // then queue up behind whatever kernel precedes it.  The call number moves on only once both kernels are launched.
+    unsigned long long* keys = ctx->lm_keys + (size_t)(ctx->lm_epoch & 1u) * ctx->max_dims.total_nodes;
+    unsigned long long* idle_keys = ctx->lm_keys + (size_t)((ctx->lm_epoch + 1u) & 1u) * ctx->max_dims.total_nodes;
+    rc = launch_gemm<gemm_path::kEpiArgmax>(ctx, hidden, weight, d->total_nodes, d->vocab, hidden_dim, keys, nullptr, 0, stream);
     if (rc != OWL_OK) return rc;
     AcceptParams p{};
     p.draft_tokens = draft_tokens; p.node_offsets = node_offsets; p.tree_parent = tree_parent;
     p.accept_len = accept_len; p.accept_path = accept_path; p.bonus_token = bonus_token; p.node_argmax = node_argmax;
-    p.part_keys = ctx->lm_keys;
+    p.part_keys = keys;
     p.chunks = 1;
     p.status = ctx->status;
     p.batch = d->batch; p.total_nodes = d->total_nodes; p.nodes_uniform = d->total_nodes / d->batch;
     p.max_nodes = d->max_nodes; p.vocab = d->vocab; p.path_stride = d->path_stride;
-    gemm_path::accept_walk_kernel<<<d->batch, kArgmaxThreads, 0, stream>>>(p);
+    launch_dependent(gemm_path::accept_walk_kernel, dim3((unsigned)d->batch), dim3(kArgmaxThreads), stream, p, idle_keys,
+                     ctx->max_dims.total_nodes);
     ++ctx->launches;
-    e = cudaGetLastError();
+    cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(ctx, e, "owl_lm_head_accept launch");
+    ++ctx->lm_epoch;
     return OWL_OK;
 }
 

@@ -99,6 +99,17 @@ def test_lm_head_accept_small(trees, K, V):
     ctx.close()
 
 
+def test_lm_head_accept_calls_of_different_sizes_on_one_context():
+    """The row keys live in two sets that alternate between calls, each cleared as a whole by the call before: a
+    200-row call, an 8-row call, a 200-row call and a 23-row call through one context (two launches each inside
+    the helper, so every set is reused after a larger and after a smaller call) all match the oracle."""
+    ctx = OwlContext(make_dims(batch=8, total_nodes=384, max_nodes=64, vocab=5000))
+    big = [("tree", 64, 8)] * 3 + [("chain", 8)]
+    for k, trees in enumerate([big, [("chain", 8)], big, [("tree", 20, 4), ("chain", 3)]]):
+        _lm_head_case(ctx, 4000 + k, trees, 128, 5000)
+    ctx.close()
+
+
 def test_lm_head_accept_full_vocabulary():
     """The 8B shape's head: hidden 4096, vocabulary 128256 (1002 column tiles over 148 CTAs), a 32-node tree."""
     ctx = OwlContext(make_dims(batch=1, total_nodes=32, max_nodes=32, vocab=W.VOCAB))
