@@ -12,7 +12,7 @@
 
 #include "accept.cuh"
 #include "combine.cuh"
-#include "gemm_umma.cuh"
+#include "gemm_umma_pair.cuh"
 #include "owl_common.cuh"
 #include "spec_loop.cuh"
 #include "verify_attn_umma.cuh"
@@ -185,6 +185,34 @@ static int launch_gemm(owl_ctx* ctx, const void* a, const void* b, int M, int N,
     gemm_path::GemmParams g{};
     g.M = M; g.N = N; g.K = K;
     g.row_blocks = (M + gemm_path::kBM - 1) / gemm_path::kBM;
+    g.status = ctx->status;
+    g.row_key = row_key; g.c = c; g.ldc = ldc;
+    if (g.row_blocks == 2 && ctx->sm_count >= 2 && K % (2 * gemm_path::kBK) == 0) {
+        // 129 to 256 rows: CTA pairs (gemm_umma_pair.cuh).  The columns are dealt out to the pairs as to single CTAs
+        // below; a CTA stages half of a tile's rows of B.
+        const int units = (N + 15) / 16, max_pairs = ctx->sm_count / 2;
+        const int pairs = units < max_pairs ? units : max_pairs;
+        const int per_pair = (units + pairs - 1) / pairs;
+        g.rounds = (per_pair + 15) / 16;
+        g.w_lo = per_pair / g.rounds * 16;
+        g.wide_rounds = per_pair % g.rounds;
+        g.a_bytes = gemm_path::kTileBytes;
+        g.stage_bytes = 2 * (g.a_bytes + (g.w_lo + (g.wide_rounds ? 16 : 0)) / 2 * gemm_path::kBK * 2);   // two k-blocks
+        const int fit = (gemm_path::kSmemLimit - gemm_path::kAuxBytes) / g.stage_bytes;
+        g.stages = fit < gemm_path::kMaxStages ? fit : gemm_path::kMaxStages;
+        CUtensorMap amap, bmap_hi, bmap_lo;
+        const int ra = gemm_path::make_operand_map(ctx->encode, &amap, a, M, K, gemm_path::kBM);
+        int rb = gemm_path::make_operand_map(ctx->encode, &bmap_lo, b, N, K, g.w_lo / 2);
+        if (rb == 0) rb = g.wide_rounds ? gemm_path::make_operand_map(ctx->encode, &bmap_hi, b, N, K, (g.w_lo + 16) / 2) : (bmap_hi = bmap_lo, 0);
+        if (ra != 0 || rb != 0) {
+            snprintf(ctx->err, sizeof ctx->err, "cuTensorMapEncodeTiled failed (%d, %d): operands must be 16-byte aligned", ra, rb);
+            return OWL_ERR_CUDA;
+        }
+        launch_dependent_smem(gemm_path::gemm_umma_pair_kernel<kEpi>, dim3(2u * (unsigned)pairs), dim3(gemm_path::kThreads),
+                              (size_t)(gemm_path::kAuxBytes + g.stages * g.stage_bytes), stream, g, amap, bmap_hi, bmap_lo);
+        ++ctx->launches;
+        return OWL_OK;
+    }
     // every CTA gets the same number of 16-column units, cut into as few tiles as the width limit allows
     const int units = (N + 15) / 16;
     const int grid = units < ctx->sm_count ? units : ctx->sm_count;
@@ -198,8 +226,6 @@ static int launch_gemm(owl_ctx* ctx, const void* a, const void* b, int M, int N,
     g.a_bytes = (g.row_blocks - 1) * gemm_path::kTileBytes + last_rows * gemm_path::kBK * 2;
     g.stage_bytes = g.a_bytes + (g.w_lo + (g.wide_rounds ? 16 : 0)) * gemm_path::kBK * 2;
     g.stages = gemm_path::ring_stages(g.stage_bytes);
-    g.status = ctx->status;
-    g.row_key = row_key; g.c = c; g.ldc = ldc;
     CUtensorMap amap, amap_last, bmap_hi, bmap_lo;
     int ra = gemm_path::make_operand_map(ctx->encode, &amap, a, M, K, gemm_path::kBM);
     if (ra == 0) ra = gemm_path::make_operand_map(ctx->encode, &amap_last, a, M, K, last_rows);
@@ -296,6 +322,10 @@ int owl_create(owl_ctx** out, int device, const owl_dims* max_dims) {
         ok = cudaFuncSetAttribute(gemm_path::gemm_umma_kernel<gemm_path::kEpiArgmax>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                   gemm_path::kSmemLimit) == cudaSuccess &&
              cudaFuncSetAttribute(gemm_path::gemm_umma_kernel<gemm_path::kEpiStore>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  gemm_path::kSmemLimit) == cudaSuccess &&
+             cudaFuncSetAttribute(gemm_path::gemm_umma_pair_kernel<gemm_path::kEpiArgmax>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  gemm_path::kSmemLimit) == cudaSuccess &&
+             cudaFuncSetAttribute(gemm_path::gemm_umma_pair_kernel<gemm_path::kEpiStore>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                   gemm_path::kSmemLimit) == cudaSuccess;
     }
     if (!ok || cudaDeviceSynchronize() != cudaSuccess) {
