@@ -94,6 +94,8 @@ def _lm_head_case(ctx, seed, trees, K, V, plant=0.7):
     ([("tree", 64, 8)] * 2 + [("chain", 2)], 128, 16),              # 130 rows on a CTA pair: one stage per tile, one 16-column tile
     ([("tree", 64, 8)] * 4, 128, 1000),                             # 256 rows on CTA pairs: 63 pairs with a 16-column tile each
     ([("tree", 40, 6)] * 4, 384, 40000),                            # 160 rows on 74 pairs: two rounds (144 + 128 columns), three stages per tile
+    ([("tree", 64, 8)] * 6, 128, 40000),                            # 384 rows: three row blocks, K a multiple of 128
+    ([("tree", 64, 8)] * 4 + [("chain", 1)], 256, 2000),            # 257 rows: one row in the third row block
 ])
 def test_lm_head_accept_small(trees, K, V):
     ctx = OwlContext(make_dims(batch=8, total_nodes=384, max_nodes=64, vocab=V))
@@ -189,6 +191,7 @@ def _cell_case(ctx, seed, M, d_in, d, affine, steps=1):
     (1, 64, 16384, True),           # the widest cell: four columns per thread, two rounds of product tiles
     (256, 128, 4096, False),        # two full row blocks on CTA pairs, store epilogue, four rounds of 224 / 208 columns
     (129, 384, 36, True),           # one row in the second row block; 144 columns in all
+    (300, 256, 512, True),          # three row blocks, store epilogue, K a multiple of 128
 ])
 def test_lstm_cell_small(M, d_in, d, affine):
     ctx = OwlContext(make_dims(batch=1, total_nodes=1, max_nodes=1))
