@@ -217,7 +217,7 @@ static int launch_gemm(owl_ctx* ctx, const void* a, const void* b, int M, int N,
     const int units = (N + 15) / 16;
     const int grid = units < ctx->sm_count ? units : ctx->sm_count;
     const int per_cta = (units + grid - 1) / grid;
-    const int wmax_units = gemm_path::b_boxes(g.row_blocks) * gemm_path::kBN / 16;
+    const int wmax_units = gemm_path::max_tile_width(g.row_blocks) / 16;
     g.rounds = (per_cta + wmax_units - 1) / wmax_units;
     g.w_lo = per_cta / g.rounds * 16;
     g.wide_rounds = per_cta % g.rounds;
