@@ -121,15 +121,17 @@ __device__ __forceinline__ void accept_walk_seq(const AcceptParams& p, const int
         __syncthreads();
         if (i == 0) p.spec_node[b] = s_leaf < kMaxNodes ? s_leaf : -1;
     }
-    if (i == 0) {
+    {
         const int win = kMaxNodes - 1 - (s_win & 0xff);
         const int len = s_win >> 8;
-        p.accept_len[b] = len;
-        p.bonus_token[b] = s_am[win];
         int32_t* path = p.accept_path + (long long)b * p.path_stride;
-        for (int k = len; k < p.path_stride; ++k) path[k] = -1;
-        int k = len - 1;
-        for (int c = win; c >= 0 && k >= 0; c = s_parent[c]) path[k--] = c;
+        for (int k = len + i; k < p.path_stride; k += blockDim.x) path[k] = -1;     // the padding, all threads
+        if (i == 0) {
+            p.accept_len[b] = len;
+            p.bonus_token[b] = s_am[win];
+            int k = len - 1;
+            for (int c = win; c >= 0 && k >= 0; c = s_parent[c]) path[k--] = c;
+        }
     }
 }
 
