@@ -27,8 +27,14 @@ constexpr int kCombineWarps = 8;
 //
 // kGroup: partials fetched per round, 16 or 32.  A unit cut into 17 to 32 pieces (8 units of a 32K context over 148
 // CTAs: 18 or 19) costs a second round of loads with 16, which is a whole memory round trip of a kernel that is
-// all latency; with 32 the registers of a thread double, which costs occupancy where there are rows enough to
-// fill the machine.  The host takes 32 up to 4096 output rows.
+// all latency.  A round's rows go through a warp-private stage in shared memory (16 or 8 KB per warp: 128 or 64 KB
+// per CTA, which is what limits 32 to launches with few rows; the host takes it up to 4096 output rows).
+//
+// The stage is there for the sake of the code's length, not of the data: with the rows in registers the fetch and
+// the fold were two loops unrolled 32 times, some 450 instructions that a warp with one row executes exactly once,
+// at the pace of instruction fetches from L2.  Copied with cp.async in a short rolled loop and folded in another,
+// the same work is two dozen instructions executed from the instruction cache after their first trip (attention +
+// merge call at 32K context 37.5 -> 36.8 us, with 8192 output rows 586 -> 578 us).
 template <bool kFused, int kGroup>
 __global__ void __launch_bounds__(kCombineWarps * 32) combine_sched_kernel(const AttnParams p, const AcceptParams ap) {
     const long long rows = (long long)p.total_nodes * p.num_q_heads;
@@ -45,6 +51,8 @@ __global__ void __launch_bounds__(kCombineWarps * 32) combine_sched_kernel(const
     // The row CTAs are persistent: a warp derives the schedule once and then takes rows first, first + stride, ...
     // (one CTA per eight rows cost a launch of 8192 rows 19 us, most of it the schedule derived 8192 times).
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    extern __shared__ float4 combine_stage[];          // [warps][kGroup][32]: a round's partial rows, warp-private
+    float4* stage = combine_stage + warp * kGroup * 32;
     const long long first = (long long)blockIdx.x * kCombineWarps + warp, stride = (long long)row_ctas * kCombineWarps;
     const bool small = p.batch <= 32;
     WarpSchedule ws{};
@@ -118,13 +126,15 @@ __global__ void __launch_bounds__(kCombineWarps * 32) combine_sched_kernel(const
             const bool have = mine < count;
             const long long prow = base == 0 ? prow_first : row_of(c0 + (have ? mine : 0));
             const float my_lse = have ? __ldcg(p.part_lse + prow) : -INFINITY;
-            float4 v[kGroup];
-#pragma unroll
-            for (int j = 0; j < kGroup; ++j) {
+            const int cnt = count - base < kGroup ? count - base : kGroup;
+            if (base > 0) __syncwarp();                  // the stage's rows of the round before have been folded
+#pragma unroll 1
+            for (int j = 0; j < cnt; ++j) {
                 const long long pj = __shfl_sync(0xffffffffu, prow, j);
-                v[j] = base + j < count ? __ldcg(reinterpret_cast<const float4*>(p.part_o + pj * kHeadDim + lane * 4))
-                                        : make_float4(0.f, 0.f, 0.f, 0.f);
+                const uint32_t dst = (uint32_t)__cvta_generic_to_shared(stage + j * 32 + lane);
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(p.part_o + pj * kHeadDim + lane * 4) : "memory");
             }
+            asm volatile("cp.async.commit_group;" ::: "memory");
             float gmx = my_lse;
 #pragma unroll
             for (int o = kGroup / 2; o > 0; o >>= 1) gmx = fmaxf(gmx, __shfl_xor_sync(0xffffffffu, gmx, o));
@@ -134,13 +144,17 @@ __global__ void __launch_bounds__(kCombineWarps * 32) combine_sched_kernel(const
                 acc.x *= rescale; acc.y *= rescale; acc.z *= rescale; acc.w *= rescale;
                 sum *= rescale;
                 const float w = have ? __expf(my_lse - mx_new) : 0.f;     // -inf partial: weight 0
-#pragma unroll
-                for (int j = 0; j < kGroup; ++j) {
+                asm volatile("cp.async.wait_group 0;" ::: "memory");
+#pragma unroll 1
+                for (int j = 0; j < cnt; ++j) {
                     const float wj = __shfl_sync(0xffffffffu, w, j);
-                    acc.x += wj * v[j].x; acc.y += wj * v[j].y; acc.z += wj * v[j].z; acc.w += wj * v[j].w;
+                    const float4 v = stage[j * 32 + lane];                 // this lane's own copy: no barrier needed
+                    acc.x += wj * v.x; acc.y += wj * v.y; acc.z += wj * v.z; acc.w += wj * v.w;
                     sum += wj;
                 }
                 mx = mx_new;
+            } else {
+                asm volatile("cp.async.wait_group 0;" ::: "memory");
             }
         }
         if (bad_epoch == p.epoch) continue;            // the pass found a bad tree or page in this sequence: no output

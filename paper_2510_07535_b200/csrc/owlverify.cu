@@ -319,6 +319,13 @@ int owl_create(owl_ctx** out, int device, const owl_dims* max_dims) {
         ok = set_umma_smem_attr();
     }
     if (ok) {
+        const int big = kCombineWarps * 32 * 32 * (int)sizeof(float4), small_ = big / 2;
+        ok = cudaFuncSetAttribute(combine_sched_kernel<true, 32>, cudaFuncAttributeMaxDynamicSharedMemorySize, big) == cudaSuccess &&
+             cudaFuncSetAttribute(combine_sched_kernel<false, 32>, cudaFuncAttributeMaxDynamicSharedMemorySize, big) == cudaSuccess &&
+             cudaFuncSetAttribute(combine_sched_kernel<true, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, small_) == cudaSuccess &&
+             cudaFuncSetAttribute(combine_sched_kernel<false, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, small_) == cudaSuccess;
+    }
+    if (ok) {
         ok = cudaFuncSetAttribute(gemm_path::gemm_umma_kernel<gemm_path::kEpiArgmax>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                   gemm_path::kSmemLimit) == cudaSuccess &&
              cudaFuncSetAttribute(gemm_path::gemm_umma_kernel<gemm_path::kEpiStore>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -457,12 +464,13 @@ static int verify_attn_impl(owl_ctx* ctx, const owl_dims* d, const void* q, cons
     ++ctx->launches;
     if (ctx->profiling) cudaEventRecord(ctx->ev[1], stream);
     const bool few_rows = rows <= 4096;      // latency-bound merge: 32 partials per round (see combine.cuh)
+    const size_t stage_bytes = (size_t)kCombineWarps * (few_rows ? 32 : 16) * 32 * sizeof(float4);
     if (ap)
-        launch_dependent(few_rows ? combine_sched_kernel<true, 32> : combine_sched_kernel<true, 16>,
-                         dim3(grid + (unsigned)d->batch), dim3(kCombineWarps * 32), stream, p, *ap);
+        launch_dependent_smem(few_rows ? combine_sched_kernel<true, 32> : combine_sched_kernel<true, 16>,
+                              dim3(grid + (unsigned)d->batch), dim3(kCombineWarps * 32), stage_bytes, stream, p, *ap);
     else
-        launch_dependent(few_rows ? combine_sched_kernel<false, 32> : combine_sched_kernel<false, 16>, dim3(grid),
-                         dim3(kCombineWarps * 32), stream, p, AcceptParams{});
+        launch_dependent_smem(few_rows ? combine_sched_kernel<false, 32> : combine_sched_kernel<false, 16>, dim3(grid),
+                              dim3(kCombineWarps * 32), stage_bytes, stream, p, AcceptParams{});
     ++ctx->launches;
     if (ctx->profiling) { cudaEventRecord(ctx->ev[2], stream); ctx->ev_attn_valid = true; }
     cudaError_t e = cudaGetLastError();
