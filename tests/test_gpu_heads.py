@@ -148,7 +148,7 @@ def test_lm_head_accept_errors():
 
 # ----------------------------------------------------------------------------- drafter cell
 
-def _cell_case(ctx, seed, M, d_in, d, affine, steps=1):
+def _cell_case(ctx, seed, M, d_in, d, affine, steps=1, z_mean=0.0):
     rng = np.random.default_rng(seed)
     hb = _normal_bits(seed, (M, d_in))
     eb = _normal_bits(seed + 1, (M, d))
@@ -157,7 +157,7 @@ def _cell_case(ctx, seed, M, d_in, d, affine, steps=1):
     ln_c = (rng.uniform(0.5, 1.5, d).astype(np.float32), rng.normal(0, 0.2, d).astype(np.float32)) if affine else (None, None)
     ln_z = (rng.uniform(0.5, 1.5, d).astype(np.float32), rng.normal(0, 0.2, d).astype(np.float32)) if affine else (None, None)
     t = lambda a: None if a is None else torch.from_numpy(a).to(DEV)
-    z = rng.standard_normal((M, d)).astype(np.float32) if steps == 1 else np.zeros((M, d), np.float32)
+    z = (z_mean + rng.standard_normal((M, d))).astype(np.float32) if steps == 1 else np.zeros((M, d), np.float32)
     zd = torch.from_numpy(z.copy()).to(DEV)
     hf = torch.zeros((M, d), dtype=torch.float32, device=DEV)
     hb16 = torch.zeros((M, d), dtype=torch.bfloat16, device=DEV)
@@ -196,6 +196,16 @@ def _cell_case(ctx, seed, M, d_in, d, affine, steps=1):
 def test_lstm_cell_small(M, d_in, d, affine):
     ctx = OwlContext(make_dims(batch=1, total_nodes=1, max_nodes=1))
     _cell_case(ctx, 500 + M, M, d_in, d, affine)
+    ctx.close()
+
+
+def test_lstm_cell_state_with_a_large_mean():
+    """z ~ +-300 + N(0, 1): z' = z g^f + ... is of the order of a hundred with a non-zero mean, so the second layer
+    normalisation works far from the origin (the kernel takes its variance about the mean: per-CTA means and sums of
+    squared deviations, combined).  Same tolerance as everywhere; the oracle carries the same z in fp64."""
+    ctx = OwlContext(make_dims(batch=1, total_nodes=1, max_nodes=1))
+    _cell_case(ctx, 950, 3, 128, 4096, True, z_mean=300.0)
+    _cell_case(ctx, 951, 130, 128, 260, False, z_mean=-300.0)
     ctx.close()
 
 
